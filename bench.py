@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-prefix decode-attention step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+One "step" is one pass of the whole hot path over the workload: append one token per candidate (for
+the configurations that sweep appends), prefix pass, suffix pass, merge.  The metric is the unique
+K/V + Q + O (+LSE) bytes of a step divided by its device time, in GB/s.  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_05475_b200 import workload as wl  # noqa: E402
+
+METRIC = "decode_attn_unique_kv_gbs"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------------
+def host_rows(cfg: wl.Config, rows):
+    """Logical K/V histories of the sampled (b, hq) rows, drawn on the host with the workload's
+    distributions (lengths are the workload's own draws)."""
+    prefix_len, suffix_len = wl.draw_lengths(cfg)
+    q_all = wl.draw_q(cfg, 0)
+    out = []
+    for i, (b, hq) in enumerate(rows):
+        j = b // cfg.C
+        n = int(prefix_len[j]) + int(suffix_len[b])
+        k, v = wl.draw_single_head_history(cfg, i, n)
+        out.append((q_all[b, hq], k, v))
+    return out, prefix_len, suffix_len
+
+
+def time_oracle(cfg: wl.Config, n_rows: int, repeats: int = 1):
+    """Times oracle.attend over n_rows sampled rows on the host cores; returns (seconds per repeat list,
+    cores used, bytes-equivalent of the sample in the metric's accounting)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import attention as orc
+    import contextlib
+    try:
+        from threadpoolctl import threadpool_limits
+        blas_one_thread = lambda: threadpool_limits(limits=1)
+    except Exception:  # pragma: no cover
+        blas_one_thread = contextlib.nullcontext
+    rng = np.random.default_rng(12345)
+    rows = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq))) for _ in range(n_rows)]
+    data, prefix_len, suffix_len = host_rows(cfg, rows)
+    cores = max(1, min(os.cpu_count() or 1, n_rows))
+    ub = wl.unique_bytes(cfg, prefix_len, suffix_len)
+    # A whole step is B*Hq rows; the sample's share of the step's unique bytes is n_rows / (B*Hq).
+    sample_bytes = ub["total"] * n_rows / float(cfg.B * cfg.Hq)
+
+    def one(item):
+        q, k, v = item
+        return orc.attend(q, k, v, cfg.scale)[1]
+
+    times = []
+    with blas_one_thread(), ThreadPoolExecutor(max_workers=cores) as ex:
+        for _ in range(repeats):
+            t0 = time.perf_counter()
+            list(ex.map(one, data))
+            times.append(time.perf_counter() - t0)
+    return times, cores, sample_bytes
+
+
+def oracle_sample_rows(cfg: wl.Config) -> int:
+    """Rows whose fp64 attention costs roughly 10-20 s of CPU work in total."""
+    prefix_len, suffix_len = wl.draw_lengths(cfg)
+    mean_n = float(prefix_len.mean() + suffix_len.mean())
+    per_row_s = max(1e-4, mean_n * cfg.d * 1.2e-8)          # ~12 ns per (token, channel) for convert + 2 gemv + exp
+    return int(max(8, min(cfg.B * cfg.Hq, 12.0 / per_row_s)))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg = wl.CONFIGS[args.workload]
+    n_rows = max(8, oracle_sample_rows(cfg) // 4)
+    times, cores, sample_bytes = time_oracle(cfg, n_rows, repeats=args.warmup + args.steps)
+    timed = times[args.warmup:]
+    sec = sum(timed) / len(timed)
+    value = sample_bytes / sec / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": "%d of %d (candidate, head) rows per step" % (n_rows, cfg.B * cfg.Hq)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "%d of %d rows of %s, fp64 numpy, one thread per row" % (n_rows, cfg.B * cfg.Hq, cfg.name)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.idx = device_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2601_05475_b200 import binding as mc
+    from paper_2601_05475_b200.harness import device_append, device_q, make_device_problem
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    mc.lib()  # fail loudly here if the extension is missing
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def measure(name, steps, warmup, want_kernel_split):
+        cfg = wl.CONFIGS[name]
+        appends = cfg.append_steps > 0
+        total_steps = 2 * (steps + warmup) + 8
+        dp = make_device_problem(cfg, headroom_tokens=total_steps + 1 if appends else 1)
+        stream = torch.cuda.current_stream().cuda_stream
+        qs = [device_q(cfg, i) for i in range(4)]
+        kv = [device_append(cfg, i) for i in range(4)] if appends else None
+        len0 = dp.suffix_len.clone()
+        ub0 = wl.unique_bytes(cfg, dp.prefix_len.cpu().numpy(), len0.cpu().numpy())
+        per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+
+        def step(i):
+            if appends:
+                mc.mc_kv_append(dp.layout, kv[i % 4][0], kv[i % 4][1], stream)
+            mc.mc_decode_attn(dp.layout, qs[i % 4], cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes, stream)
+
+        for i in range(warmup):
+            step(i)
+        barrier()
+        sampler = ClockSampler(torch.cuda.current_device())
+        if rank == 0:
+            sampler.start()
+        n0 = mc.mc_launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for i in range(steps):
+            step(warmup + i)
+        ev1.record()
+        barrier()
+        launches = mc.mc_launch_count() - n0
+        clocks = sampler.stop() if rank == 0 else None
+        ms = ev0.elapsed_time(ev1) / steps
+        if mc.mc_get_last_status(dp.layout) != mc.MC_OK:
+            raise RuntimeError("device status word reports an error")
+        # bytes of the average timed step (suffixes grow by one token per step when appending)
+        grow = (warmup + (steps + 1) / 2.0) * cfg.B * per_tok if appends else 0.0
+        step_bytes = ub0["total"] + grow + (2 * cfg.B * cfg.Hkv * cfg.d * cfg.elem_bytes if appends else 0)
+        res = {"ms": ms, "bytes": step_bytes, "launches": launches, "clocks": clocks, "cfg": cfg}
+
+        # end to end through the host-buffer entry point: pinned host q / k_new / v_new in, o / lse out
+        pin = lambda t: t.cpu().pin_memory()
+        hq = [pin(x) for x in qs]
+        hkv = [(pin(a), pin(b)) for a, b in kv] if appends else None
+        ho = torch.empty(dp.o.shape, dtype=dp.o.dtype).pin_memory()
+        hl = torch.empty(dp.lse.shape, dtype=torch.float32).pin_memory()
+        e2e_steps = max(3, min(steps, 10))
+
+        def host_step(i):
+            mc.mc_decode_step_host(dp.layout, hkv[i % 4][0] if appends else None, hkv[i % 4][1] if appends else None,
+                                   hq[i % 4], cfg.scale, ho, hl, dp.ws_ptr, dp.ws_bytes, stream)
+
+        host_step(0)
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            host_step(1 + i)
+        e1.record()
+        barrier()
+        wall_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+        res["e2e_ms"] = max(e0.elapsed_time(e1) / e2e_steps, wall_ms if world == 1 else 0.0)
+        res["h2d"] = hq[0].numel() * hq[0].element_size() + (2 * hkv[0][0].numel() * hkv[0][0].element_size() if appends else 0)
+        res["d2h"] = ho.numel() * ho.element_size() + hl.numel() * 4
+
+        if want_kernel_split:
+            # the dominant kernel alone, on the launching stream, same data
+            g = dp.geom
+            lse_off = (g.rows * g.n_parts * g.head_dim * 4 + 255) // 256 * 256
+            o_ptr, l_ptr = dp.ws_ptr, dp.ws_ptr + lse_off
+            for fn_name, fn in (("suffix", mc.mc_suffix_attn), ("prefix", mc.mc_prefix_attn)):
+                for _ in range(3):
+                    fn(dp.layout, qs[0], cfg.scale, o_ptr, l_ptr, stream)
+                torch.cuda.synchronize()
+                k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                k0.record()
+                for i in range(steps):
+                    fn(dp.layout, qs[i % 4], cfg.scale, o_ptr, l_ptr, stream)
+                k1.record()
+                torch.cuda.synchronize()
+                res[fn_name + "_ms"] = k0.elapsed_time(k1) / steps
+            cur = dp.suffix_len.cpu().numpy().astype(np.int64)
+            res["suffix_bytes"] = float(cur.sum()) * per_tok
+            res["prefix_bytes"] = float(dp.prefix_len.cpu().numpy().astype(np.int64).sum()) * per_tok
+            res["prefix_flops"] = 4.0 * cfg.Hq * cfg.d * float(
+                (dp.prefix_len.cpu().numpy().astype(np.int64) * cfg.C).sum())
+        dp.close()
+        del dp
+        torch.cuda.empty_cache()
+        return res
+
+    main = measure(args.workload, args.steps, args.warmup, True)
+    others = {}
+    if args.all_configs:
+        for name in ("cfg2", "cfg3", "cfg4"):
+            if name != args.workload:
+                others[name] = measure(name, args.steps, args.warmup, True)
+
+    # max over ranks of the step time
+    ms = main["ms"]
+    e2e_ms = main["e2e_ms"]
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        cfg = main["cfg"]
+        peaks, peak_kind = measured_peaks()
+        peak = float(peaks["hbm_gbs"])
+        value = world * main["bytes"] / (ms * 1e-3) / 1e9
+        suffix_gbs = main["suffix_bytes"] / (main["suffix_ms"] * 1e-3) / 1e9
+
+        def summary(r):
+            gbs = r["bytes"] / (r["ms"] * 1e-3) / 1e9
+            out = {"gbs": round(gbs, 1), "frac_of_8tbs": round(gbs / NOMINAL_HBM_GBS, 4), "ms_per_step": round(r["ms"], 5),
+                   "candidate_tokens_per_s": round(r["cfg"].B / (r["ms"] * 1e-3), 1)}
+            if "suffix_ms" in r:
+                out["suffix_ms"] = round(r["suffix_ms"], 5)
+                out["suffix_gbs"] = round(r["suffix_bytes"] / (r["suffix_ms"] * 1e-3) / 1e9, 1)
+                out["prefix_ms"] = round(r["prefix_ms"], 5)
+                out["prefix_tflops"] = round(r["prefix_flops"] / (r["prefix_ms"] * 1e-3) / 1e12, 2)
+            return out
+
+        n_rows = oracle_sample_rows(cfg)
+        times, cores, sample_bytes = time_oracle(cfg, n_rows, repeats=1)
+        cpu_value = sample_bytes / times[0] / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "groups": cfg.G, "candidates_per_group": cfg.C, "q_heads": cfg.Hq,
+                       "kv_heads": cfg.Hkv, "head_dim": cfg.d, "page_tokens": wl.PAGE,
+                       "step": ("append + " if cfg.append_steps else "") + "prefix + suffix + merge",
+                       "bytes_per_step": main["bytes"], "l2": "inputs larger than L2 (no flush needed)",
+                       "multi_gpu": "replicas only"},
+            "frac_of_8tbs": value / world / NOMINAL_HBM_GBS,
+            "candidate_tokens_per_s": world * cfg.B / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel<suffix>", "achieved": suffix_gbs, "peak": peak,
+                         "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": suffix_gbs / peak,
+                         "frac_of_8tbs": suffix_gbs / NOMINAL_HBM_GBS, "traffic": None,
+                         "kernel_ms": main["suffix_ms"], "algorithmic_bytes": main["suffix_bytes"]},
+            "prefix_pass": {"ms": main["prefix_ms"], "tflops": main["prefix_flops"] / (main["prefix_ms"] * 1e-3) / 1e12,
+                            "bf16_peak_tflops": peaks.get("bf16_tflops")},
+            "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "%d of %d (candidate, head) rows of %s, fp64 numpy, one thread per row"
+                                       % (n_rows, cfg.B * cfg.Hq, cfg.name)},
+            "e2e": {"value": world * main["bytes"] / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": main["h2d"], "d2h_bytes_per_step": main["d2h"], "ms_per_step": e2e_ms},
+            "gpu_launches": int(main["launches"]),
+            "clocks": main["clocks"],
+            "per_config": {**{cfg.name: summary(main)}, **{k: summary(v) for k, v in others.items()}},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg4", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
+                    help="time only --workload (default: also cfg2/cfg3/cfg4 summaries under per_config)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

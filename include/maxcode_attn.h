@@ -1,0 +1,165 @@
+/*
+ * maxcode_attn.h - C ABI of the shared-prefix grouped-query decode-attention library (B200, sm_100a).
+ *
+ * Operation.  One decode step for B candidate rollouts organised in G prompt groups.  All candidates of
+ * a group share the group's prompt (the "prefix"); each candidate has a private continuation (the
+ * "suffix").  This is the workload of the max-reward search of Section 2.2 ("Max-Reward Search": k
+ * candidate actions are sampled from one state s_i) with the budgets of Section 3.1 ("Experimental
+ * Setup": K = 8 candidates x depth 8; flat sampling with n = 64).  For candidate b (group j), query
+ * head hq and its kv head h = hq / (Hq / Hkv):
+ *
+ *     K    = concat(Kprefix_j[0:P_j, h], Ksuffix_b[0:s_b, h])          (V likewise)
+ *     z_t  = scale * <q[b, hq], K_t>
+ *     lse  = log sum_t exp(z_t)                  natural logarithm
+ *     o    = sum_t exp(z_t - lse) * V_t
+ *
+ * The library computes this as three passes: a prefix pass (each group's prefix is attended by the
+ * stacked queries of all its candidates), a suffix pass (each candidate's private tokens, split into
+ * token chunks) and a log-sum-exp merge of the partial results.
+ *
+ * Memory layout (all DEVICE memory, owned by the caller, borrowed by the layout object):
+ *   k_pool, v_pool  [num_pages][Hkv][16][d]   elements of `dtype`; 16-byte aligned.  One (page, kv head)
+ *                                              slab is 16*d contiguous elements.
+ *   prefix_pages    int32 [G][max_prefix_pages]   physical page ids of group j's prefix, in token order
+ *   prefix_len      int32 [G]                     tokens (the last page may be partially filled)
+ *   suffix_pages    int32 [B][max_suffix_pages]   physical page ids of candidate b's suffix
+ *   suffix_len      int32 [B]                     tokens; read on the device at every call, advanced
+ *                                                 by mc_kv_append
+ *   group_offsets   int32 [G+1]                   candidates group_offsets[j] .. group_offsets[j+1]-1
+ *                                                 belong to group j (contiguous in b)
+ *   q               [B][Hq][d] `dtype`            o  [B][Hq][d] `dtype`        lse  [B][Hq] float
+ * Page-table entries beyond a sequence's pages are never dereferenced.  Slots of a page beyond the
+ * sequence length may hold any finite values.  A page id outside [0, num_pages) makes the kernels skip
+ * that page and latch MC_ERR_INVALID_ARG in the device status word (see mc_get_last_status).
+ *
+ * Partial results ("parts").  rows = B*Hq, row = b*Hq + hq.  Each row has n_parts slots:
+ *   parts [0, n_prefix_parts)            prefix splits of prefix_part_tokens tokens each
+ *   parts [n_prefix_parts, n_parts)      suffix chunks of suffix_part_tokens tokens each
+ *   o_part   float [rows][n_parts][d]    normalised partial output of that token range
+ *   lse_part float [rows][n_parts]       its log-sum-exp; -inf marks an empty part (o_part undefined)
+ *
+ * Conventions.  All hot calls (append, prefix, suffix, merge, decode) are asynchronous on `stream`
+ * (a cudaStream_t passed as void*; NULL is the default stream), allocate nothing and do not
+ * synchronise.  Errors detectable on the host are returned immediately; conditions detected on the
+ * device are latched in a status word.  A layout handle is not thread-safe; distinct handles are
+ * independent.  No entry point throws.
+ */
+#ifndef MAXCODE_ATTN_H_
+#define MAXCODE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MC_OK = 0,
+  MC_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, inconsistent sizes, bad page id, full suffix */
+  MC_ERR_UNSUPPORTED = 2,        /* dtype / head_dim / page_size / head ratio outside the supported set */
+  MC_ERR_OUT_OF_MEMORY = 3,
+  MC_ERR_WORKSPACE_TOO_SMALL = 4,
+  MC_ERR_CUDA = 5,               /* a CUDA runtime call failed */
+  MC_ERR_TIMEOUT = 6             /* a bounded device-side wait gave up */
+} mc_status_t;
+
+typedef enum { MC_F32 = 0, MC_BF16 = 1 } mc_dtype_t;
+
+typedef struct mc_kv_layout mc_kv_layout_t;   /* opaque, owned by the library */
+
+typedef struct {
+  int32_t num_groups;            /* G >= 1 */
+  int32_t batch;                 /* B >= 1, total candidates */
+  int32_t num_q_heads;           /* Hq, a multiple of Hkv */
+  int32_t num_kv_heads;          /* Hkv */
+  int32_t head_dim;              /* d: 64 or 128 */
+  int32_t page_size;             /* must be 16 */
+  int32_t num_pages;             /* pages in each pool */
+  int32_t max_prefix_pages;      /* row stride of prefix_pages */
+  int32_t max_suffix_pages;      /* row stride of suffix_pages */
+  int32_t dtype;                 /* mc_dtype_t */
+  void *k_pool, *v_pool;         /* device */
+  const int32_t *group_offsets;  /* device, [G+1] */
+  const int32_t *prefix_pages;   /* device, [G][max_prefix_pages] */
+  const int32_t *prefix_len;     /* device, [G] */
+  const int32_t *suffix_pages;   /* device, [B][max_suffix_pages] */
+  int32_t *suffix_len;           /* device, [B]; mc_kv_append increments it */
+} mc_kv_layout_desc_t;
+
+typedef struct {
+  int32_t rows;                  /* B*Hq */
+  int32_t n_parts;               /* part slots per row */
+  int32_t n_prefix_parts;
+  int32_t prefix_part_tokens;    /* tokens per prefix split (multiple of 16) */
+  int32_t suffix_part_tokens;    /* tokens per suffix chunk (multiple of 16) */
+  int32_t head_dim;
+} mc_part_geometry_t;
+
+/* Builds the layout object (step 1 of the path, the paged-KV layout): validates the descriptor, fixes
+ * the part geometry from the table strides and allocates the handle's small device state (status word).
+ * May synchronise the device.  Pointers in `desc` are borrowed and must outlive the handle.
+ * Returns MC_ERR_INVALID_ARG / MC_ERR_UNSUPPORTED / MC_ERR_OUT_OF_MEMORY / MC_ERR_CUDA on failure
+ * (*out is then NULL). */
+mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *desc, mc_kv_layout_t **out);
+
+/* Frees the handle and its device state.  NULL is accepted. */
+mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout);
+
+/* Debug aid: checks on the device that group_offsets is increasing and ends at B, that lengths fit the
+ * table strides, that every referenced page id lies in [0, num_pages) and that no page is referenced
+ * twice.  Synchronises `stream`.  `scratch` is device memory of at least num_pages*4 bytes. */
+mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t scratch_bytes, void *stream);
+
+/* Part geometry chosen at create time (needed to size and index o_part / lse_part). */
+mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry_t *out);
+
+/* Bytes of device workspace that mc_decode_attn and mc_decode_step_host need (partials + staging). */
+size_t mc_workspace_bytes(const mc_kv_layout_t *layout);
+
+/* Appends one token per candidate: writes k_new/v_new [B][Hkv][d] (device, `dtype`) into slot
+ * suffix_len[b] % 16 of page suffix_pages[b][suffix_len[b] / 16], then increments suffix_len[b], all on
+ * the device.  A candidate whose page row is full is left unchanged and MC_ERR_INVALID_ARG is latched. */
+mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *stream);
+
+/* Prefix pass: for every group and kv head, the stacked queries of all the group's candidates attend
+ * to the group's prefix; writes parts [0, n_prefix_parts) of every row.  q: device [B][Hq][d]. */
+mc_status_t mc_prefix_attn(mc_kv_layout_t *layout, const void *q, float scale,
+                           float *o_part, float *lse_part, void *stream);
+
+/* Suffix pass: every candidate attends to its private suffix, chunk by chunk; writes parts
+ * [n_prefix_parts, n_parts) of every row. */
+mc_status_t mc_suffix_attn(mc_kv_layout_t *layout, const void *q, float scale,
+                           float *o_part, float *lse_part, void *stream);
+
+/* Log-sum-exp merge over the n_parts slots of every row:  m = max_i lse_i, w_i = exp(lse_i - m),
+ * o = sum_i w_i o_i / sum_i w_i, lse = m + log sum_i w_i.  Parts with lse = -inf are skipped; a row with
+ * no non-empty part gets o = 0, lse = -inf.  o: device [B][Hq][d] `dtype`; lse: device [B][Hq] float. */
+mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const float *lse_part,
+                         void *o, float *lse, void *stream);
+
+/* The whole step: prefix pass, suffix pass, merge.  `ws` is device memory of at least
+ * mc_workspace_bytes(layout) bytes, 256-byte aligned (else MC_ERR_WORKSPACE_TOO_SMALL / INVALID_ARG). */
+mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale,
+                           void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
+
+/* Same step for a caller that keeps its per-step tensors on the HOST: copies q (and, if k_new/v_new are
+ * non-NULL, the appended token) host->device into the workspace, appends, runs mc_decode_attn, copies o
+ * and lse device->host and synchronises `stream`.  Host pointers should be pinned for the copies to be
+ * asynchronous.  The KV pools stay resident on the device. */
+mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, const void *v_new_host,
+                                const void *q_host, float scale, void *o_host, float *lse_host,
+                                void *ws, size_t ws_bytes, void *stream);
+
+/* Reads and clears the device status word (synchronises `stream`): MC_OK, or the first latched error. */
+mc_status_t mc_get_last_status(mc_kv_layout_t *layout, void *stream);
+
+/* Kernel launches issued by this library since it was loaded (all handles, all threads). */
+uint64_t mc_launch_count(void);
+
+const char *mc_status_string(mc_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAXCODE_ATTN_H_ */

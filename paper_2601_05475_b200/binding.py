@@ -1,0 +1,152 @@
+"""ctypes binding of the C-ABI library (include/maxcode_attn.h): same names, argument marshalling only.
+
+Device buffers are torch tensors (torch is used for device memory and streams only); every entry point
+takes raw device pointers.  There is no fallback: if the shared library is missing or fails to load,
+`lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_float, c_int32, c_size_t, c_uint64, c_void_p
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmaxcode_attn.so")
+_lib = None
+
+MC_OK, MC_ERR_INVALID_ARG, MC_ERR_UNSUPPORTED, MC_ERR_OUT_OF_MEMORY, MC_ERR_WORKSPACE_TOO_SMALL, MC_ERR_CUDA, \
+    MC_ERR_TIMEOUT = range(7)
+MC_F32, MC_BF16 = 0, 1
+
+
+class LayoutDesc(ctypes.Structure):
+    _fields_ = [(n, c_int32) for n in ("num_groups", "batch", "num_q_heads", "num_kv_heads", "head_dim", "page_size",
+                                       "num_pages", "max_prefix_pages", "max_suffix_pages", "dtype")] + \
+               [(n, c_void_p) for n in ("k_pool", "v_pool", "group_offsets", "prefix_pages", "prefix_len",
+                                        "suffix_pages", "suffix_len")]
+
+
+class PartGeometry(ctypes.Structure):
+    _fields_ = [(n, c_int32) for n in ("rows", "n_parts", "n_prefix_parts", "prefix_part_tokens",
+                                       "suffix_part_tokens", "head_dim")]
+
+
+EXPORTS = {
+    "mc_kv_layout_create": (c_int32, [POINTER(LayoutDesc), POINTER(c_void_p)]),
+    "mc_kv_layout_destroy": (c_int32, [c_void_p]),
+    "mc_kv_layout_validate": (c_int32, [c_void_p, c_void_p, c_size_t, c_void_p]),
+    "mc_kv_layout_geometry": (c_int32, [c_void_p, POINTER(PartGeometry)]),
+    "mc_workspace_bytes": (c_size_t, [c_void_p]),
+    "mc_kv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "mc_prefix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
+    "mc_suffix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
+    "mc_merge_lse": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "mc_decode_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "mc_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p,
+                                      c_void_p, c_size_t, c_void_p]),
+    "mc_get_last_status": (c_int32, [c_void_p, c_void_p]),
+    "mc_launch_count": (c_uint64, []),
+    "mc_status_string": (c_char_p, [c_int32]),
+}
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built (python -m paper_2601_05475_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("%s is missing: build it with `python -m paper_2601_05475_b200.build`; "
+                               "there is no fallback path" % _LIB_PATH)
+        l = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(l, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = l
+    return _lib
+
+
+class McError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, mc_status_string(status), status))
+
+
+def _check(status: int, where: str) -> None:
+    if status != MC_OK:
+        raise McError(status, where)
+
+
+def _ptr(x) -> int:
+    """Raw address of a torch tensor (device or host), an int, or None."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def mc_status_string(status: int) -> str:
+    return lib().mc_status_string(status).decode()
+
+
+def mc_launch_count() -> int:
+    return int(lib().mc_launch_count())
+
+
+def mc_kv_layout_create(desc: LayoutDesc) -> int:
+    h = c_void_p()
+    _check(lib().mc_kv_layout_create(byref(desc), byref(h)), "mc_kv_layout_create")
+    return h.value
+
+
+def mc_kv_layout_destroy(layout: int) -> None:
+    _check(lib().mc_kv_layout_destroy(layout), "mc_kv_layout_destroy")
+
+
+def mc_kv_layout_geometry(layout: int) -> PartGeometry:
+    g = PartGeometry()
+    _check(lib().mc_kv_layout_geometry(layout, byref(g)), "mc_kv_layout_geometry")
+    return g
+
+
+def mc_workspace_bytes(layout: int) -> int:
+    return int(lib().mc_workspace_bytes(layout))
+
+
+def mc_kv_layout_validate(layout: int, scratch, scratch_bytes: int, stream: int = 0) -> int:
+    return lib().mc_kv_layout_validate(layout, _ptr(scratch), scratch_bytes, stream)
+
+
+def mc_kv_append(layout: int, k_new, v_new, stream: int = 0) -> None:
+    _check(lib().mc_kv_append(layout, _ptr(k_new), _ptr(v_new), stream), "mc_kv_append")
+
+
+def mc_prefix_attn(layout: int, q, scale: float, o_part, lse_part, stream: int = 0) -> None:
+    _check(lib().mc_prefix_attn(layout, _ptr(q), scale, _ptr(o_part), _ptr(lse_part), stream), "mc_prefix_attn")
+
+
+def mc_suffix_attn(layout: int, q, scale: float, o_part, lse_part, stream: int = 0) -> None:
+    _check(lib().mc_suffix_attn(layout, _ptr(q), scale, _ptr(o_part), _ptr(lse_part), stream), "mc_suffix_attn")
+
+
+def mc_merge_lse(layout: int, o_part, lse_part, o, lse, stream: int = 0) -> None:
+    _check(lib().mc_merge_lse(layout, _ptr(o_part), _ptr(lse_part), _ptr(o), _ptr(lse), stream), "mc_merge_lse")
+
+
+def mc_decode_attn(layout: int, q, scale: float, o, lse, ws, ws_bytes: int, stream: int = 0) -> None:
+    _check(lib().mc_decode_attn(layout, _ptr(q), scale, _ptr(o), _ptr(lse), _ptr(ws), ws_bytes, stream),
+           "mc_decode_attn")
+
+
+def mc_decode_step_host(layout: int, k_new_host, v_new_host, q_host, scale: float, o_host, lse_host, ws,
+                        ws_bytes: int, stream: int = 0) -> None:
+    _check(lib().mc_decode_step_host(layout, _ptr(k_new_host), _ptr(v_new_host), _ptr(q_host), scale,
+                                     _ptr(o_host), _ptr(lse_host), _ptr(ws), ws_bytes, stream),
+           "mc_decode_step_host")
+
+
+def mc_get_last_status(layout: int, stream: int = 0) -> int:
+    return lib().mc_get_last_status(layout, stream)

@@ -1,0 +1,333 @@
+// C-ABI entry points: argument checking, layout object, append, validation, status word, and the
+// drivers that enqueue the passes.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "mc_internal.cuh"
+
+namespace mc {
+
+struct Layout {
+  mc_kv_layout_desc_t desc;
+  Params p;
+  int32_t *dev_status;   // device int
+  int32_t *host_status;  // pinned host int, target of the status read-back
+  size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
+  bool use_mma;
+};
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+mc_status_t check_launch() { return cudaPeekAtLastError() == cudaSuccess ? MC_OK : MC_ERR_CUDA; }
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+int pow2_floor(int x) { int r = 1; while (r * 2 <= x) r *= 2; return r; }
+int env_int(const char *name, int dflt) {
+  const char *s = std::getenv(name);
+  if (!s || !*s) return dflt;
+  int v = std::atoi(s);
+  return v > 0 ? v : dflt;
+}
+
+// ------------------------------------------------------------------------------------------------
+// append: one block per candidate copies the new token's K and V rows of every kv head
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__restrict__ k_new,
+                                                     const uint4 *__restrict__ v_new, int32_t *suffix_len,
+                                                     int elem_bytes) {
+  const int b = blockIdx.x;
+  const int s = suffix_len[b];
+  const int pg = s >> 4;
+  int page = -1;
+  if (s >= 0 && pg < p.max_sp) page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + pg);
+  if ((unsigned)page >= (unsigned)p.num_pages) {  // row full, or a bad table entry: leave the candidate alone
+    if (threadIdx.x == 0) latch(p, kDevBadPage);
+    return;
+  }
+  const int row_vec = p.d * elem_bytes / 16;  // uint4 per (token, kv head) row
+  const int n_vec = p.Hkv * row_vec;
+  uint4 *kp = reinterpret_cast<uint4 *>(const_cast<void *>(p.k_pool));
+  uint4 *vp = reinterpret_cast<uint4 *>(const_cast<void *>(p.v_pool));
+  for (int i = threadIdx.x; i < 2 * n_vec; i += blockDim.x) {
+    const int which = i >= n_vec, j = which ? i - n_vec : i;
+    const int h = j / row_vec, c = j % row_vec;
+    const size_t dst = (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + c;
+    const size_t src = ((size_t)b * p.Hkv + h) * row_vec + c;
+    if (which) vp[dst] = v_new[src]; else kp[dst] = k_new[src];
+  }
+  __syncthreads();  // every thread has read s and issued its stores before the length moves
+  if (threadIdx.x == 0) suffix_len[b] = s + 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// validation
+// ------------------------------------------------------------------------------------------------
+__global__ void validate_kernel(Params p, int32_t *refs) {
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  if (tid == 0) {
+    if (__ldg(p.group_offsets) != 0 || __ldg(p.group_offsets + p.G) != p.B) latch(p, kDevBadPage);
+    for (int j = 0; j < p.G; ++j)
+      if (__ldg(p.group_offsets + j + 1) < __ldg(p.group_offsets + j)) latch(p, kDevBadPage);
+  }
+  const long long np = (long long)p.G * p.max_pp, ns = (long long)p.B * p.max_sp;
+  for (long long i = tid; i < np + ns; i += nth) {
+    int page, used;
+    if (i < np) {
+      const int j = (int)(i / p.max_pp), k = (int)(i % p.max_pp);
+      const int len = __ldg(p.prefix_len + j);
+      if (k == 0 && (len < 0 || len > p.max_pp * kPage)) latch(p, kDevBadPage);
+      used = k < (len + kPage - 1) / kPage;
+      page = __ldg(p.prefix_pages + i);
+    } else {
+      const long long r = i - np;
+      const int b = (int)(r / p.max_sp), k = (int)(r % p.max_sp);
+      const int len = __ldg(p.suffix_len + b);
+      if (k == 0 && (len < 0 || len > p.max_sp * kPage)) latch(p, kDevBadPage);
+      // pages pre-assigned for future appends count as referenced when their id is non-negative
+      page = __ldg(p.suffix_pages + r);
+      used = k < (len + kPage - 1) / kPage || page >= 0;
+    }
+    if (!used) continue;
+    if ((unsigned)page >= (unsigned)p.num_pages) { latch(p, kDevBadPage); continue; }
+    if (atomicAdd(refs + page, 1) != 0) latch(p, kDevBadPage);
+  }
+}
+
+mc_status_t check_q(const Layout *L, const void *q) {
+  if (!L || !q) return MC_ERR_INVALID_ARG;
+  if (!aligned16(q)) return MC_ERR_INVALID_ARG;
+  return MC_OK;
+}
+
+mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
+                     cudaStream_t st) {
+  if (L->use_mma) return launch_mma(L->p, mode, q, scale, o_part, lse_part, st);
+  return launch_fma(L->p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
+}
+
+}  // namespace
+}  // namespace mc
+
+using mc::Layout;
+
+extern "C" {
+
+const char *mc_status_string(mc_status_t s) {
+  switch (s) {
+    case MC_OK: return "ok";
+    case MC_ERR_INVALID_ARG: return "invalid argument";
+    case MC_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MC_ERR_OUT_OF_MEMORY: return "out of memory";
+    case MC_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MC_ERR_CUDA: return "CUDA runtime error";
+    case MC_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+uint64_t mc_launch_count(void) { return mc::g_launches.load(std::memory_order_relaxed); }
+
+mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **out) {
+  if (out) *out = nullptr;
+  if (!d || !out) return MC_ERR_INVALID_ARG;
+  if (d->num_groups < 1 || d->batch < 1 || d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_pages < 1 ||
+      d->max_prefix_pages < 1 || d->max_suffix_pages < 1 || d->batch < d->num_groups)
+    return MC_ERR_INVALID_ARG;
+  if (d->num_q_heads % d->num_kv_heads != 0) return MC_ERR_INVALID_ARG;
+  if (!d->k_pool || !d->v_pool || !d->group_offsets || !d->prefix_pages || !d->prefix_len || !d->suffix_pages ||
+      !d->suffix_len)
+    return MC_ERR_INVALID_ARG;
+  if (!mc::aligned16(d->k_pool) || !mc::aligned16(d->v_pool)) return MC_ERR_INVALID_ARG;
+  if (d->page_size != mc::kPage) return MC_ERR_UNSUPPORTED;
+  if (d->dtype != MC_F32 && d->dtype != MC_BF16) return MC_ERR_UNSUPPORTED;
+  if (d->head_dim != 64 && d->head_dim != 128) return MC_ERR_UNSUPPORTED;
+  if ((long long)d->batch * d->num_q_heads > (1ll << 30)) return MC_ERR_UNSUPPORTED;
+
+  Layout *L = new (std::nothrow) Layout();
+  if (!L) return MC_ERR_OUT_OF_MEMORY;
+  L->desc = *d;
+  mc::Params &p = L->p;
+  p.k_pool = d->k_pool; p.v_pool = d->v_pool;
+  p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
+  p.suffix_pages = d->suffix_pages; p.suffix_len = d->suffix_len;
+  p.G = d->num_groups; p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.d = d->head_dim;
+  p.g = d->num_q_heads / d->num_kv_heads;
+  p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
+
+  // Part geometry from the table strides (the lengths themselves live on the device and may grow).
+  const int max_p = d->max_prefix_pages * mc::kPage, max_s = d->max_suffix_pages * mc::kPage;
+  int tp = mc::pow2_floor(max_p / 8 > 256 ? max_p / 8 : 256);
+  if (tp > 4096) tp = 4096;
+  int ts = mc::pow2_floor(max_s / 16 > 256 ? max_s / 16 : 256);
+  if (ts > 4096) ts = 4096;
+  tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
+  ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
+  if (tp < mc::kPage) tp = mc::kPage;
+  if (ts < mc::kPage) ts = mc::kPage;
+  p.prefix_part_tokens = tp;
+  p.suffix_part_tokens = ts;
+  p.n_prefix_parts = (max_p + tp - 1) / tp;
+  p.n_parts = p.n_prefix_parts + (max_s + ts - 1) / ts;
+  L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
+
+  const size_t rows = (size_t)p.B * p.Hq, e = d->dtype == MC_F32 ? 4 : 2;
+  L->o_part_bytes = mc::align_up(rows * p.n_parts * p.d * sizeof(float), 256);
+  L->lse_part_bytes = mc::align_up(rows * p.n_parts * sizeof(float), 256);
+  size_t off = L->o_part_bytes + L->lse_part_bytes;
+  const size_t qb = mc::align_up(rows * p.d * e, 256), kvb = mc::align_up((size_t)p.B * p.Hkv * p.d * e, 256);
+  const size_t sizes[5] = {qb, kvb, kvb, qb, mc::align_up(rows * sizeof(float), 256)};  // q, k_new, v_new, o, lse
+  for (int i = 0; i < 5; ++i) { L->staging_off[i] = off; off += sizes[i]; }
+  L->ws_bytes = off;
+
+  if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) { delete L; return MC_ERR_OUT_OF_MEMORY; }
+  if (cudaMemset(L->dev_status, 0, 256) != cudaSuccess ||
+      cudaMallocHost(&L->host_status, sizeof(int32_t)) != cudaSuccess) {
+    cudaFree(L->dev_status);
+    delete L;
+    return MC_ERR_CUDA;
+  }
+  *L->host_status = 0;
+  p.status = L->dev_status;
+  *out = reinterpret_cast<mc_kv_layout_t *>(L);
+  return MC_OK;
+}
+
+mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L) return MC_OK;
+  cudaFree(L->dev_status);
+  cudaFreeHost(L->host_status);
+  delete L;
+  return MC_OK;
+}
+
+mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry_t *g) {
+  const Layout *L = reinterpret_cast<const Layout *>(layout);
+  if (!L || !g) return MC_ERR_INVALID_ARG;
+  g->rows = L->p.B * L->p.Hq;
+  g->n_parts = L->p.n_parts;
+  g->n_prefix_parts = L->p.n_prefix_parts;
+  g->prefix_part_tokens = L->p.prefix_part_tokens;
+  g->suffix_part_tokens = L->p.suffix_part_tokens;
+  g->head_dim = L->p.d;
+  return MC_OK;
+}
+
+size_t mc_workspace_bytes(const mc_kv_layout_t *layout) {
+  const Layout *L = reinterpret_cast<const Layout *>(layout);
+  return L ? L->ws_bytes : 0;
+}
+
+mc_status_t mc_get_last_status(mc_kv_layout_t *layout, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L) return MC_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(L->host_status, L->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(L->dev_status, 0, sizeof(int32_t), st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return MC_ERR_CUDA;
+  const int32_t v = *L->host_status;
+  return v >= MC_OK && v <= MC_ERR_TIMEOUT ? static_cast<mc_status_t>(v) : MC_ERR_CUDA;
+}
+
+mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t scratch_bytes, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !scratch) return MC_ERR_INVALID_ARG;
+  if (scratch_bytes < (size_t)L->p.num_pages * sizeof(int32_t)) return MC_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(scratch, 0, (size_t)L->p.num_pages * sizeof(int32_t), st) != cudaSuccess) return MC_ERR_CUDA;
+  mc::validate_kernel<<<148, 256, 0, st>>>(L->p, reinterpret_cast<int32_t *>(scratch));
+  mc::count_launch();
+  if (mc::check_launch() != MC_OK) return MC_ERR_CUDA;
+  return mc_get_last_status(layout, stream);
+}
+
+mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new)) return MC_ERR_INVALID_ARG;
+  const int e = L->desc.dtype == MC_F32 ? 4 : 2;
+  mc::append_kernel<<<L->p.B, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      L->p, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), L->desc.suffix_len, e);
+  mc::count_launch();
+  return mc::check_launch();
+}
+
+mc_status_t mc_prefix_attn(mc_kv_layout_t *layout, const void *q, float scale, float *o_part, float *lse_part,
+                           void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  mc_status_t s = mc::check_q(L, q);
+  if (s != MC_OK) return s;
+  if (!o_part || !lse_part || !mc::aligned16(o_part)) return MC_ERR_INVALID_ARG;
+  return mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, reinterpret_cast<cudaStream_t>(stream));
+}
+
+mc_status_t mc_suffix_attn(mc_kv_layout_t *layout, const void *q, float scale, float *o_part, float *lse_part,
+                           void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  mc_status_t s = mc::check_q(L, q);
+  if (s != MC_OK) return s;
+  if (!o_part || !lse_part || !mc::aligned16(o_part)) return MC_ERR_INVALID_ARG;
+  return mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, reinterpret_cast<cudaStream_t>(stream));
+}
+
+mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const float *lse_part, void *o, float *lse,
+                         void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !o_part || !lse_part || !o || !lse || !mc::aligned16(o_part) || !mc::aligned16(o))
+    return MC_ERR_INVALID_ARG;
+  return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, reinterpret_cast<cudaStream_t>(stream));
+}
+
+mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, void *o, float *lse, void *ws,
+                           size_t ws_bytes, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  mc_status_t s = mc::check_q(L, q);
+  if (s != MC_OK) return s;
+  if (!o || !lse || !ws || !mc::aligned16(o)) return MC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MC_ERR_INVALID_ARG;
+  if (ws_bytes < L->ws_bytes) return MC_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  float *o_part = reinterpret_cast<float *>(ws);
+  float *lse_part = reinterpret_cast<float *>(static_cast<char *>(ws) + L->o_part_bytes);
+  if ((s = mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+  if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+  return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
+}
+
+mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, const void *v_new_host,
+                                const void *q_host, float scale, void *o_host, float *lse_host, void *ws,
+                                size_t ws_bytes, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !q_host || !o_host || !lse_host || !ws) return MC_ERR_INVALID_ARG;
+  if ((k_new_host == nullptr) != (v_new_host == nullptr)) return MC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MC_ERR_INVALID_ARG;
+  if (ws_bytes < L->ws_bytes) return MC_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char *base = static_cast<char *>(ws);
+  const size_t e = L->desc.dtype == MC_F32 ? 4 : 2, rows = (size_t)L->p.B * L->p.Hq;
+  const size_t q_bytes = rows * L->p.d * e, kv_bytes = (size_t)L->p.B * L->p.Hkv * L->p.d * e;
+  void *q_dev = base + L->staging_off[0], *k_dev = base + L->staging_off[1], *v_dev = base + L->staging_off[2];
+  void *o_dev = base + L->staging_off[3];
+  float *lse_dev = reinterpret_cast<float *>(base + L->staging_off[4]);
+  if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MC_ERR_CUDA;
+  mc_status_t s;
+  if (k_new_host) {
+    if (cudaMemcpyAsync(k_dev, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(v_dev, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return MC_ERR_CUDA;
+    if ((s = mc_kv_append(layout, k_dev, v_dev, stream)) != MC_OK) return s;
+  }
+  if ((s = mc_decode_attn(layout, q_dev, scale, o_dev, lse_dev, ws, ws_bytes, stream)) != MC_OK) return s;
+  if (cudaMemcpyAsync(o_host, o_dev, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(lse_host, lse_dev, rows * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return MC_ERR_CUDA;
+  return MC_OK;
+}
+
+}  // extern "C"

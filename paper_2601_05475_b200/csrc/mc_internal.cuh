@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "maxcode_attn.h"
+
+namespace mc {
+
+constexpr int kPage = 16;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// status bits latched on the device (first non-zero value wins through atomicCAS)
+constexpr int kDevBadPage = MC_ERR_INVALID_ARG;
+constexpr int kDevTimeout = MC_ERR_TIMEOUT;
+
+// Everything a kernel needs to walk the paged cache; passed by value.
+struct Params {
+  const void *k_pool, *v_pool;
+  const int32_t *group_offsets, *prefix_pages, *prefix_len, *suffix_pages, *suffix_len;
+  int32_t G, B, Hq, Hkv, d, g;
+  int32_t num_pages, max_pp, max_sp;
+  int32_t n_parts, n_prefix_parts, prefix_part_tokens, suffix_part_tokens;
+  int32_t *status;
+};
+
+enum Mode : int { kPrefix = 0, kSuffix = 1 };
+
+// Which token range an item covers, resolved on the device from the device-resident lengths.
+struct Span {
+  const int32_t *pages;  // page-table row
+  int32_t lo, hi;        // token range [lo, hi) of the sequence, lo a multiple of 16
+  int32_t part;          // part slot the result goes to
+};
+
+__device__ __forceinline__ int group_of(const Params &p, int b) {
+  int lo = 0, hi = p.G;  // invariant: offsets[lo] <= b < offsets[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(p.group_offsets + mid) <= b) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ void latch(const Params &p, int code) { atomicCAS(p.status, 0, code); }
+
+template <int MODE>
+__device__ __forceinline__ Span resolve_span(const Params &p, int b, int part) {
+  Span s;
+  int len, cap, tokens;
+  if (MODE == kPrefix) {
+    int j = group_of(p, b);
+    s.pages = p.prefix_pages + (size_t)j * p.max_pp;
+    len = __ldg(p.prefix_len + j);
+    cap = p.max_pp * kPage;
+    tokens = p.prefix_part_tokens;
+    s.part = part;
+  } else {
+    s.pages = p.suffix_pages + (size_t)b * p.max_sp;
+    len = __ldg(p.suffix_len + b);
+    cap = p.max_sp * kPage;
+    tokens = p.suffix_part_tokens;
+    s.part = p.n_prefix_parts + part;
+  }
+  if (len > cap || len < 0) {  // a length the table cannot hold: clamp and report
+    latch(p, kDevBadPage);
+    len = len < 0 ? 0 : cap;
+  }
+  s.lo = part * tokens;
+  s.hi = min(len, s.lo + tokens);
+  return s;
+}
+
+struct Layout;  // the opaque handle
+
+void count_launch();
+mc_status_t check_launch();
+
+// launchers (each enqueues on `stream` and returns the launch status)
+mc_status_t launch_fma(const Params &p, int dtype, int mode, const void *q, float scale, float *o_part,
+                       float *lse_part, cudaStream_t stream);
+mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
+                       cudaStream_t stream);
+mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
+                         float *lse, cudaStream_t stream);
+bool mma_supported(const Params &p, int dtype);
+
+}  // namespace mc

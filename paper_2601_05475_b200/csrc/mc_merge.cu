@@ -1,0 +1,99 @@
+// Log-sum-exp merge of the per-part partial results: one warp per output row, lanes split the head
+// dimension.  Reads only the parts whose lse is finite.
+#include "mc_internal.cuh"
+
+namespace mc {
+namespace {
+
+constexpr int kWarpsPerBlock = 4;
+
+template <typename T, int VEC>
+__device__ __forceinline__ void store_row(T *dst, const float (&v)[VEC]);
+
+template <>
+__device__ __forceinline__ void store_row<float, 2>(float *dst, const float (&v)[2]) {
+  *reinterpret_cast<float2 *>(dst) = make_float2(v[0], v[1]);
+}
+template <>
+__device__ __forceinline__ void store_row<float, 4>(float *dst, const float (&v)[4]) {
+  *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <>
+__device__ __forceinline__ void store_row<__nv_bfloat16, 2>(__nv_bfloat16 *dst, const float (&v)[2]) {
+  *reinterpret_cast<__nv_bfloat162 *>(dst) = __floats2bfloat162_rn(v[0], v[1]);
+}
+template <>
+__device__ __forceinline__ void store_row<__nv_bfloat16, 4>(__nv_bfloat16 *dst, const float (&v)[4]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  uint2 w;
+  w.x = *reinterpret_cast<uint32_t *>(&a);
+  w.y = *reinterpret_cast<uint32_t *>(&b);
+  *reinterpret_cast<uint2 *>(dst) = w;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+merge_lse_kernel(int rows, int n_parts, const float *__restrict__ o_part, const float *__restrict__ lse_part,
+                 T *__restrict__ o, float *__restrict__ lse) {
+  constexpr int VEC = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float *lp = lse_part + (size_t)row * n_parts;
+  float m = -INFINITY;
+  for (int i = lane; i < n_parts; i += 32) m = fmaxf(m, lp[i]);
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, sh));
+  float acc[VEC];
+#pragma unroll
+  for (int c = 0; c < VEC; ++c) acc[c] = 0.f;
+  float s = 0.f;
+  if (m > -INFINITY) {
+    const float *op = o_part + (size_t)row * n_parts * D + lane * VEC;
+    for (int i = 0; i < n_parts; ++i) {
+      const float li = lp[i];  // same address in every lane: one broadcast load
+      if (li == -INFINITY) continue;
+      const float w = expf(li - m);
+      s += w;
+      if constexpr (VEC == 4) {
+        const float4 v = *reinterpret_cast<const float4 *>(op + (size_t)i * D);
+        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+        acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+      } else {
+        const float2 v = *reinterpret_cast<const float2 *>(op + (size_t)i * D);
+        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+      }
+    }
+    const float inv = 1.f / s;
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) acc[c] *= inv;
+  }
+  store_row<T, VEC>(o + (size_t)row * D + lane * VEC, acc);
+  if (lane == 0) lse[row] = m > -INFINITY ? m + logf(s) : -INFINITY;
+}
+
+template <typename T, int D>
+mc_status_t launch_t(const Params &p, const float *o_part, const float *lse_part, void *o, float *lse,
+                     cudaStream_t stream) {
+  const int rows = p.B * p.Hq;
+  const unsigned grid = (unsigned)((rows + kWarpsPerBlock - 1) / kWarpsPerBlock);
+  merge_lse_kernel<T, D><<<grid, kWarpsPerBlock * 32, 0, stream>>>(rows, p.n_parts, o_part, lse_part, (T *)o, lse);
+  count_launch();
+  return check_launch();
+}
+
+}  // namespace
+
+mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
+                         float *lse, cudaStream_t stream) {
+  if (dtype == MC_F32) {
+    if (p.d == 64) return launch_t<float, 64>(p, o_part, lse_part, o, lse, stream);
+    if (p.d == 128) return launch_t<float, 128>(p, o_part, lse_part, o, lse, stream);
+  } else if (dtype == MC_BF16) {
+    if (p.d == 64) return launch_t<__nv_bfloat16, 64>(p, o_part, lse_part, o, lse, stream);
+    if (p.d == 128) return launch_t<__nv_bfloat16, 128>(p, o_part, lse_part, o, lse, stream);
+  }
+  return MC_ERR_UNSUPPORTED;
+}
+
+}  // namespace mc

@@ -1,0 +1,142 @@
+"""Device-side set-up shared by tests, the smoke check and the benchmark: moves a workload to the GPU as
+torch tensors and wraps the layout handle.  Memory and marshalling only; all arithmetic happens in the
+library's kernels."""
+from __future__ import annotations
+
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as mc
+from . import workload as wl
+
+
+def to_device(cfg: wl.Config, x: np.ndarray, device="cuda") -> torch.Tensor:
+    """float32 values (storage-representable) -> device tensor of the storage dtype."""
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
+    if cfg.dtype == "bf16":
+        t = t.to(torch.bfloat16)
+    return t.to(device)
+
+
+def storage_to_device(cfg: wl.Config, a: np.ndarray, device="cuda") -> torch.Tensor:
+    """Storage array (float32, or uint16 bf16 bits) -> device tensor."""
+    if cfg.dtype == "f32":
+        return torch.from_numpy(a).to(device)
+    return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DeviceProblem:
+    """Pools, tables and lengths on the device plus the library's layout handle and workspace."""
+
+    def __init__(self, cfg: wl.Config, tables: wl.PageTables, prefix_len: np.ndarray, suffix_len: np.ndarray,
+                 k_pool: torch.Tensor, v_pool: torch.Tensor, device="cuda"):
+        self.cfg, self.tables, self.device = cfg, tables, device
+        self.k_pool, self.v_pool = k_pool, v_pool
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        self.prefix_pages, self.suffix_pages = i32(tables.prefix_pages), i32(tables.suffix_pages)
+        self.prefix_len, self.suffix_len = i32(prefix_len), i32(suffix_len)
+        self.group_offsets = i32(tables.group_offsets)
+        d = mc.LayoutDesc()
+        d.num_groups, d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = cfg.G, cfg.B, cfg.Hq, cfg.Hkv, cfg.d
+        d.page_size, d.num_pages = wl.PAGE, tables.num_pages
+        d.max_prefix_pages, d.max_suffix_pages = tables.max_prefix_pages, tables.max_suffix_pages
+        d.dtype = mc.MC_F32 if cfg.dtype == "f32" else mc.MC_BF16
+        d.k_pool, d.v_pool = k_pool.data_ptr(), v_pool.data_ptr()
+        d.group_offsets, d.prefix_pages = self.group_offsets.data_ptr(), self.prefix_pages.data_ptr()
+        d.prefix_len, d.suffix_pages = self.prefix_len.data_ptr(), self.suffix_pages.data_ptr()
+        d.suffix_len = self.suffix_len.data_ptr()
+        self.desc = d
+        self.layout = mc.mc_kv_layout_create(d)
+        self.geom = mc.mc_kv_layout_geometry(self.layout)
+        self.ws_bytes = mc.mc_workspace_bytes(self.layout)
+        self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=device)
+        self.ws_ptr = (self.ws.data_ptr() + 255) // 256 * 256
+        self.tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+        self.o = torch.empty(cfg.B, cfg.Hq, cfg.d, dtype=self.tdtype, device=device)
+        self.lse = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device=device)
+
+    @classmethod
+    def from_host(cls, hp: wl.HostProblem, device="cuda") -> "DeviceProblem":
+        return cls(hp.cfg, hp.tables, hp.prefix_len, hp.suffix_len,
+                   storage_to_device(hp.cfg, hp.k_pool, device), storage_to_device(hp.cfg, hp.v_pool, device), device)
+
+    def new_parts(self):
+        g = self.geom
+        o_part = torch.full((g.rows, g.n_parts, g.head_dim), float("nan"), dtype=torch.float32, device=self.device)
+        lse_part = torch.full((g.rows, g.n_parts), float("nan"), dtype=torch.float32, device=self.device)
+        return o_part, lse_part
+
+    def decode(self, q: torch.Tensor, scale: Optional[float] = None, stream: int = 0):
+        mc.mc_decode_attn(self.layout, q, self.cfg.scale if scale is None else scale, self.o, self.lse,
+                          self.ws_ptr, self.ws_bytes, stream)
+        return self.o, self.lse
+
+    def close(self):
+        if self.layout:
+            mc.mc_kv_layout_destroy(self.layout)
+            self.layout = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, device="cuda") -> DeviceProblem:
+    """Full-size instance whose pools are drawn on the device (torch's seeded generator) instead of being
+    built on the host: lengths and page tables come from `workload`, every slot of both pools is N(0,1)
+    rounded to the storage dtype, and K rows are turned into outliers with the configured probability."""
+    prefix_len, suffix_len = wl.draw_lengths(cfg)
+    tables = wl.build_page_tables(cfg, prefix_len, suffix_len, headroom_tokens)
+    tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    gen = torch.Generator(device=device)
+    gen.manual_seed(cfg.seed * 1000003 + 17)
+    shape = (tables.num_pages, cfg.Hkv, wl.PAGE, cfg.d)
+    k_pool = torch.empty(shape, dtype=tdtype, device=device)
+    v_pool = torch.empty(shape, dtype=tdtype, device=device)
+    step = max(1, (1 << 28) // (cfg.Hkv * wl.PAGE * cfg.d))          # pages per chunk, bounds temporaries
+    for lo in range(0, tables.num_pages, step):
+        hi = min(tables.num_pages, lo + step)
+        k_pool[lo:hi].normal_(generator=gen)
+        v_pool[lo:hi].normal_(generator=gen)
+        if cfg.k_outlier_prob > 0.0:
+            mask = torch.rand((hi - lo, cfg.Hkv, wl.PAGE, 1), device=device, generator=gen) < cfg.k_outlier_prob
+            k_pool[lo:hi] = torch.where(mask, k_pool[lo:hi] * cfg.k_outlier_scale, k_pool[lo:hi])
+    return DeviceProblem(cfg, tables, prefix_len, suffix_len, k_pool, v_pool, device)
+
+
+def device_q(cfg: wl.Config, step: int, device="cuda") -> torch.Tensor:
+    gen = torch.Generator(device=device)
+    gen.manual_seed(cfg.seed * 7919 + 101 + step)
+    tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    return torch.empty((cfg.B, cfg.Hq, cfg.d), dtype=tdtype, device=device).normal_(generator=gen)
+
+
+def device_append(cfg: wl.Config, step: int, device="cuda"):
+    gen = torch.Generator(device=device)
+    gen.manual_seed(cfg.seed * 104729 + 211 + step)
+    tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    k = torch.empty((cfg.B, cfg.Hkv, cfg.d), dtype=tdtype, device=device).normal_(generator=gen)
+    v = torch.empty((cfg.B, cfg.Hkv, cfg.d), dtype=tdtype, device=device).normal_(generator=gen)
+    return k, v
+
+
+def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int] = None):
+    """Copies candidate b's whole history for kv head h to the host, in token order, by plain indexing
+    through the page tables: returns (K [n][d], V [n][d]) as float32 numpy arrays."""
+    j = int(np.searchsorted(dp.tables.group_offsets, b, side="right") - 1)
+    P = int(dp.prefix_len[j].item())
+    s = int(dp.suffix_len[b].item()) if suffix_len_now is None else suffix_len_now
+    out = []
+    for pool in (dp.k_pool, dp.v_pool):
+        parts = []
+        for pages_row, n in ((dp.tables.prefix_pages[j], P), (dp.tables.suffix_pages[b], s)):
+            n_pages = (n + wl.PAGE - 1) // wl.PAGE
+            if n_pages:
+                ids = torch.from_numpy(np.ascontiguousarray(pages_row[:n_pages], dtype=np.int64)).to(pool.device)
+                parts.append(pool[ids, h].reshape(n_pages * wl.PAGE, -1)[:n].float().cpu().numpy())
+        out.append(np.concatenate(parts, axis=0) if parts else np.zeros((0, dp.cfg.d), dtype=np.float32))
+    return out[0], out[1]

@@ -245,6 +245,17 @@ def draw_append(cfg: Config, step: int) -> Tuple[np.ndarray, np.ndarray]:
     return k, v
 
 
+def draw_single_head_history(cfg: Config, index: int, n_tokens: int) -> Tuple[np.ndarray, np.ndarray]:
+    """K [n][d] and V [n][d] of ONE kv head with the configuration's value distribution (outlier rows
+    included), for timing or checking a single (candidate, head) row without building whole pools."""
+    k = _normal(_rng(cfg.seed, _T_KS, 1_000_000 + index), (n_tokens, cfg.d))
+    if cfg.k_outlier_prob > 0.0:
+        mask = _rng(cfg.seed, _T_OUTLIER, 1_000_000 + index).random(n_tokens) < cfg.k_outlier_prob
+        k = np.where(mask[:, None], k * np.float32(cfg.k_outlier_scale), k)
+    v = _normal(_rng(cfg.seed, _T_VS, 1_000_000 + index), (n_tokens, cfg.d))
+    return _round_to_dtype(cfg, k), _round_to_dtype(cfg, v)
+
+
 @dataclasses.dataclass
 class HostProblem:
     """A fully host-resident instance: the logical (unpaged) K/V and, built from it by a separate

@@ -1,0 +1,82 @@
+"""Full-size configurations in the launch configuration the benchmark times: sampled output rows against
+the CPU oracle (each row's whole history is copied back through the page tables and attended in fp64),
+plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as orc
+from paper_2601_05475_b200 import binding as mc
+from paper_2601_05475_b200 import workload as wl
+from paper_2601_05475_b200.harness import device_append, device_q, logical_rows, make_device_problem
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+
+def check_rows(dp, q, o, lse, rows):
+    cfg = dp.cfg
+    errs, lerrs = [], []
+    for (b, hq) in rows:
+        K, V = logical_rows(dp, b, hq // cfg.g)
+        o_ref, lse_ref = orc.attend(q[b, hq].float().cpu().numpy(), K, V, cfg.scale)
+        errs.append(np.abs(o[b, hq].float().cpu().numpy().astype(np.float64) - o_ref))
+        lerrs.append(abs(float(lse[b, hq]) - lse_ref))
+    errs = np.stack(errs)
+    assert errs.max() <= 2e-2 and errs.mean() <= 2e-3, (errs.max(), errs.mean())
+    assert max(lerrs) <= 1e-3, max(lerrs)
+
+
+def sample_rows(cfg, n, seed):
+    rng = np.random.default_rng(seed)
+    rows = [(int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq))) for _ in range(n)]
+    return rows + [(0, 0), (cfg.B - 1, cfg.Hq - 1)]
+
+
+@pytest.mark.parametrize("name,n_rows,steps", [("cfg2", 24, 3), ("cfg3", 24, 0), ("cfg4", 10, 2)])
+def test_full_size_sampled_rows(name, n_rows, steps):
+    cfg = wl.CONFIGS[name]
+    dp = make_device_problem(cfg)
+    q = device_q(cfg, 0)
+    o, lse = dp.decode(q)
+    torch.cuda.synchronize()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    check_rows(dp, q, o, lse, sample_rows(cfg, n_rows, 1))
+    # the first steps of the append sweep
+    for step in range(1, steps + 1):
+        k_new, v_new = device_append(cfg, step)
+        before = dp.suffix_len.clone()
+        mc.mc_kv_append(dp.layout, k_new, v_new)
+        q = device_q(cfg, step)
+        o, lse = dp.decode(q)
+        torch.cuda.synchronize()
+        assert torch.equal(dp.suffix_len, before + 1)
+        rows = sample_rows(cfg, 6, 10 + step)
+        check_rows(dp, q, o, lse, rows)
+        # the appended token is the last row of each sampled candidate's history
+        b, hq = rows[0]
+        K, V = logical_rows(dp, b, hq // cfg.g)
+        np.testing.assert_array_equal(K[-1], k_new[b, hq // cfg.g].float().cpu().numpy())
+        np.testing.assert_array_equal(V[-1], v_new[b, hq // cfg.g].float().cpu().numpy())
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    dp.close()
+
+
+def test_full_size_properties_cfg2():
+    """Any-size properties: constant V gives that constant; candidates of one group with identical queries
+    and empty suffixes give identical outputs; lse grows by log 2 when the history is duplicated."""
+    cfg = wl.CONFIGS["cfg2"]
+    dp = make_device_problem(cfg)
+    q = device_q(cfg, 0)
+    dp.v_pool.fill_(0.5)
+    o, _ = dp.decode(q)
+    torch.cuda.synchronize()
+    assert (o.float() - 0.5).abs().max().item() <= 4e-3
+    dp.suffix_len.zero_()
+    q[:] = q[0:1]
+    o, lse = dp.decode(q)
+    torch.cuda.synchronize()
+    assert torch.equal(o[0], o[17]) and torch.equal(lse[0], lse[63])
+    dp.close()

@@ -1,0 +1,302 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, element by element, on the
+same seeded inputs.  Tolerances: fp32 max-abs 1e-5; bf16 max-abs 2e-2 and mean-abs 2e-3; lse 1e-3 per row."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as orc
+from paper_2601_05475_b200 import binding as mc
+from paper_2601_05475_b200 import workload as wl
+from paper_2601_05475_b200.harness import DeviceProblem, to_device
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+
+def check_close(cfg, o_gpu, lse_gpu, o_ref, lse_ref, rows=None):
+    o = o_gpu.float().cpu().numpy().astype(np.float64)
+    lse = lse_gpu.cpu().numpy().astype(np.float64)
+    if rows is not None:
+        idx = tuple(np.array(rows).T)
+        o, lse, o_ref, lse_ref = o[idx], lse[idx], o_ref[idx], lse_ref[idx]
+    err = np.abs(o - o_ref)
+    assert np.isfinite(o).all()
+    if cfg.dtype == "f32":
+        assert err.max() <= 1e-5, err.max()
+    else:
+        assert err.max() <= 2e-2, err.max()
+        assert err.mean() <= 2e-3, err.mean()
+    both_inf = np.isneginf(lse) & np.isneginf(lse_ref)
+    lerr = np.where(both_inf, 0.0, np.abs(lse - lse_ref))
+    assert np.nanmax(lerr) <= 1e-3, np.nanmax(lerr)
+    return err.max(), err.mean()
+
+
+def oracle_full(hp, q, rows=None):
+    return orc.decode_attention(q, hp.k_prefix, hp.v_prefix, hp.k_suffix, hp.v_suffix,
+                                hp.tables.group_offsets.tolist(), hp.cfg.scale, rows=rows)
+
+
+def run_decode(hp, q_np):
+    dp = DeviceProblem.from_host(hp)
+    q = to_device(hp.cfg, q_np)
+    o, lse = dp.decode(q)
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    return dp, o, lse
+
+
+SMALL = {
+    "cfg0": wl.CONFIGS["cfg0"],
+    "cfg1": wl.CONFIGS["cfg1"],
+    "cfg2s": wl.scaled_down(wl.CONFIGS["cfg2"], "cfg2s", C=8, prefix=("fixed", 1040), suffix=("uniform", 0, 600),
+                            append_steps=4),
+    "cfg3s": wl.scaled_down(wl.CONFIGS["cfg3"], "cfg3s", G=3, C=4, prefix=("loguniform", 90, 1500),
+                            suffix=("uniform", 0, 700)),
+    "cfg3sp": wl.scaled_down(wl.CONFIGS["cfg3"], "cfg3sp", G=3, C=4, prefix=("loguniform", 90, 1500),
+                             suffix=("uniform", 0, 700), permute_pages=True),
+    "cfg4s": wl.scaled_down(wl.CONFIGS["cfg4"], "cfg4s", G=2, C=3, prefix=("fixed", 512),
+                            suffix=("uniform", 1000, 2100), append_steps=2),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_decode_matches_oracle(name):
+    cfg = SMALL[name]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    o_ref, lse_ref = oracle_full(hp, q)
+    check_close(cfg, o, lse, o_ref, lse_ref)
+    dp.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2s", "cfg4s"])
+def test_append_sweep_matches_oracle_every_step(name):
+    cfg = SMALL[name]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    for step in range(1, cfg.append_steps + 1):
+        k_new, v_new = wl.draw_append(cfg, step)
+        mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
+        hp.append(k_new, v_new)
+        q = wl.draw_q(cfg, step)
+        o, lse = dp.decode(to_device(cfg, q))
+        torch.cuda.synchronize()
+        check_close(cfg, o, lse, *oracle_full(hp, q))
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    np.testing.assert_array_equal(dp.suffix_len.cpu().numpy(), hp.suffix_len)
+    # one more append than the head-room allows: rows that are full are refused and reported
+    for _ in range(wl.PAGE + 1):
+        mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_ERR_INVALID_ARG
+    dp.close()
+
+
+def test_parts_match_oracle_on_their_token_ranges():
+    cfg = SMALL["cfg2s"]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp = DeviceProblem.from_host(hp)
+    o_part, lse_part = dp.new_parts()
+    qd = to_device(cfg, q)
+    mc.mc_prefix_attn(dp.layout, qd, cfg.scale, o_part, lse_part)
+    mc.mc_suffix_attn(dp.layout, qd, cfg.scale, o_part, lse_part)
+    torch.cuda.synchronize()
+    g = dp.geom
+    op, lp = o_part.cpu().numpy().astype(np.float64), lse_part.cpu().numpy().astype(np.float64)
+    assert not np.isnan(lp).any()                      # every part slot was written
+    rng = np.random.default_rng(0)
+    for _ in range(40):
+        b, hq = int(rng.integers(cfg.B)), int(rng.integers(cfg.Hq))
+        h, row = hq // cfg.g, b * cfg.Hq + hq
+        for part in range(g.n_parts):
+            if part < g.n_prefix_parts:
+                K, V = hp.k_prefix[0][:, h], hp.v_prefix[0][:, h]
+                lo = part * g.prefix_part_tokens
+                hi = lo + g.prefix_part_tokens
+            else:
+                K, V = hp.k_suffix[b][:, h], hp.v_suffix[b][:, h]
+                lo = (part - g.n_prefix_parts) * g.suffix_part_tokens
+                hi = lo + g.suffix_part_tokens
+            o_ref, lse_ref = orc.token_range_partial(q[b, hq], K, V, cfg.scale, lo, hi)
+            if lse_ref == -np.inf:
+                assert lp[row, part] == -np.inf
+            else:
+                assert abs(lp[row, part] - lse_ref) <= 1e-3
+                assert np.abs(op[row, part] - o_ref).max() <= 2e-2
+    # merging the GPU's partials with the oracle's merge reproduces the oracle's full result
+    o_ref, lse_ref = oracle_full(hp, q, rows=[(1, 3)])
+    om, lm = orc.merge_partials(op[1 * cfg.Hq + 3], lp[1 * cfg.Hq + 3])
+    assert np.abs(om - o_ref[1, 3]).max() <= 2e-2 and abs(lm - lse_ref[1, 3]) <= 1e-3
+    dp.close()
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1"])
+def test_merge_alone_against_oracle_merge(name):
+    cfg = SMALL[name]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    g = dp.geom
+    rng = np.random.default_rng(5)
+    op = rng.normal(size=(g.rows, g.n_parts, g.head_dim)).astype(np.float32)
+    lp = (rng.normal(size=(g.rows, g.n_parts)) * 4).astype(np.float32)
+    lp[rng.random(size=lp.shape) < 0.3] = -np.inf
+    lp[0, :] = -np.inf                                  # a row with no tokens at all
+    lp[1, 1:] = -np.inf                                 # a row with exactly one part
+    lp[2, 0] = 80.0                                     # one dominant part
+    op[np.isneginf(lp)] = np.nan                        # empty parts carry garbage that must not leak
+    mc.mc_merge_lse(dp.layout, torch.from_numpy(op).cuda(), torch.from_numpy(lp).cuda(), dp.o, dp.lse)
+    torch.cuda.synchronize()
+    o, lse = dp.o.float().cpu().numpy().reshape(g.rows, -1), dp.lse.cpu().numpy().reshape(-1)
+    tol = 1e-5 if cfg.dtype == "f32" else 2e-2
+    for r in range(g.rows):
+        o_ref, lse_ref = orc.merge_partials(op[r], lp[r])
+        if lse_ref == -np.inf:
+            assert lse[r] == -np.inf and (o[r] == 0).all()
+        else:
+            assert abs(lse[r] - lse_ref) <= 1e-3 * max(1.0, abs(lse_ref) / 50) and np.abs(o[r] - o_ref).max() <= tol
+    dp.close()
+
+
+EDGE = [
+    # name, dtype, G, C, Hq, Hkv, d, prefix lengths, suffix lengths
+    ("all-suffix-empty", "bf16", 1, 3, 8, 2, 128, [33], [0, 0, 0]),
+    ("prefix-one-token", "bf16", 1, 2, 8, 1, 128, [1], [0, 5]),
+    ("chunk-boundaries", "bf16", 1, 6, 16, 2, 128, [256], [15, 16, 17, 255, 256, 257]),
+    ("mha-g1", "bf16", 1, 2, 4, 4, 128, [70], [40, 300]),
+    ("g2", "bf16", 2, 2, 4, 2, 128, [100, 17], [3, 0, 290, 31]),
+    ("g16-falls-back", "bf16", 1, 2, 16, 1, 128, [50], [10, 90]),
+    ("d64-bf16", "bf16", 1, 2, 8, 2, 64, [50], [10, 90]),
+    ("f32-d128", "f32", 2, 2, 4, 2, 128, [40, 300], [0, 1, 16, 700]),
+    ("single-candidate", "bf16", 1, 1, 8, 1, 128, [512], [513]),
+    ("empty-prefix", "bf16", 1, 2, 8, 2, 128, [0], [20, 0]),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_edge_shapes(case):
+    name, dtype, G, C, Hq, Hkv, d, pl, sl = case
+    cfg = wl.Config(name, dtype, G, C, Hq, Hkv, d, ("fixed", 0), ("fixed", tuple(sl)), permute_pages=True, seed=3)
+    hp = wl.make_host_problem(cfg, prefix_len=np.array(pl, dtype=np.int32), suffix_len=np.array(sl, dtype=np.int32))
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    o_ref, lse_ref = oracle_full(hp, q)
+    check_close(cfg, o, lse, o_ref, lse_ref)
+    if name == "empty-prefix":                          # candidate 1 has no tokens at all
+        assert torch.isneginf(lse[1]).all() and (o[1] == 0).all()
+    dp.close()
+
+
+def test_unequal_group_sizes():
+    cfg = wl.Config("unequal", "bf16", 2, 2, 8, 2, 128, ("fixed", 0), ("fixed", (5, 40, 0, 100)), seed=4)
+    hp = wl.make_host_problem(cfg, prefix_len=np.array([64, 200], dtype=np.int32))
+    hp.tables.group_offsets = np.array([0, 3, 4], dtype=np.int32)        # 3 candidates, then 1
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+def test_forced_alu_path_matches_oracle(monkeypatch):
+    """The plain-ALU split-KV kernels (no tensor cores) on a bf16 configuration."""
+    monkeypatch.setenv("MC_FORCE_FMA", "1")
+    cfg = SMALL["cfg2s"]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+@pytest.mark.parametrize("tp,ts", [(16, 16), (64, 48), (4096, 4096)])
+def test_result_does_not_depend_on_part_geometry(monkeypatch, tp, ts):
+    monkeypatch.setenv("MC_PREFIX_PART_TOKENS", str(tp))
+    monkeypatch.setenv("MC_SUFFIX_PART_TOKENS", str(ts))
+    cfg = SMALL["cfg3s"]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    assert dp.geom.prefix_part_tokens == tp and dp.geom.suffix_part_tokens == ts
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+def test_bad_page_id_is_reported_not_dereferenced():
+    cfg = SMALL["cfg1"]
+    hp = wl.make_host_problem(cfg)
+    hp.tables.suffix_pages[2, 0] = hp.tables.num_pages + 7
+    hp.tables.prefix_pages[0, 3] = -5
+    dp = DeviceProblem.from_host(hp)
+    dp.decode(to_device(cfg, wl.draw_q(cfg, 0)))
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_ERR_INVALID_ARG
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK          # reading clears the word
+    assert torch.isfinite(dp.o.float()).all()
+    dp.close()
+
+
+def test_validate_accepts_good_tables_and_rejects_aliased_pages():
+    cfg = SMALL["cfg1"]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    scratch = torch.empty(hp.tables.num_pages, dtype=torch.int32, device="cuda")
+    assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_OK
+    dp.close()
+    hp.tables.suffix_pages[3, 0] = hp.tables.suffix_pages[4, 0]
+    dp = DeviceProblem.from_host(hp)
+    assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_ERR_INVALID_ARG
+    assert mc.mc_kv_layout_validate(dp.layout, scratch, 4) == mc.MC_ERR_WORKSPACE_TOO_SMALL
+    dp.close()
+
+
+def test_host_errors_are_returned_immediately():
+    cfg = SMALL["cfg0"]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    q = to_device(cfg, wl.draw_q(cfg, 0))
+    L = mc.lib()
+    assert L.mc_decode_attn(dp.layout, q.data_ptr(), cfg.scale, dp.o.data_ptr(), dp.lse.data_ptr(), dp.ws_ptr,
+                            dp.ws_bytes - 1, 0) == mc.MC_ERR_WORKSPACE_TOO_SMALL
+    assert L.mc_decode_attn(dp.layout, q.data_ptr() + 4, cfg.scale, dp.o.data_ptr(), dp.lse.data_ptr(), dp.ws_ptr,
+                            dp.ws_bytes, 0) == mc.MC_ERR_INVALID_ARG
+    assert L.mc_decode_attn(dp.layout, 0, cfg.scale, dp.o.data_ptr(), dp.lse.data_ptr(), dp.ws_ptr, dp.ws_bytes,
+                            0) == mc.MC_ERR_INVALID_ARG
+    bad = mc.LayoutDesc.from_buffer_copy(dp.desc)
+    bad.page_size = 32
+    h = mc.c_void_p()
+    assert L.mc_kv_layout_create(mc.byref(bad), mc.byref(h)) == mc.MC_ERR_UNSUPPORTED and not h.value
+    bad = mc.LayoutDesc.from_buffer_copy(dp.desc)
+    bad.num_q_heads = 3
+    bad.num_kv_heads = 2
+    assert L.mc_kv_layout_create(mc.byref(bad), mc.byref(h)) == mc.MC_ERR_INVALID_ARG
+    dp.close()
+
+
+def test_host_buffer_step_matches_device_step():
+    cfg = SMALL["cfg2s"]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    k_new, v_new = wl.draw_append(cfg, 1)
+    q = wl.draw_q(cfg, 1)
+    pin = lambda x: to_device(cfg, x, "cpu").pin_memory()
+    o_h = torch.empty(cfg.B, cfg.Hq, cfg.d, dtype=dp.tdtype).pin_memory()
+    lse_h = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32).pin_memory()
+    mc.mc_decode_step_host(dp.layout, pin(k_new), pin(v_new), pin(q), cfg.scale, o_h, lse_h, dp.ws_ptr, dp.ws_bytes)
+    hp.append(k_new, v_new)
+    check_close(cfg, o_h, lse_h, *oracle_full(hp, q))
+    dp.close()
+
+
+def test_launch_counter_counts_kernels():
+    cfg = SMALL["cfg0"]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    n0 = mc.mc_launch_count()
+    dp.decode(to_device(cfg, wl.draw_q(cfg, 0)))
+    assert mc.mc_launch_count() - n0 >= 3
+    dp.close()
