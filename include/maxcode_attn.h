@@ -151,6 +151,34 @@ mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, 
                                 const void *q_host, float scale, void *o_host, float *lse_host,
                                 void *ws, size_t ws_bytes, void *stream);
 
+/* (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * The whole step - prefix pass, suffix pass, merge - without a layout handle, a workspace or any
+ * allocation.  It is meant for code that runs where cudaMalloc is off limits: inside a serving loop
+ * whose memory was carved up at start-up by another allocator, in a plug-in that is forbidden to touch
+ * the device heap, or late in a process whose GPU memory is already fully committed.  The partial results
+ * go to a fixed scratch array compiled into the library (mc_static_scratch_bytes() bytes, 16 MiB, resident
+ * on every GPU that loads the library until the process exits).  The call itself calls no cudaMalloc /
+ * cudaFree and no allocating library routine.
+ *   desc        same descriptor as mc_kv_layout_create (all pointers DEVICE memory, borrowed for the call)
+ *   q, o, lse   device, as for mc_decode_attn
+ *   dev_status  optional device int32: set to 0, then to MC_ERR_INVALID_ARG if a bad page id or length is
+ *               met (such pages are skipped).  NULL: the condition is recorded nowhere the caller can read.
+ * Limits and rules:
+ *   - status(256 B) + rows*n_parts*(d+1)*4 bytes of partials must fit the scratch array, with rows = B*Hq
+ *     and n_parts as mc_kv_layout_geometry would report; otherwise MC_ERR_WORKSPACE_TOO_SMALL and nothing
+ *     is launched.  (Configuration 1 needs about 1.7 MiB; the large benchmark configurations do not fit.)
+ *   - The first call on each device looks up the scratch array's device address (the device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents (the call clears the status
+ *     word it uses; every part slot is rewritten).  Two calls whose kernels overlap on the GPU - different
+ *     streams, or different threads - race on it: serialise them.
+ *   - Asynchronous on `stream`, like the other hot calls.  Both passes run on the warp-level kernels. */
+mc_status_t mc_decode_attn_static(const mc_kv_layout_desc_t *desc, const void *q, float scale, void *o,
+                                  float *lse, int32_t *dev_status, void *stream);
+
+/* Size in bytes of the scratch array behind mc_decode_attn_static. */
+size_t mc_static_scratch_bytes(void);
+
 /* Reads and clears the device status word (synchronises `stream`): MC_OK, or the first latched error. */
 mc_status_t mc_get_last_status(mc_kv_layout_t *layout, void *stream);
 

@@ -43,6 +43,8 @@ EXPORTS = {
     "mc_decode_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "mc_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p,
                                       c_void_p, c_size_t, c_void_p]),
+    "mc_decode_attn_static": (c_int32, [POINTER(LayoutDesc), c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "mc_static_scratch_bytes": (c_size_t, []),
     "mc_get_last_status": (c_int32, [c_void_p, c_void_p]),
     "mc_launch_count": (c_uint64, []),
     "mc_status_string": (c_char_p, [c_int32]),
@@ -146,6 +148,16 @@ def mc_decode_step_host(layout: int, k_new_host, v_new_host, q_host, scale: floa
     _check(lib().mc_decode_step_host(layout, _ptr(k_new_host), _ptr(v_new_host), _ptr(q_host), scale,
                                      _ptr(o_host), _ptr(lse_host), _ptr(ws), ws_bytes, stream),
            "mc_decode_step_host")
+
+
+def mc_decode_attn_static(desc: LayoutDesc, q, scale: float, o, lse, dev_status=None, stream: int = 0) -> int:
+    """The step without handle, workspace or allocation (scratch compiled into the library).  Returns the
+    status code instead of raising, so callers can test for MC_ERR_WORKSPACE_TOO_SMALL."""
+    return lib().mc_decode_attn_static(byref(desc), _ptr(q), scale, _ptr(o), _ptr(lse), _ptr(dev_status), stream)
+
+
+def mc_static_scratch_bytes() -> int:
+    return int(lib().mc_static_scratch_bytes())
 
 
 def mc_get_last_status(layout: int, stream: int = 0) -> int:
