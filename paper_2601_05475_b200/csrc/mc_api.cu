@@ -16,6 +16,9 @@ struct Layout {
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
+  PrefixTcPlan *tc_plan;      // non-null: the prefix pass runs on the tcgen05 kernel
+  cudaStream_t side_stream;   // the prefix pass of mc_decode_attn runs here, beside the suffix pass
+  cudaEvent_t fork_ev, join_ev;
 };
 
 static std::atomic<uint64_t> g_launches{0};
@@ -31,7 +34,7 @@ int env_int(const char *name, int dflt) {
   const char *s = std::getenv(name);
   if (!s || !*s) return dflt;
   int v = std::atoi(s);
-  return v > 0 ? v : dflt;
+  return v >= 0 ? v : dflt;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -106,6 +109,7 @@ mc_status_t check_q(const Layout *L, const void *q) {
 
 mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t st) {
+  if (mode == kPrefix && L->tc_plan) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
   if (L->use_mma) return launch_mma(L->p, mode, q, scale, o_part, lse_part, st);
   return launch_fma(L->p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
 }
@@ -165,8 +169,8 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   if (tp > 4096) tp = 4096;
   int ts = mc::pow2_floor(max_s / 16 > 256 ? max_s / 16 : 256);
   if (ts > 4096) ts = 4096;
-  tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
-  ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
+  if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0) tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
+  if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
   if (tp < mc::kPage) tp = mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
   p.prefix_part_tokens = tp;
@@ -193,6 +197,28 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   }
   *L->host_status = 0;
   p.status = L->dev_status;
+
+  // Tensor-core prefix pass: needs the largest group (read once from the device) and tensor maps over the pools.
+  L->tc_plan = nullptr;
+  if (mc::prefix_tc_supported(p, d->dtype) && mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0)) {
+    int32_t *go = new (std::nothrow) int32_t[p.G + 1];
+    int dev = 0, sms = 148;
+    if (go && cudaMemcpy(go, d->group_offsets, sizeof(int32_t) * (p.G + 1), cudaMemcpyDeviceToHost) == cudaSuccess &&
+        cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
+      int max_group = 1;
+      for (int j = 0; j < p.G; ++j) max_group = go[j + 1] - go[j] > max_group ? go[j + 1] - go[j] : max_group;
+      if (max_group <= p.B) L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, mc::env_int("MC_PREFIX_CTAS", 0));
+    }
+    delete[] go;
+    (void)cudaGetLastError();
+  }
+  if (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&L->fork_ev, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&L->join_ev, cudaEventDisableTiming) != cudaSuccess) {
+    mc_kv_layout_destroy(reinterpret_cast<mc_kv_layout_t *>(L));
+    return MC_ERR_CUDA;
+  }
   *out = reinterpret_cast<mc_kv_layout_t *>(L);
   return MC_OK;
 }
@@ -200,6 +226,10 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
 mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   Layout *L = reinterpret_cast<Layout *>(layout);
   if (!L) return MC_OK;
+  if (L->side_stream) cudaStreamDestroy(L->side_stream);
+  if (L->fork_ev) cudaEventDestroy(L->fork_ev);
+  if (L->join_ev) cudaEventDestroy(L->join_ev);
+  mc::prefix_tc_plan_free(L->tc_plan);
   cudaFree(L->dev_status);
   cudaFreeHost(L->host_status);
   delete L;
@@ -294,8 +324,15 @@ mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, v
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   float *o_part = reinterpret_cast<float *>(ws);
   float *lse_part = reinterpret_cast<float *>(static_cast<char *>(ws) + L->o_part_bytes);
+  // The prefix pass (tensor-bound) runs on the handle's side stream beside the suffix pass (HBM-bound);
+  // the two write disjoint part slots.  The merge joins them.
+  if (cudaEventRecord(L->fork_ev, st) != cudaSuccess ||
+      cudaStreamWaitEvent(L->side_stream, L->fork_ev, 0) != cudaSuccess)
+    return MC_ERR_CUDA;
+  if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, L->side_stream)) != MC_OK) return s;
+  if (cudaEventRecord(L->join_ev, L->side_stream) != cudaSuccess) return MC_ERR_CUDA;
   if ((s = mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
-  if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+  if (cudaStreamWaitEvent(st, L->join_ev, 0) != cudaSuccess) return MC_ERR_CUDA;
   return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
 }
 

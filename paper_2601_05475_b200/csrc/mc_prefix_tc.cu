@@ -1,0 +1,540 @@
+// Prefix pass on the 5th-generation tensor cores (bf16, d = 128).
+//
+// For one (group, kv head) the queries of all the group's candidates that map to that kv head are
+// stacked into dense 128-row tiles (row = candidate * g + head-in-group), so the group's prefix K/V is
+// streamed once for the whole group instead of once per candidate:
+//     S = Q_s K^T          128 x 128 tile, tcgen05.mma, operands in shared memory, accumulator in TMEM
+//     P = exp2(S*c - m)    one thread per row reads its row of S from TMEM, writes bf16 P to shared memory
+//     O += P V             tcgen05.mma, V consumed in its natural [token][d] layout (MN-major B operand)
+// K/V pages reach shared memory by TMA (one 16-token x 64-element box per page and head-dim half,
+// 128-byte swizzle) through a tensor map laid over the paged pool; the page id is a TMA coordinate.
+//
+// Work item = (group, kv head, prefix split, 128-row tile); persistent CTAs take items round-robin.
+// Warp roles: warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs (warp 1 owns the TMEM allocation),
+// warps 2-5 (128 threads, one per TMEM lane) do the softmax, the rescale and the epilogue.
+// Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
+// (bounded) for its outstanding copies, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "mc_internal.cuh"
+
+namespace mc {
+namespace {
+
+constexpr int D = 128;
+constexpr int kTileM = 128;      // stacked query rows per tile
+constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
+constexpr int kPagesPerTile = kTileN / kPage;
+constexpr int kStages = 2;
+constexpr int kThreads = 192;
+constexpr uint32_t kHalfBytes = kTileN * 64 * 2;        // one head-dim (or token) half of a 128x128 bf16 tile
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;         // 32 KB
+constexpr uint32_t kBoxBytes = kPage * 64 * 2;          // one TMA box: 16 tokens x 64 elements
+constexpr uint32_t kTmemCols = 256;                     // S: columns [0,128), O: columns [128,256)
+constexpr long long kWaitCycles = 2000000000ll;         // ~1 s
+
+struct __align__(1024) Smem {
+  uint8_t q[kTileBytes];
+  uint8_t p[kTileBytes];
+  uint8_t k[kStages][kTileBytes];
+  uint8_t v[kStages][kTileBytes];
+  uint64_t full_k[kStages], full_v[kStages], empty[kStages];
+  uint64_t q_ready, s_full, p_full, pv_done;
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit expires or another
+// role has already aborted.
+__device__ __forceinline__ bool mbar_wait(Smem &sm, const Params &p, uint64_t *bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (sm.abort) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      sm.abort = 1;
+      latch(p, kDevTimeout);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_box(void *dst, const CUtensorMap *map, int x, int tok, int head, int page,
+                                             uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(tok), "r"(head), "r"(page), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  `lbo`/`sbo` in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3fffu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3fffu) << 32;
+  d |= 1ull << 46;   // descriptor version of this architecture
+  d |= 2ull << 61;   // 128-byte swizzle
+  return d;
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> f32, M = 128, N = 128
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) |
+                                ((uint32_t)(kTileM >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;                // A, B both K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // B (= V) MN-major
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+struct Item {
+  int j, h, sp, mt;      // group, kv head, prefix split, row tile
+  int b0, n_cand;        // first candidate of the group, candidates in the group
+  int lo, hi;            // token range of this split
+  const int32_t *pages;
+};
+
+__device__ __forceinline__ Item decode_item(const Params &p, int item, int n_mt) {
+  Item it;
+  it.mt = item % n_mt;
+  int r = item / n_mt;
+  it.sp = r % p.n_prefix_parts;
+  r /= p.n_prefix_parts;
+  it.h = r % p.Hkv;
+  it.j = r / p.Hkv;
+  it.b0 = __ldg(p.group_offsets + it.j);
+  it.n_cand = __ldg(p.group_offsets + it.j + 1) - it.b0;
+  int len = __ldg(p.prefix_len + it.j);
+  const int cap = p.max_pp * kPage;
+  if (len < 0 || len > cap) {
+    latch(p, kDevBadPage);
+    len = len < 0 ? 0 : cap;
+  }
+  it.lo = it.sp * p.prefix_part_tokens;
+  it.hi = min(len, it.lo + p.prefix_part_tokens);
+  it.pages = p.prefix_pages + (size_t)it.j * p.max_pp;
+  return it;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                 const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
+                 float *__restrict__ lse_part, int n_items, int n_mt) {
+  extern __shared__ uint8_t smem_raw[];
+  Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = p.g, cand_per_tile = kTileM / g;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.full_k[s], 1);
+      mbar_init(&sm.full_v[s], 1);
+      mbar_init(&sm.empty[s], 1);
+    }
+    mbar_init(&sm.q_ready, 128);
+    mbar_init(&sm.s_full, 1);
+    mbar_init(&sm.p_full, 128);
+    mbar_init(&sm.pv_done, 1);
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+  const uint32_t tmem_s = tmem, tmem_o = tmem + kTileN;
+
+  // Tile counters advance identically in every role: `kt` counts K/V tiles, `it_n` counts non-empty items.
+  uint32_t kt = 0, it_n = 0;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
+        const Item it = decode_item(p, item, n_mt);
+        if (it.lo >= it.hi || it.mt * cand_per_tile >= it.n_cand) continue;
+        const int last_pg = (it.hi - 1) >> 4;
+        for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
+          const int s = kt % kStages;
+          if (!mbar_wait(sm, p, &sm.empty[s], ((kt / kStages) & 1) ^ 1)) break;
+          mbar_expect_tx(&sm.full_k[s], kTileBytes);
+          mbar_expect_tx(&sm.full_v[s], kTileBytes);
+#pragma unroll 1
+          for (int pg = 0; pg < kPagesPerTile; ++pg) {
+            // pages past the end of the prefix repeat the last valid page: finite data, masked later
+            int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
+            if ((unsigned)pid >= (unsigned)p.num_pages) pid = 0;   // reported and masked by the softmax role
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+              tma_load_box(sm.k[s] + hf * kHalfBytes + pg * kBoxBytes, &k_map, hf * 64, 0, it.h, pid, &sm.full_k[s]);
+          }
+#pragma unroll 1
+          for (int pg = 0; pg < kPagesPerTile; ++pg) {
+            int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
+            if ((unsigned)pid >= (unsigned)p.num_pages) pid = 0;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+              tma_load_box(sm.v[s] + hf * kHalfBytes + pg * kBoxBytes, &v_map, hf * 64, 0, it.h, pid, &sm.full_v[s]);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t q_addr = smem_u32(sm.q), p_addr = smem_u32(sm.p);
+      for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
+        const Item it = decode_item(p, item, n_mt);
+        if (it.lo >= it.hi || it.mt * cand_per_tile >= it.n_cand) continue;
+        if (!mbar_wait(sm, p, &sm.q_ready, it_n & 1)) break;
+        ++it_n;
+        tc_fence_after();
+        const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+        // Iteration t issues S(t) = Q K(t)^T (S is free: P(t-1) has been written) and then
+        // O += P(t-1) V(t-1); the softmax of tile t overlaps the second product.
+        bool ok = true;
+        for (int t = 0; t <= n_tiles && ok; ++t) {
+          if (t < n_tiles) {
+            const uint32_t ktq = kt + t;
+            const int s = ktq % kStages;
+            if (t > 0) ok = mbar_wait(sm, p, &sm.p_full, (ktq - 1) & 1);   // S(t-1) consumed, P(t-1) staged
+            ok = ok && mbar_wait(sm, p, &sm.full_k[s], (ktq / kStages) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t k_addr = smem_u32(sm.k[s]);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+              umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
+            }
+            umma_commit(&sm.s_full);
+          }
+          if (t > 0) {
+            const uint32_t ktp = kt + t - 1;
+            const int s = ktp % kStages;
+            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full_v[s], (ktp / kStages) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t v_addr = smem_u32(sm.v[s]);
+#pragma unroll
+            for (int kk = 0; kk < kTileN / 16; ++kk) {
+              const uint32_t a_off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+              umma_ss(tmem_o, smem_desc(p_addr + a_off, 16, 1024), smem_desc(v_addr + kk * 2048, kHalfBytes, 1024),
+                      kIdescPV, (t > 1) || (kk > 0));
+            }
+            umma_commit(&sm.empty[s]);
+            umma_commit(&sm.pv_done);
+          }
+        }
+        if (!ok) break;
+        kt += n_tiles;
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax / epilogue (128 threads)
+    const int quad = warp & 3;                 // TMEM lane quadrant this warp may access
+    const int r = quad * 32 + lane;            // row of the tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
+      const Item it = decode_item(p, item, n_mt);
+      if (it.mt * cand_per_tile >= it.n_cand) continue;
+      const int cand = it.mt * cand_per_tile + r / g;
+      const bool row_ok = cand < it.n_cand;
+      const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
+      const size_t slot = qrow * p.n_parts + it.sp;
+      if (it.lo >= it.hi) {
+        if (row_ok) lse_part[slot] = -INFINITY;
+        continue;
+      }
+      // stage this tile's stacked queries: row r, 16-byte chunk c of half hf -> swizzled position
+      {
+        const uint4 *src = reinterpret_cast<const uint4 *>(q + qrow * D);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (row_ok) v = __ldg(src + c);
+          *reinterpret_cast<uint4 *>(sm.q + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+        }
+        fence_async_proxy();
+        mbar_arrive(&sm.q_ready);
+      }
+      float m = -INFINITY, l = 0.f;
+      const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+      bool alive = true;
+      for (int t = 0; t < n_tiles && alive; ++t, ++kt) {
+        const int t0 = it.lo + t * kTileN;
+        // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
+        uint32_t page_ok = 0;
+#pragma unroll
+        for (int pg = 0; pg < kPagesPerTile; ++pg) {
+          const int tok = t0 + pg * kPage;
+          if (tok < it.hi) {
+            const int pid = __ldg(it.pages + (tok >> 4));
+            if ((unsigned)pid < (unsigned)p.num_pages) page_ok |= 1u << pg; else latch(p, kDevBadPage);
+          }
+        }
+        alive = mbar_wait(sm, p, &sm.s_full, kt & 1);
+        alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
+        if (!alive) break;
+        tc_fence_after();
+        // pass 1: row maximum
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kTileN; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_s + lane_addr + c0, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int col = c0 + i;
+            const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
+            if (ok) mx = fmaxf(mx, __uint_as_float(v[i]) * sl2);
+          }
+        }
+        // The running maximum moves only when the new one is clearly larger (2^8): P stays bounded by
+        // 2^8 and the accumulator in TMEM is rescaled rarely.
+        float m_use = m;
+        bool rescale = false;
+        if (mx > m + 8.f) {
+          m_use = mx;
+          rescale = t > 0 && m > -INFINITY;
+        }
+        const float alpha = rescale ? fast_exp2(m - m_use) : 1.f;
+        // P(t-1) V(t-1) must have completed before P is overwritten or O is touched
+        if (t > 0) {
+          alive = mbar_wait(sm, p, &sm.pv_done, (kt - 1) & 1);
+          alive = __all_sync(0xffffffffu, alive);
+          if (!alive) break;
+          tc_fence_after();
+        }
+        if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_o + lane_addr + c0, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+            tmem_st32(tmem_o + lane_addr + c0, v);
+          }
+          tmem_wait_st();
+        }
+        l *= alpha;
+        m = m_use;
+        const float mref = m == -INFINITY ? 0.f : m;
+        // pass 2: probabilities, bf16, into the swizzled A-operand tile
+#pragma unroll 1
+        for (int c0 = 0; c0 < kTileN; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_s + lane_addr + c0, v);
+          tmem_wait_ld();
+          float pr[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int col = c0 + i;
+            const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
+            pr[i] = ok ? fast_exp2(__uint_as_float(v[i]) * sl2 - mref) : 0.f;
+            l += pr[i];
+          }
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {   // 4 chunks of 8 tokens
+            uint4 w;
+            w.x = pack_bf16x2(pr[8 * c + 0], pr[8 * c + 1]);
+            w.y = pack_bf16x2(pr[8 * c + 2], pr[8 * c + 3]);
+            w.z = pack_bf16x2(pr[8 * c + 4], pr[8 * c + 5]);
+            w.w = pack_bf16x2(pr[8 * c + 6], pr[8 * c + 7]);
+            const int chunk = (c0 >> 3) + c;   // 0..15 along the token axis
+            *reinterpret_cast<uint4 *>(sm.p + (chunk >> 3) * kHalfBytes + r * 128 + (((chunk & 7) ^ (r & 7)) << 4)) = w;
+          }
+        }
+        tc_fence_before();
+        fence_async_proxy();
+        mbar_arrive(&sm.p_full);
+      }
+      if (!alive) break;
+      // epilogue: O / l -> o_part, lse
+      alive = mbar_wait(sm, p, &sm.pv_done, (kt - 1) & 1);
+      if (!__all_sync(0xffffffffu, alive)) break;
+      tc_fence_after();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      float *dst = o_part + slot * D;
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_o + lane_addr + c0, v);
+        tmem_wait_ld();
+        if (row_ok && l > 0.f) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4)
+            *reinterpret_cast<float4 *>(dst + c0 + i) =
+                make_float4(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv,
+                            __uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+        }
+      }
+      if (row_ok) lse_part[slot] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+      tc_fence_before();
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (sm.abort && warp == 0 && lane == 0) {
+    // give copies that are still in flight a bounded time to land before the CTA's shared memory goes away
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv) {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !sym)
+      return false;
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  // pool[page][head][token][d]: innermost first
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)kPage, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
+  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)kPage, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct PrefixTcPlan {
+  CUtensorMap k_map, v_map;
+  int n_mt, n_items, grid;
+};
+
+bool prefix_tc_supported(const Params &p, int dtype) {
+  return dtype == MC_BF16 && p.d == D && p.g >= 1 && p.g <= kTileM && kTileM % p.g == 0 &&
+         p.prefix_part_tokens % kTileN == 0;
+}
+
+// Host-side preparation at layout-create time: tensor maps over the two pools and the item count.
+// `max_group` is the largest number of candidates in one group.  Returns nullptr when unavailable.
+PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int max_ctas) {
+  PrefixTcPlan *plan = new PrefixTcPlan();
+  if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv) ||
+      !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv)) {
+    delete plan;
+    return nullptr;
+  }
+  plan->n_mt = (max_group * p.g + kTileM - 1) / kTileM;
+  plan->n_items = p.G * p.Hkv * p.n_prefix_parts * plan->n_mt;
+  int grid = plan->n_items < sm_count ? plan->n_items : sm_count;
+  if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
+  plan->grid = grid < 1 ? 1 : grid;
+  if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(sizeof(Smem) + 1024)) != cudaSuccess) {
+    delete plan;
+    return nullptr;
+  }
+  return plan;
+}
+
+void prefix_tc_plan_free(PrefixTcPlan *plan) { delete plan; }
+
+mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
+                             float *lse_part, cudaStream_t stream) {
+  prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem) + 1024, stream>>>(
+      p, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
+      plan->n_items, plan->n_mt);
+  count_launch();
+  return check_launch();
+}
+
+}  // namespace mc
