@@ -165,7 +165,8 @@ mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, 
  *               met (such pages are skipped).  NULL: the condition is recorded nowhere the caller can read.
  * Limits and rules:
  *   - status(256 B) + rows*n_parts*(d+1)*4 bytes of partials must fit the scratch array, with rows = B*Hq
- *     and n_parts as mc_kv_layout_geometry would report; otherwise MC_ERR_WORKSPACE_TOO_SMALL and nothing
+ *     and n_parts = ceil(max_prefix_tokens/Tp) + ceil(max_suffix_tokens/Ts), Tp and Ts its own fixed rule
+ *     (about 8 prefix splits and 16 suffix chunks, 256..4096 tokens); otherwise MC_ERR_WORKSPACE_TOO_SMALL and nothing
  *     is launched.  (Configuration 1 needs about 1.7 MiB; the large benchmark configurations do not fit.)
  *   - The first call on each device looks up the scratch array's device address (the device must be
  *     current); make that first call outside any stream capture.

@@ -17,7 +17,7 @@ struct Layout {
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
   PrefixTcPlan *tc_plan;      // non-null: the prefix pass runs on the tcgen05 kernel
-  cudaStream_t side_stream;   // the prefix pass of mc_decode_attn runs here, beside the suffix pass
+  cudaStream_t side_stream;   // the suffix pass of mc_decode_attn runs here, beside the prefix pass
   cudaEvent_t fork_ev, join_ev;
 };
 
@@ -109,7 +109,7 @@ mc_status_t check_q(const Layout *L, const void *q) {
 
 mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t st) {
-  if (mode == kPrefix && L->tc_plan) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
+  if (mode == kPrefix && L->tc_plan && scale != 0.f) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
   if (L->use_mma) return launch_mma(L->p, mode, q, scale, o_part, lse_part, st);
   return launch_fma(L->p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
 }
@@ -165,8 +165,15 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
 
   // Part geometry from the table strides (the lengths themselves live on the device and may grow).
   const int max_p = d->max_prefix_pages * mc::kPage, max_s = d->max_suffix_pages * mc::kPage;
-  int tp = mc::pow2_floor(max_p / 8 > 256 ? max_p / 8 : 256);
-  if (tp > 4096) tp = 4096;
+  // Prefix splits: each (group, kv head, 128-row tile) is cut into just enough token ranges for about 160
+  // work items in all (a few dozen persistent CTAs share them); long ranges keep the per-item prologue and
+  // epilogue small against the streamed tiles.
+  const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
+  const long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
+  int nsp = (int)((160 + pairs - 1) / pairs);
+  if (nsp > 8) nsp = 8;
+  if (nsp < 1) nsp = 1;
+  int tp = ((max_p + nsp - 1) / nsp + 127) / 128 * 128;
   int ts = mc::pow2_floor(max_s / 16 > 256 ? max_s / 16 : 256);
   if (ts > 4096) ts = 4096;
   if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0) tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
@@ -208,7 +215,29 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
       int max_group = 1;
       for (int j = 0; j < p.G; ++j) max_group = go[j + 1] - go[j] > max_group ? go[j + 1] - go[j] : max_group;
-      if (max_group <= p.B) L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, mc::env_int("MC_PREFIX_CTAS", 0));
+      // How many SMs the prefix pass should hold: enough to finish within the suffix pass's HBM time, no
+      // more, because every SM it holds runs the suffix pass at half occupancy.  Estimated once from the
+      // lengths as they are now (tile time and stream rate are measured constants of this kernel pair).
+      int ctas = mc::env_int("MC_PREFIX_CTAS", 0);
+      int32_t *pl = new (std::nothrow) int32_t[p.G], *sl = new (std::nothrow) int32_t[p.B];
+      if (ctas == 0 && pl && sl &&
+          cudaMemcpy(pl, d->prefix_len, sizeof(int32_t) * p.G, cudaMemcpyDeviceToHost) == cudaSuccess &&
+          cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
+        double tiles = 0.0, suffix_tokens = 0.0;
+        for (int j = 0; j < p.G; ++j) {
+          const int rows = (go[j + 1] - go[j]) * p.g;
+          tiles += (double)((pl[j] + 127) / 128) * p.Hkv * ((rows + 127) / 128);
+        }
+        for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
+        const double suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * e / 6.0e6;   // ~6 TB/s
+        const double prefix_sm_us = tiles * 2.6;                                  // ~2.6 us per tile beside the stream
+        ctas = suffix_us > 1.0 ? (int)(prefix_sm_us / suffix_us * 1.1) + 1 : sms;
+        if (ctas < 8) ctas = 8;
+        if (ctas > sms) ctas = sms;
+      }
+      delete[] pl;
+      delete[] sl;
+      if (max_group <= p.B) L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, ctas);
     }
     delete[] go;
     (void)cudaGetLastError();
@@ -324,15 +353,18 @@ mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, v
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   float *o_part = reinterpret_cast<float *>(ws);
   float *lse_part = reinterpret_cast<float *>(static_cast<char *>(ws) + L->o_part_bytes);
-  // The prefix pass (tensor-bound) runs on the handle's side stream beside the suffix pass (HBM-bound);
-  // the two write disjoint part slots.  The merge joins them.
+  // The two passes write disjoint part slots and run side by side: the prefix pass (tensor-bound, a few
+  // persistent CTAs per SM's shared memory) is launched first, on the caller's stream, so that its CTAs are
+  // resident before the suffix pass (HBM-bound, thousands of short CTAs) floods the SMs from the handle's
+  // side stream.  The merge joins them.
   if (cudaEventRecord(L->fork_ev, st) != cudaSuccess ||
       cudaStreamWaitEvent(L->side_stream, L->fork_ev, 0) != cudaSuccess)
     return MC_ERR_CUDA;
-  if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, L->side_stream)) != MC_OK) return s;
-  if (cudaEventRecord(L->join_ev, L->side_stream) != cudaSuccess) return MC_ERR_CUDA;
-  if ((s = mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
-  if (cudaStreamWaitEvent(st, L->join_ev, 0) != cudaSuccess) return MC_ERR_CUDA;
+  if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+  if ((s = mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, L->side_stream)) != MC_OK) return s;
+  if (cudaEventRecord(L->join_ev, L->side_stream) != cudaSuccess ||
+      cudaStreamWaitEvent(st, L->join_ev, 0) != cudaSuccess)
+    return MC_ERR_CUDA;
   return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
 }
 

@@ -42,12 +42,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
+// Private suffix data is read exactly once per step: it bypasses L1 and is marked evict-first in L2 so
+// that it does not push out the shared prefix, which every step re-reads.
+__device__ __forceinline__ uint64_t l2_stream_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
 template <bool STREAM>
-__device__ __forceinline__ uint4 ld16(const uint4 *p) {
+__device__ __forceinline__ uint4 ld16(const uint4 *p, uint64_t policy) {
   uint4 v;
   if (STREAM)
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;\n"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy));
   else
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
@@ -60,17 +67,18 @@ struct PageRegs {
 };
 
 template <bool STREAM>
-__device__ __forceinline__ void issue_loads(PageRegs &r, const uint4 *kslab, const uint4 *vslab, int gid, int tig) {
+__device__ __forceinline__ void issue_loads(PageRegs &r, const uint4 *kslab, const uint4 *vslab, int gid, int tig,
+                                            uint64_t pol) {
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    r.k[j] = ld16<STREAM>(kslab + gid * 16 + tig + 4 * j);
-    r.k[4 + j] = ld16<STREAM>(kslab + (gid + 8) * 16 + tig + 4 * j);
+    r.k[j] = ld16<STREAM>(kslab + gid * 16 + tig + 4 * j, pol);
+    r.k[4 + j] = ld16<STREAM>(kslab + (gid + 8) * 16 + tig + 4 * j, pol);
   }
 #pragma unroll
   for (int x = 0; x < 4; ++x) {
     const int tok = 2 * tig + (x & 1) + (x >> 1) * 8;
-    r.v[2 * x] = ld16<STREAM>(vslab + tok * 16 + gid);
-    r.v[2 * x + 1] = ld16<STREAM>(vslab + tok * 16 + gid + 8);
+    r.v[2 * x] = ld16<STREAM>(vslab + tok * 16 + gid, pol);
+    r.v[2 * x + 1] = ld16<STREAM>(vslab + tok * 16 + gid + 8, pol);
   }
 }
 
@@ -184,11 +192,12 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
     return ((size_t)pid * p.Hkv + h) * kSlab;
   };
 
+  const uint64_t pol = l2_stream_policy();
   PageRegs ra, rb;
   int hi_a, hi_b = 0;
   {
     const size_t s = slab_of(__ldg(sp.pages + pg_first), hi_a);
-    issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig);
+    issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
   }
   int pid_next = pg_first + 1 < pg_end ? __ldg(sp.pages + pg_first + 1) : 0;
   for (int pg = pg_first; pg < pg_end; pg += 2) {
@@ -196,14 +205,14 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
     int pid_next2 = 0;
     if (has_b) {
       const size_t s = slab_of(pid_next, hi_b);
-      issue_loads<STREAM>(rb, kpool + s, vpool + s, gid, tig);
+      issue_loads<STREAM>(rb, kpool + s, vpool + s, gid, tig, pol);
       if (pg + 2 < pg_end) pid_next2 = __ldg(sp.pages + pg + 2);
     }
     compute_page(st, ra, qf, sl2, pg * kPage, hi_a, gid, tig);
     if (has_b) {
       if (pg + 2 < pg_end) {
         const size_t s = slab_of(pid_next2, hi_a);
-        issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig);
+        issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
         if (pg + 3 < pg_end) pid_next = __ldg(sp.pages + pg + 3);
       }
       compute_page(st, rb, qf, sl2, (pg + 1) * kPage, hi_b, gid, tig);

@@ -4,14 +4,15 @@
 // stacked into dense 128-row tiles (row = candidate * g + head-in-group), so the group's prefix K/V is
 // streamed once for the whole group instead of once per candidate:
 //     S = Q_s K^T          128 x 128 tile, tcgen05.mma, operands in shared memory, accumulator in TMEM
-//     P = exp2(S*c - m)    one thread per row reads its row of S from TMEM, writes bf16 P to shared memory
-//     O += P V             tcgen05.mma, V consumed in its natural [token][d] layout (MN-major B operand)
+//     P = exp2(S*c - m)    one thread per row reads its row of S from TMEM, writes bf16 P back to TMEM
+//     O += P V             tcgen05.mma, P from TMEM, V in its natural [token][d] layout (MN-major B operand)
 // K/V pages reach shared memory by TMA (one 16-token x 64-element box per page and head-dim half,
 // 128-byte swizzle) through a tensor map laid over the paged pool; the page id is a TMA coordinate.
 //
 // Work item = (group, kv head, prefix split, 128-row tile); persistent CTAs take items round-robin.
-// Warp roles: warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs (warp 1 owns the TMEM allocation),
-// warps 2-5 (128 threads, one per TMEM lane) do the softmax, the rescale and the epilogue.
+// Warp roles: warp 0 issues the TMA copies and stages the next item's query tile, warp 1 lane 0 issues
+// the MMAs (warp 1 owns the TMEM allocation), warps 2-5 (128 threads, one per TMEM lane) do the softmax,
+// the rescale and the epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -25,21 +26,20 @@ constexpr int D = 128;
 constexpr int kTileM = 128;      // stacked query rows per tile
 constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
 constexpr int kPagesPerTile = kTileN / kPage;
-constexpr int kStages = 2;
+constexpr int kSlots = 5;         // ring of 32 KB operand slots: K(t), V(t), K(t+1), V(t+1), K(t+2)
 constexpr int kThreads = 192;
 constexpr uint32_t kHalfBytes = kTileN * 64 * 2;        // one head-dim (or token) half of a 128x128 bf16 tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;         // 32 KB
 constexpr uint32_t kBoxBytes = kPage * 64 * 2;          // one TMA box: 16 tokens x 64 elements
-constexpr uint32_t kTmemCols = 256;                     // S: columns [0,128), O: columns [128,256)
+constexpr uint32_t kTmemCols = 512;                     // S: [0,128)  O: [128,256)  P (bf16 pairs): [256,320), [320,384)
 constexpr long long kWaitCycles = 2000000000ll;         // ~1 s
 
 struct __align__(1024) Smem {
-  uint8_t q[kTileBytes];
-  uint8_t p[kTileBytes];
-  uint8_t k[kStages][kTileBytes];
-  uint8_t v[kStages][kTileBytes];
-  uint64_t full_k[kStages], full_v[kStages], empty[kStages];
-  uint64_t q_ready, s_full, p_full, pv_done;
+  uint8_t q[2][kTileBytes];           // stacked query tile of the current and of the next item
+  uint8_t ring[kSlots][kTileBytes];   // load u = 2*tile + (0: K, 1: V) goes to slot u % kSlots
+  uint64_t full[kSlots], empty[kSlots];
+  uint64_t q_ready[2], q_free[2], s_full, s_free, p_full, pv_done[2];
+  uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -80,11 +80,19 @@ __device__ __forceinline__ bool mbar_wait(Smem &sm, const Params &p, uint64_t *b
   }
 }
 
+// The shared prefix is re-read by every row tile of its group and again at every decode step: its
+// lines are asked to stay in L2 (evict-last), while the private suffix streams past them.
+__device__ __forceinline__ uint64_t l2_keep_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void tma_load_box(void *dst, const CUtensorMap *map, int x, int tok, int head, int page,
-                                             uint64_t *bar) {
+                                             uint64_t *bar, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(tok), "r"(head), "r"(page), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4, %5}], [%6], %7;\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(tok), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
 
@@ -104,6 +112,17 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes x 8 columns per 16-element k-step (two bf16 per column)
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -189,7 +208,12 @@ __device__ __forceinline__ Item decode_item(const Params &p, int item, int n_mt)
   return it;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+// An item with no rows or no tokens is skipped by every role alike.
+__device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile) {
+  return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
+}
+
+__global__ void __maxnreg__(168)
 prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                  const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
                  float *__restrict__ lse_part, int n_items, int n_mt) {
@@ -199,15 +223,19 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
   const int g = p.g, cand_per_tile = kTileM / g;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.full_k[s], 1);
-      mbar_init(&sm.full_v[s], 1);
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(&sm.full[s], 1);
       mbar_init(&sm.empty[s], 1);
     }
-    mbar_init(&sm.q_ready, 128);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm.q_ready[b], 32);
+      mbar_init(&sm.q_free[b], 1);
+    }
     mbar_init(&sm.s_full, 1);
+    mbar_init(&sm.s_free, 128);
     mbar_init(&sm.p_full, 128);
-    mbar_init(&sm.pv_done, 1);
+    mbar_init(&sm.pv_done[0], 1);
+    mbar_init(&sm.pv_done[1], 1);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -220,88 +248,155 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tmem_s = tmem, tmem_o = tmem + kTileN;
+  const uint32_t tmem_s = tmem, tmem_o = tmem + kTileN, tmem_p = tmem + 2 * kTileN;
 
-  // Tile counters advance identically in every role: `kt` counts K/V tiles, `it_n` counts non-empty items.
+  // Counters advance identically in every role: `kt` counts K/V tiles, `it_n` counts items with work.
   uint32_t kt = 0, it_n = 0;
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
-        const Item it = decode_item(p, item, n_mt);
-        if (it.lo >= it.hi || it.mt * cand_per_tile >= it.n_cand) continue;
-        const int last_pg = (it.hi - 1) >> 4;
-        for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
-          const int s = kt % kStages;
-          if (!mbar_wait(sm, p, &sm.empty[s], ((kt / kStages) & 1) ^ 1)) break;
-          mbar_expect_tx(&sm.full_k[s], kTileBytes);
-          mbar_expect_tx(&sm.full_v[s], kTileBytes);
-#pragma unroll 1
-          for (int pg = 0; pg < kPagesPerTile; ++pg) {
-            // pages past the end of the prefix repeat the last valid page: finite data, masked later
-            int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
-            if ((unsigned)pid >= (unsigned)p.num_pages) pid = 0;   // reported and masked by the softmax role
+    // ---------------------------------------------------------------- producer (all 32 lanes)
+    // K/V: a tile is 32 TMA boxes (K and V, 8 pages, 2 head-dim halves), one per lane.
+    // Q:   the stacked query tile of the NEXT item is staged (plain loads, swizzled stores) into the
+    //      other Q buffer while the current item is being computed.
+    const int pg = lane & 7, hf = (lane >> 3) & 1, is_v = lane >> 4;
+    const uint64_t policy = l2_keep_policy();
+    const CUtensorMap *map = is_v ? &v_map : &k_map;
+    bool ok = true;
+
+    auto next_item = [&](int from, Item &out) -> int {
+      for (int i = from; i < n_items; i += gridDim.x) {
+        out = decode_item(p, i, n_mt);
+        if (item_has_work(out, cand_per_tile)) return i;
+      }
+      return n_items;
+    };
+    // Staging of one query tile (128 rows x 16 chunks of 16 bytes) proceeds in 8 rounds of 8 chunks per
+    // lane.  Round i's loads are issued in one call and stored (swizzled) in the next, so that their
+    // latency hides behind a K/V tile's worth of other work.
+    constexpr int kQRounds = 8;
+    uint4 qv[8];
+    auto q_load = [&](const Item &qi, int round) {
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-              tma_load_box(sm.k[s] + hf * kHalfBytes + pg * kBoxBytes, &k_map, hf * 64, 0, it.h, pid, &sm.full_k[s]);
-          }
-#pragma unroll 1
-          for (int pg = 0; pg < kPagesPerTile; ++pg) {
-            int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
-            if ((unsigned)pid >= (unsigned)p.num_pages) pid = 0;
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-              tma_load_box(sm.v[s] + hf * kHalfBytes + pg * kBoxBytes, &v_map, hf * 64, 0, it.h, pid, &sm.full_v[s]);
-          }
+      for (int i = 0; i < 8; ++i) {
+        const int idx = round * 256 + i * 32 + lane, row = idx >> 4, c = idx & 15;
+        const int cand = qi.mt * cand_per_tile + row / g;
+        qv[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (cand < qi.n_cand) {
+          const size_t qrow = (size_t)(qi.b0 + cand) * p.Hq + (size_t)qi.h * g + (row % g);
+          qv[i] = __ldg(reinterpret_cast<const uint4 *>(q + qrow * D) + c);
         }
       }
+    };
+    auto q_store = [&](uint8_t *dst, int round) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int idx = round * 256 + i * 32 + lane, row = idx >> 4, c = idx & 15;
+        *reinterpret_cast<uint4 *>(dst + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = qv[i];
+      }
+    };
+    // One step of staging item `qi` (ordinal n among items with work); `round` runs 0..kQRounds.
+    auto q_step = [&](const Item &qi, uint32_t n, int &round) -> bool {
+      const int buf = n & 1;
+      if (round == 0 && n >= 2) {   // the buffer's previous tenant (item n-2) must have finished its first products
+        bool w = mbar_wait(sm, p, &sm.q_free[buf], ((n >> 1) - 1) & 1);
+        if (!__all_sync(0xffffffffu, w)) return false;
+      }
+      if (round > 0) q_store(sm.q[buf], round - 1);
+      if (round < kQRounds) q_load(qi, round);
+      if (round == kQRounds) {
+        fence_async_proxy();
+        mbar_arrive(&sm.q_ready[buf]);
+      }
+      ++round;
+      return true;
+    };
+
+    Item it, nxt;
+    int cur = next_item(blockIdx.x, it);
+    if (cur < n_items) {
+      int round = 0;
+      while (ok && round <= kQRounds) ok = q_step(it, 0, round);
+    }
+    while (ok && cur < n_items && !sm.abort) {
+      const int nxt_idx = next_item(cur + gridDim.x, nxt);
+      int round = nxt_idx < n_items ? 0 : kQRounds + 1;   // staging state of the next item's query tile
+      const int last_pg = (it.hi - 1) >> 4;
+      for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
+        const uint32_t u = 2 * kt + is_v;           // lanes 0-15 load K(t), lanes 16-31 load V(t)
+        const int s = u % kSlots;
+        // pages past the end of the prefix repeat the last valid page: finite data, masked later
+        int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
+        const bool in_range = t0 + pg * kPage < it.hi, good = (unsigned)pid < (unsigned)p.num_pages;
+        if (in_range && !good) latch(p, kDevBadPage);
+        if (!good) pid = 0;   // a bad page id is replaced by page 0 and its 16 columns are masked
+        const uint32_t okmask = __ballot_sync(0xffffffffu, in_range && good) & 0xffu;
+        ok = mbar_wait(sm, p, &sm.empty[s], ((u / kSlots) & 1) ^ 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        // published before the arrive below; the softmax role reads it after the chain of barrier waits
+        // (full -> first product -> s_full) that this arrive starts
+        if (lane == 0) sm.page_ok[kt & 7] = okmask;
+        if ((lane & 15) == 0) mbar_expect_tx(&sm.full[s], kTileBytes);
+        __syncwarp();
+        tma_load_box(sm.ring[s] + hf * kHalfBytes + pg * kBoxBytes, map, hf * 64, 0, it.h, pid, &sm.full[s], policy);
+        if (round <= kQRounds) {
+          ok = q_step(nxt, it_n + 1, round);
+          if (!ok) break;
+        }
+      }
+      while (ok && round <= kQRounds) ok = q_step(nxt, it_n + 1, round);   // short item: finish the staging now
+      it = nxt;
+      cur = nxt_idx;
+      ++it_n;
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t q_addr = smem_u32(sm.q), p_addr = smem_u32(sm.p);
       for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
         const Item it = decode_item(p, item, n_mt);
-        if (it.lo >= it.hi || it.mt * cand_per_tile >= it.n_cand) continue;
-        if (!mbar_wait(sm, p, &sm.q_ready, it_n & 1)) break;
+        if (!item_has_work(it, cand_per_tile)) continue;
+        const int qb = it_n & 1;
+        if (!mbar_wait(sm, p, &sm.q_ready[qb], (it_n >> 1) & 1)) break;
         ++it_n;
         tc_fence_after();
+        const uint32_t q_addr = smem_u32(sm.q[qb]);
         const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
-        // Iteration t issues S(t) = Q K(t)^T (S is free: P(t-1) has been written) and then
-        // O += P(t-1) V(t-1); the softmax of tile t overlaps the second product.
+        // Iteration t issues S(t) = Q K(t)^T as soon as the softmax role holds S(t-1) in registers, then
+        // O += P(t-1) V(t-1) once P(t-1) is staged: the exponentials of tile t-1 overlap the first
+        // product, the row maxima of tile t overlap the second.  The first product of the next item
+        // follows the last second product directly and runs under this item's epilogue.
         bool ok = true;
         for (int t = 0; t <= n_tiles && ok; ++t) {
           if (t < n_tiles) {
-            const uint32_t ktq = kt + t;
-            const int s = ktq % kStages;
-            if (t > 0) ok = mbar_wait(sm, p, &sm.p_full, (ktq - 1) & 1);   // S(t-1) consumed, P(t-1) staged
-            ok = ok && mbar_wait(sm, p, &sm.full_k[s], (ktq / kStages) & 1);
+            const uint32_t ktq = kt + t, u = 2 * ktq;
+            const int s = u % kSlots;
+            if (ktq > 0) ok = mbar_wait(sm, p, &sm.s_free, (ktq - 1) & 1);
+            ok = ok && mbar_wait(sm, p, &sm.full[s], (u / kSlots) & 1);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t k_addr = smem_u32(sm.k[s]);
+            const uint32_t k_addr = smem_u32(sm.ring[s]);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
               umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
             }
+            umma_commit(&sm.empty[s]);   // K(t) is free as soon as the first product has read it
             umma_commit(&sm.s_full);
+            if (t == n_tiles - 1) umma_commit(&sm.q_free[qb]);   // last reader of this item's Q tile
           }
           if (t > 0) {
-            const uint32_t ktp = kt + t - 1;
-            const int s = ktp % kStages;
-            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full_v[s], (ktp / kStages) & 1);
+            const uint32_t ktp = kt + t - 1, u = 2 * ktp + 1;
+            const int s = u % kSlots;
+            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full[s], (u / kSlots) & 1);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t v_addr = smem_u32(sm.v[s]);
+            const uint32_t v_addr = smem_u32(sm.ring[s]), p_cols = tmem_p + (ktp & 1) * (kTileN / 2);
 #pragma unroll
-            for (int kk = 0; kk < kTileN / 16; ++kk) {
-              const uint32_t a_off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-              umma_ss(tmem_o, smem_desc(p_addr + a_off, 16, 1024), smem_desc(v_addr + kk * 2048, kHalfBytes, 1024),
-                      kIdescPV, (t > 1) || (kk > 0));
-            }
+            for (int kk = 0; kk < kTileN / 16; ++kk)
+              umma_ts(tmem_o, p_cols + kk * 8, smem_desc(v_addr + kk * 2048, kHalfBytes, 1024), kIdescPV,
+                      (t > 1) || (kk > 0));
             umma_commit(&sm.empty[s]);
-            umma_commit(&sm.pv_done);
+            umma_commit(&sm.pv_done[ktp & 1]);
           }
         }
         if (!ok) break;
@@ -324,51 +419,54 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         if (row_ok) lse_part[slot] = -INFINITY;
         continue;
       }
-      // stage this tile's stacked queries: row r, 16-byte chunk c of half hf -> swizzled position
-      {
-        const uint4 *src = reinterpret_cast<const uint4 *>(q + qrow * D);
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          uint4 v = make_uint4(0u, 0u, 0u, 0u);
-          if (row_ok) v = __ldg(src + c);
-          *reinterpret_cast<uint4 *>(sm.q + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
-        }
-        fence_async_proxy();
-        mbar_arrive(&sm.q_ready);
-      }
-      float m = -INFINITY, l = 0.f;
+      float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2)
       const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
       bool alive = true;
       for (int t = 0; t < n_tiles && alive; ++t, ++kt) {
         const int t0 = it.lo + t * kTileN;
-        // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
-        uint32_t page_ok = 0;
-#pragma unroll
-        for (int pg = 0; pg < kPagesPerTile; ++pg) {
-          const int tok = t0 + pg * kPage;
-          if (tok < it.hi) {
-            const int pid = __ldg(it.pages + (tok >> 4));
-            if ((unsigned)pid < (unsigned)p.num_pages) page_ok |= 1u << pg; else latch(p, kDevBadPage);
-          }
-        }
         alive = mbar_wait(sm, p, &sm.s_full, kt & 1);
         alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
         if (!alive) break;
         tc_fence_after();
-        // pass 1: row maximum
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTileN; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem_s + lane_addr + c0, v);
-          tmem_wait_ld();
+        // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
+        const uint32_t page_ok = sm.page_ok[kt & 7];
+        const bool full_tile = page_ok == 0xffu && t0 + kTileN <= it.hi;
+        // the whole row of S into registers, then S is free for the next tile's first product
+        uint32_t sv[4][32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = c0 + i;
-            const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
-            if (ok) mx = fmaxf(mx, __uint_as_float(v[i]) * sl2);
-          }
+        for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_addr + c * 32, sv[c]);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&sm.s_free);
+        if (!full_tile) {   // ragged tail or a bad page: masked scores become -inf (sl2 > 0) / +inf (sl2 < 0)
+          const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int col = c * 32 + i;
+              const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
+              if (!ok) sv[c][i] = masked;
+            }
         }
+        // row extremum of the raw scores; times sl2 it is the row maximum of the scaled scores
+        float e4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) e4[c] = __uint_as_float(sv[c][0]);
+        if (sl2 >= 0.f) {
+#pragma unroll
+          for (int i = 1; i < 32; ++i)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) e4[c] = fmaxf(e4[c], __uint_as_float(sv[c][i]));
+        } else {
+#pragma unroll
+          for (int i = 1; i < 32; ++i)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) e4[c] = fminf(e4[c], __uint_as_float(sv[c][i]));
+        }
+        const float ext = sl2 >= 0.f ? fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]))
+                                     : fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
+        const float mx = (ext == INFINITY || ext == -INFINITY) ? -INFINITY : ext * sl2;   // all masked -> -inf
         // The running maximum moves only when the new one is clearly larger (2^8): P stays bounded by
         // 2^8 and the accumulator in TMEM is rescaled rarely.
         float m_use = m;
@@ -378,14 +476,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
           rescale = t > 0 && m > -INFINITY;
         }
         const float alpha = rescale ? fast_exp2(m - m_use) : 1.f;
-        // P(t-1) V(t-1) must have completed before P is overwritten or O is touched
-        if (t > 0) {
-          alive = mbar_wait(sm, p, &sm.pv_done, (kt - 1) & 1);
+        if (__any_sync(0xffffffffu, rescale)) {
+          // every earlier product into O must have completed before O is rescaled in place
+          alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
           alive = __all_sync(0xffffffffu, alive);
           if (!alive) break;
           tc_fence_after();
-        }
-        if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
           for (int c0 = 0; c0 < D; c0 += 32) {
             uint32_t v[32];
@@ -399,39 +495,39 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         }
         l *= alpha;
         m = m_use;
-        const float mref = m == -INFINITY ? 0.f : m;
-        // pass 2: probabilities, bf16, into the swizzled A-operand tile
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTileN; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem_s + lane_addr + c0, v);
-          tmem_wait_ld();
-          float pr[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = c0 + i;
-            const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
-            pr[i] = ok ? fast_exp2(__uint_as_float(v[i]) * sl2 - mref) : 0.f;
-            l += pr[i];
-          }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {   // 4 chunks of 8 tokens
-            uint4 w;
-            w.x = pack_bf16x2(pr[8 * c + 0], pr[8 * c + 1]);
-            w.y = pack_bf16x2(pr[8 * c + 2], pr[8 * c + 3]);
-            w.z = pack_bf16x2(pr[8 * c + 4], pr[8 * c + 5]);
-            w.w = pack_bf16x2(pr[8 * c + 6], pr[8 * c + 7]);
-            const int chunk = (c0 >> 3) + c;   // 0..15 along the token axis
-            *reinterpret_cast<uint4 *>(sm.p + (chunk >> 3) * kHalfBytes + r * 128 + (((chunk & 7) ^ (r & 7)) << 4)) = w;
-          }
+        const float neg_m = m == -INFINITY ? 0.f : -m;
+        // P goes to TMEM as the A operand of the second product: lane = row, one column per token pair.
+        // The buffer of this tile's parity was last read by the second product of tile kt-2.
+        if (kt >= 2) {
+          alive = mbar_wait(sm, p, &sm.pv_done[kt & 1], ((kt - 2) >> 1) & 1);
+          alive = __all_sync(0xffffffffu, alive);
+          if (!alive) break;
+          tc_fence_after();
         }
+        const uint32_t p_cols = tmem_p + lane_addr + (kt & 1) * (kTileN / 2);
+        float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {     // 64 tokens -> 32 packed columns
+          uint32_t pw[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int c = half * 2 + (j >> 4), i = (2 * j) & 31;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][i]), sl2, neg_m));       // masked: exp2(-inf) = 0
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][i + 1]), sl2, neg_m));
+            lsum[j & 1] += p0;
+            lsum[2 + (j & 1)] += p1;
+            pw[j] = pack_bf16x2(p0, p1);
+          }
+          tmem_st32(p_cols + half * 32, pw);
+        }
+        l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
+        tmem_wait_st();
         tc_fence_before();
-        fence_async_proxy();
         mbar_arrive(&sm.p_full);
       }
       if (!alive) break;
       // epilogue: O / l -> o_part, lse
-      alive = mbar_wait(sm, p, &sm.pv_done, (kt - 1) & 1);
+      alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
       if (!__all_sync(0xffffffffu, alive)) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -517,6 +613,10 @@ PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int m
   plan->n_items = p.G * p.Hkv * p.n_prefix_parts * plan->n_mt;
   int grid = plan->n_items < sm_count ? plan->n_items : sm_count;
   if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
+  if (grid < 1) grid = 1;
+  // items are dealt round-robin: the fewest CTAs that keep the same number of rounds hold fewer SMs
+  const int rounds = (plan->n_items + grid - 1) / grid;
+  if (rounds > 0) grid = (plan->n_items + rounds - 1) / rounds;
   plan->grid = grid < 1 ? 1 : grid;
   if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)(sizeof(Smem) + 1024)) != cudaSuccess) {

@@ -73,7 +73,7 @@ mc_status_t mc_decode_attn_static(const mc_kv_layout_desc_t *d, const void *q, f
   p.G = d->num_groups; p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.d = d->head_dim;
   p.g = d->num_q_heads / d->num_kv_heads;
   p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
-  // same part geometry rule as the layout object: about 8 prefix splits and 16 suffix chunks per row
+  // fixed part geometry: about 8 prefix splits and 16 suffix chunks per row, 256..4096 tokens each
   const long long max_p = (long long)d->max_prefix_pages * mc::kPage, max_s = (long long)d->max_suffix_pages * mc::kPage;
   int tp = mc::pow2_floor((int)(max_p / 8 > 256 ? max_p / 8 : 256)), ts = mc::pow2_floor((int)(max_s / 16 > 256 ? max_s / 16 : 256));
   if (tp > 4096) tp = 4096;
