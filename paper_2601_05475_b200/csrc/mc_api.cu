@@ -165,14 +165,57 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
 
   // Part geometry from the table strides (the lengths themselves live on the device and may grow).
   const int max_p = d->max_prefix_pages * mc::kPage, max_s = d->max_suffix_pages * mc::kPage;
-  // Prefix splits: each (group, kv head, 128-row tile) is cut into just enough token ranges for about 160
-  // work items in all (a few dozen persistent CTAs share them); long ranges keep the per-item prologue and
-  // epilogue small against the streamed tiles.
-  const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
-  const long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
-  int nsp = (int)((160 + pairs - 1) / pairs);
-  if (nsp > 8) nsp = 8;
-  if (nsp < 1) nsp = 1;
+  // Prefix splits and the number of persistent CTAs of the tensor-core prefix pass are sized together, once,
+  // from the lengths as they are now.  The prefix pass should finish inside the suffix pass's HBM time while
+  // holding as few SMs as possible (an SM it holds runs the suffix pass at half occupancy), and every work
+  // item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be long: as few
+  // splits as still let one item fit the time budget.  Constants are measured for this kernel pair.
+  int nsp = 0, tc_ctas = mc::env_int("MC_PREFIX_CTAS", 0), max_group = (p.B + p.G - 1) / p.G;
+  {
+    const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
+    long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
+    double tiles = (double)pairs * ((max_p + 127) / 128), suffix_us = 0.0;
+    int32_t *go = new (std::nothrow) int32_t[p.G + 1], *pl = new (std::nothrow) int32_t[p.G];
+    int32_t *sl = new (std::nothrow) int32_t[p.B];
+    const size_t eb = d->dtype == MC_F32 ? 4 : 2;
+    if (go && pl && sl &&
+        cudaMemcpy(go, d->group_offsets, sizeof(int32_t) * (p.G + 1), cudaMemcpyDeviceToHost) == cudaSuccess &&
+        cudaMemcpy(pl, d->prefix_len, sizeof(int32_t) * p.G, cudaMemcpyDeviceToHost) == cudaSuccess &&
+        cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
+      pairs = 0;
+      tiles = 0.0;
+      max_group = 1;
+      for (int j = 0; j < p.G; ++j) {
+        const int c = go[j + 1] - go[j];
+        if (c > max_group) max_group = c;
+        const long long pj = (long long)p.Hkv * ((c * p.g + 127) / 128);
+        pairs += pj;
+        tiles += (double)pj * ((pl[j] + 127) / 128);
+      }
+      double suffix_tokens = 0.0;
+      for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
+      suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * eb / 6.8e6;   // the stream runs at about 6.8 TB/s
+    }
+    (void)cudaGetLastError();
+    delete[] go;
+    delete[] pl;
+    delete[] sl;
+    if (pairs < 1) pairs = 1;
+    const double tile_us = 1.6, item_us = 6.0;                      // per 128x128 tile; per item
+    const double budget = suffix_us * 0.9, max_pair_tiles = (max_p + 127) / 128;
+    for (nsp = 1; nsp < 8; ++nsp)
+      if ((max_pair_tiles + nsp - 1) / nsp * tile_us + item_us <= budget) break;
+    if (budget < item_us + tile_us) nsp = (int)((160 + pairs - 1) / pairs);   // nothing to hide under: many items
+    if (nsp > 8) nsp = 8;
+    if (nsp < 1) nsp = 1;
+    if (tc_ctas == 0) {
+      const double items = (double)pairs * nsp, avg_item_us = tiles / items * tile_us + item_us;
+      int rounds = (int)(0.7 * budget / avg_item_us);
+      if (rounds < 1) rounds = 1;
+      tc_ctas = (int)((items + rounds - 1) / rounds);
+      if (tc_ctas < 8) tc_ctas = 8;
+    }
+  }
   int tp = ((max_p + nsp - 1) / nsp + 127) / 128 * 128;
   int ts = mc::pow2_floor(max_s / 16 > 256 ? max_s / 16 : 256);
   if (ts > 4096) ts = 4096;
@@ -205,41 +248,13 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   *L->host_status = 0;
   p.status = L->dev_status;
 
-  // Tensor-core prefix pass: needs the largest group (read once from the device) and tensor maps over the pools.
+  // Tensor-core prefix pass: tensor maps over the pools and the persistent grid.
   L->tc_plan = nullptr;
   if (mc::prefix_tc_supported(p, d->dtype) && mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0)) {
-    int32_t *go = new (std::nothrow) int32_t[p.G + 1];
     int dev = 0, sms = 148;
-    if (go && cudaMemcpy(go, d->group_offsets, sizeof(int32_t) * (p.G + 1), cudaMemcpyDeviceToHost) == cudaSuccess &&
-        cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
-      int max_group = 1;
-      for (int j = 0; j < p.G; ++j) max_group = go[j + 1] - go[j] > max_group ? go[j + 1] - go[j] : max_group;
-      // How many SMs the prefix pass should hold: enough to finish within the suffix pass's HBM time, no
-      // more, because every SM it holds runs the suffix pass at half occupancy.  Estimated once from the
-      // lengths as they are now (tile time and stream rate are measured constants of this kernel pair).
-      int ctas = mc::env_int("MC_PREFIX_CTAS", 0);
-      int32_t *pl = new (std::nothrow) int32_t[p.G], *sl = new (std::nothrow) int32_t[p.B];
-      if (ctas == 0 && pl && sl &&
-          cudaMemcpy(pl, d->prefix_len, sizeof(int32_t) * p.G, cudaMemcpyDeviceToHost) == cudaSuccess &&
-          cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
-        double tiles = 0.0, suffix_tokens = 0.0;
-        for (int j = 0; j < p.G; ++j) {
-          const int rows = (go[j + 1] - go[j]) * p.g;
-          tiles += (double)((pl[j] + 127) / 128) * p.Hkv * ((rows + 127) / 128);
-        }
-        for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
-        const double suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * e / 6.0e6;   // ~6 TB/s
-        const double prefix_sm_us = tiles * 2.6;                                  // ~2.6 us per tile beside the stream
-        ctas = suffix_us > 1.0 ? (int)(prefix_sm_us / suffix_us * 1.1) + 1 : sms;
-        if (ctas < 8) ctas = 8;
-        if (ctas > sms) ctas = sms;
-      }
-      delete[] pl;
-      delete[] sl;
-      if (max_group <= p.B) L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, ctas);
-    }
-    delete[] go;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && max_group <= p.B)
+      L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, tc_ctas > sms ? sms : tc_ctas);
     (void)cudaGetLastError();
   }
   if (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||

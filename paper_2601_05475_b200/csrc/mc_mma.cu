@@ -11,6 +11,8 @@
 // fragment wants are assembled from two token rows with byte permutes.  The 16x8 probability tile is
 // moved from accumulator layout to B-operand layout with two 8x8 matrix transposes.
 // Softmax statistics are kept per lane for the two heads the lane's accumulators belong to.
+#include <cstdlib>
+
 #include "mc_internal.cuh"
 
 namespace mc {
@@ -48,6 +50,10 @@ __device__ __forceinline__ uint64_t l2_stream_policy() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
   return pol;
+}
+// Asks L2 to fetch one 4 KB (page, kv head) slab; costs no registers and no shared memory.
+__device__ __forceinline__ void l2_prefetch_slab(const void *p) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(p), "r"(kPage * D * 2) : "memory");
 }
 template <bool STREAM>
 __device__ __forceinline__ uint4 ld16(const uint4 *p, uint64_t policy) {
@@ -139,7 +145,7 @@ __device__ __forceinline__ void compute_page(State &st, const PageRegs &r, const
 template <int MODE>
 __global__ void __launch_bounds__(kWarps * 32, 2)
 attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
-                float *__restrict__ lse_part) {
+                float *__restrict__ lse_part, int prefetch_pages) {
   constexpr bool STREAM = MODE == kSuffix;  // private suffix data is read exactly once
   const int lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
   const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.n_prefix_parts;
@@ -200,9 +206,26 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
     issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
   }
   int pid_next = pg_first + 1 < pg_end ? __ldg(sp.pages + pg_first + 1) : 0;
+  // The register double buffer covers one page of latency; the stream from HBM is kept kPrefetch pages
+  // further ahead by asking L2 for the slabs (lanes 0 and 1, one page each per two-page iteration).
+  const int kPrefetch = prefetch_pages;
+  auto prefetch_page = [&](int pgi, int pid) {
+    if (pgi < pg_end && (unsigned)pid < (unsigned)p.num_pages) {
+      const size_t s = ((size_t)pid * p.Hkv + h) * kSlab;
+      l2_prefetch_slab(kpool + s);
+      l2_prefetch_slab(vpool + s);
+    }
+  };
+  if (STREAM && lane < kPrefetch) {   // kPrefetch <= 32
+    const int pgi = pg_first + 2 + lane;
+    if (pgi < pg_end) prefetch_page(pgi, __ldg(sp.pages + pgi));
+  }
   for (int pg = pg_first; pg < pg_end; pg += 2) {
     const bool has_b = pg + 1 < pg_end;
     int pid_next2 = 0;
+    const int pf_pg = pg + 2 + kPrefetch + (lane & 1);
+    int pf_pid = -1;
+    if (STREAM && pf_pg < pg_end) pf_pid = __ldg(sp.pages + pf_pg);   // used at the end of the iteration
     if (has_b) {
       const size_t s = slab_of(pid_next, hi_b);
       issue_loads<STREAM>(rb, kpool + s, vpool + s, gid, tig, pol);
@@ -217,6 +240,7 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
       }
       compute_page(st, rb, qf, sl2, (pg + 1) * kPage, hi_b, gid, tig);
     }
+    if (STREAM && lane < 2) prefetch_page(pf_pg, pf_pid);
   }
 
   float l0 = st.l0, l1 = st.l1;
@@ -249,6 +273,18 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
 
 }  // namespace
 
+// L2 prefetch distance of the suffix stream in pages (MC_SUFFIX_PREFETCH, default 2, 0 disables).
+static int suffix_prefetch_pages() {
+  static int v = -1;
+  if (v < 0) {
+    const char *e = std::getenv("MC_SUFFIX_PREFETCH");
+    v = e && *e ? std::atoi(e) : 2;
+    if (v < 0) v = 0;
+    if (v > 32) v = 32;
+  }
+  return v;
+}
+
 bool mma_supported(const Params &p, int dtype) { return dtype == MC_BF16 && p.d == 128 && p.g >= 1 && p.g <= 8; }
 
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
@@ -260,9 +296,9 @@ mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, fl
   const float sl2 = scale * kLog2e;
   const __nv_bfloat16 *qb = reinterpret_cast<const __nv_bfloat16 *>(q);
   if (mode == kPrefix)
-    attn_mma_kernel<kPrefix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part);
+    attn_mma_kernel<kPrefix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, 0);
   else
-    attn_mma_kernel<kSuffix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part);
+    attn_mma_kernel<kSuffix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, suffix_prefetch_pages());
   count_launch();
   return check_launch();
 }

@@ -6,13 +6,13 @@
 //     S = Q_s K^T          128 x 128 tile, tcgen05.mma, operands in shared memory, accumulator in TMEM
 //     P = exp2(S*c - m)    one thread per row reads its row of S from TMEM, writes bf16 P back to TMEM
 //     O += P V             tcgen05.mma, P from TMEM, V in its natural [token][d] layout (MN-major B operand)
-// K/V pages reach shared memory by TMA (one 16-token x 64-element box per page and head-dim half,
-// 128-byte swizzle) through a tensor map laid over the paged pool; the page id is a TMA coordinate.
+// K/V pages reach shared memory by TMA through tensor maps laid over the paged pools (the page id is a TMA
+// coordinate): V as one 4 KB box per page, K as two 2 KB boxes per page (one per 64-element d half).
 //
 // Work item = (group, kv head, prefix split, 128-row tile); persistent CTAs take items round-robin.
 // Warp roles: warp 0 issues the TMA copies and stages the next item's query tile, warp 1 lane 0 issues
-// the MMAs (warp 1 owns the TMEM allocation), warps 2-5 (128 threads, one per TMEM lane) do the softmax,
-// the rescale and the epilogue.
+// the MMAs (warp 1 owns the TMEM allocation), warps 2-9 (256 threads, two per TMEM lane, each owning
+// 64 of the tile's 128 columns) do the softmax, the rescale and the epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -26,19 +26,24 @@ constexpr int D = 128;
 constexpr int kTileM = 128;      // stacked query rows per tile
 constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
 constexpr int kPagesPerTile = kTileN / kPage;
-constexpr int kSlots = 5;         // ring of 32 KB operand slots: K(t), V(t), K(t+1), V(t+1), K(t+2)
-constexpr int kThreads = 192;
+constexpr int kKSlots = 3;        // K tiles in flight or in use (TMA, two 2 KB boxes per page: one per d half)
+constexpr int kVSlots = 2;        // V tiles (TMA, one 4 KB box per page)
+constexpr int kSoftmaxThreads = 256;   // two threads per row: columns [0,64) and [64,128)
+constexpr int kThreads = 64 + kSoftmaxThreads;
 constexpr uint32_t kHalfBytes = kTileN * 64 * 2;        // one head-dim (or token) half of a 128x128 bf16 tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;         // 32 KB
-constexpr uint32_t kBoxBytes = kPage * 64 * 2;          // one TMA box: 16 tokens x 64 elements
+constexpr uint32_t kPageBytes = kPage * D * 2;          // one (page, kv head) slab; one TMA box for V
 constexpr uint32_t kTmemCols = 512;                     // S: [0,128)  O: [128,256)  P (bf16 pairs): [256,320), [320,384)
 constexpr long long kWaitCycles = 2000000000ll;         // ~1 s
 
-struct __align__(1024) Smem {
+struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint8_t q[2][kTileBytes];           // stacked query tile of the current and of the next item
-  uint8_t ring[kSlots][kTileBytes];   // load u = 2*tile + (0: K, 1: V) goes to slot u % kSlots
-  uint64_t full[kSlots], empty[kSlots];
+  uint8_t k[kKSlots][kTileBytes];     // [d half][128 tokens][64], 128-byte swizzle
+  uint8_t v[kVSlots][kTileBytes];     // [page][d half][16 tokens][64], 128-byte swizzle
+  uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
   uint64_t q_ready[2], q_free[2], s_full, s_free, p_full, pv_done[2];
+  uint64_t pair[4];                   // the two warps that share a TMEM lane quadrant meet here
+  float xch[2][2][kTileM];            // [tile parity][column half][row]: row extremum / row sum exchange
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
   volatile int abort;
@@ -87,12 +92,23 @@ __device__ __forceinline__ uint64_t l2_keep_policy() {
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
   return pol;
 }
-__device__ __forceinline__ void tma_load_box(void *dst, const CUtensorMap *map, int x, int tok, int head, int page,
-                                             uint64_t *bar, uint64_t policy) {
+// One (page, kv head) slab of V: both 64-element halves of its 16 token rows, 4 KB, one box.
+__device__ __forceinline__ void tma_load_page(void *dst, const CUtensorMap *map, int head, int page, uint64_t *bar,
+                                              uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(0), "r"(0), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+// One d half (64 elements) of the 16 token rows of a (page, kv head) slab of K: 2 KB.  The swizzle span caps
+// a box at 64 elements per row, and the K-major operand wants each half's 128 token rows contiguous.
+__device__ __forceinline__ void tma_load_half_page(void *dst, const CUtensorMap *map, int x, int head, int page,
+                                                   uint64_t *bar, uint64_t policy) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%2, %3, %4, %5}], [%6], %7;\n"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(tok), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(0), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
 
@@ -213,27 +229,36 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
   return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
 }
 
-__global__ void __maxnreg__(168)
+__global__ void __maxnreg__(104)
 prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                  const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
                  float *__restrict__ lse_part, int n_items, int n_mt) {
-  extern __shared__ uint8_t smem_raw[];
-  Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
+  if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0) latch(p, MC_ERR_CUDA);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = p.g, cand_per_tile = kTileM / g;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&sm.full[s], 1);
-      mbar_init(&sm.empty[s], 1);
+    for (int s = 0; s < kKSlots; ++s) {
+      mbar_init(&sm.full_k[s], 1);
+      mbar_init(&sm.empty_k[s], 1);
+    }
+    for (int s = 0; s < kVSlots; ++s) {
+      mbar_init(&sm.full_v[s], 1);
+      mbar_init(&sm.empty_v[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm.q_ready[b], 32);
       mbar_init(&sm.q_free[b], 1);
     }
     mbar_init(&sm.s_full, 1);
-    mbar_init(&sm.s_free, 128);
-    mbar_init(&sm.p_full, 128);
+    mbar_init(&sm.s_free, kSoftmaxThreads);
+    mbar_init(&sm.p_full, kSoftmaxThreads);
+    for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[i], 64);
     mbar_init(&sm.pv_done[0], 1);
     mbar_init(&sm.pv_done[1], 1);
     sm.abort = 0;
@@ -258,9 +283,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
     // K/V: a tile is 32 TMA boxes (K and V, 8 pages, 2 head-dim halves), one per lane.
     // Q:   the stacked query tile of the NEXT item is staged (plain loads, swizzled stores) into the
     //      other Q buffer while the current item is being computed.
-    const int pg = lane & 7, hf = (lane >> 3) & 1, is_v = lane >> 4;
     const uint64_t policy = l2_keep_policy();
-    const CUtensorMap *map = is_v ? &v_map : &k_map;
     bool ok = true;
 
     auto next_item = [&](int from, Item &out) -> int {
@@ -322,23 +345,38 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
       int round = nxt_idx < n_items ? 0 : kQRounds + 1;   // staging state of the next item's query tile
       const int last_pg = (it.hi - 1) >> 4;
       for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
-        const uint32_t u = 2 * kt + is_v;           // lanes 0-15 load K(t), lanes 16-31 load V(t)
-        const int s = u % kSlots;
-        // pages past the end of the prefix repeat the last valid page: finite data, masked later
-        int pid = __ldg(it.pages + min((t0 >> 4) + pg, last_pg));
-        const bool in_range = t0 + pg * kPage < it.hi, good = (unsigned)pid < (unsigned)p.num_pages;
-        if (in_range && !good) latch(p, kDevBadPage);
+        // page ids of the tile's 8 pages (lane pg holds page pg); pages past the end of the prefix repeat the
+        // last valid page: finite data, masked later
+        int pid = __ldg(it.pages + min((t0 >> 4) + (lane & 7), last_pg));
+        const bool in_range = t0 + (lane & 7) * kPage < it.hi, good = (unsigned)pid < (unsigned)p.num_pages;
+        if (lane < 8 && in_range && !good) latch(p, kDevBadPage);
         if (!good) pid = 0;   // a bad page id is replaced by page 0 and its 16 columns are masked
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range && good) & 0xffu;
-        ok = mbar_wait(sm, p, &sm.empty[s], ((u / kSlots) & 1) ^ 1);
+        // ---- K(t): 16 boxes of 2 KB (lanes 0-15: page = lane & 7, d half = lane >> 3)
+        const int sk = kt % kKSlots;
+        ok = mbar_wait(sm, p, &sm.empty_k[sk], ((kt / kKSlots) & 1) ^ 1);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (lane == 0) mbar_expect_tx(&sm.full_k[sk], kTileBytes);
+        __syncwarp();
+        if (lane < 16)
+          tma_load_half_page(sm.k[sk] + (lane >> 3) * kHalfBytes + (lane & 7) * (kPageBytes / 2), &k_map, (lane >> 3) * 64,
+                             it.h, pid, &sm.full_k[sk], policy);
+        // ---- V(t): 8 boxes of 4 KB
+        const int sv = kt % kVSlots;
+        ok = mbar_wait(sm, p, &sm.empty_v[sv], ((kt / kVSlots) & 1) ^ 1);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         // published before the arrive below; the softmax role reads it after the chain of barrier waits
-        // (full -> first product -> s_full) that this arrive starts
-        if (lane == 0) sm.page_ok[kt & 7] = okmask;
-        if ((lane & 15) == 0) mbar_expect_tx(&sm.full[s], kTileBytes);
+        // (full -> second/first product -> s_full of a later tile is not enough: it is read after s_full of
+        // THIS tile, which follows full_k of this tile, announced by this warp after this store)
+        if (lane == 0) {
+          sm.page_ok[kt & 7] = okmask;
+          mbar_expect_tx(&sm.full_v[sv], kTileBytes);
+        }
         __syncwarp();
-        tma_load_box(sm.ring[s] + hf * kHalfBytes + pg * kBoxBytes, map, hf * 64, 0, it.h, pid, &sm.full[s], policy);
+        if (lane >= 16 && lane < 24)
+          tma_load_page(sm.v[sv] + (lane & 7) * kPageBytes, &v_map, it.h, pid, &sm.full_v[sv], policy);
         if (round <= kQRounds) {
           ok = q_step(nxt, it_n + 1, round);
           if (!ok) break;
@@ -368,34 +406,35 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         bool ok = true;
         for (int t = 0; t <= n_tiles && ok; ++t) {
           if (t < n_tiles) {
-            const uint32_t ktq = kt + t, u = 2 * ktq;
-            const int s = u % kSlots;
+            const uint32_t ktq = kt + t;
+            const int s = ktq % kKSlots;
             if (ktq > 0) ok = mbar_wait(sm, p, &sm.s_free, (ktq - 1) & 1);
-            ok = ok && mbar_wait(sm, p, &sm.full[s], (u / kSlots) & 1);
+            ok = ok && mbar_wait(sm, p, &sm.full_k[s], (ktq / kKSlots) & 1);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t k_addr = smem_u32(sm.ring[s]);
+            const uint32_t k_addr = smem_u32(sm.k[s]);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
               umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
             }
-            umma_commit(&sm.empty[s]);   // K(t) is free as soon as the first product has read it
+            umma_commit(&sm.empty_k[s]);   // K(t) is free as soon as the first product has read it
             umma_commit(&sm.s_full);
             if (t == n_tiles - 1) umma_commit(&sm.q_free[qb]);   // last reader of this item's Q tile
           }
           if (t > 0) {
-            const uint32_t ktp = kt + t - 1, u = 2 * ktp + 1;
-            const int s = u % kSlots;
-            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full[s], (u / kSlots) & 1);
+            const uint32_t ktp = kt + t - 1;
+            const int s = ktp % kVSlots;
+            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t v_addr = smem_u32(sm.ring[s]), p_cols = tmem_p + (ktp & 1) * (kTileN / 2);
+            const uint32_t v_addr = smem_u32(sm.v[s]), p_cols = tmem_p + (ktp & 1) * (kTileN / 2);
+            // one k-step per page: its 16 token rows x both 64-element halves (2 KB apart) are one 4 KB box
 #pragma unroll
             for (int kk = 0; kk < kTileN / 16; ++kk)
-              umma_ts(tmem_o, p_cols + kk * 8, smem_desc(v_addr + kk * 2048, kHalfBytes, 1024), kIdescPV,
+              umma_ts(tmem_o, p_cols + kk * 8, smem_desc(v_addr + kk * kPageBytes, kPageBytes / 2, 1024), kIdescPV,
                       (t > 1) || (kk > 0));
-            umma_commit(&sm.empty[s]);
+            umma_commit(&sm.empty_v[s]);
             umma_commit(&sm.pv_done[ktp & 1]);
           }
         }
@@ -404,10 +443,22 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
       }
     }
   } else {
-    // ---------------------------------------------------------------- softmax / epilogue (128 threads)
+    // ---------------------------------------------------------------- softmax / epilogue (256 threads)
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may access
+    const int half = (warp - 2) >> 2;          // which 64 of the tile's 128 columns this thread owns
     const int r = quad * 32 + lane;            // row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    uint32_t pair_n = 0;                       // completed meetings of this warp pair
+    // Exchanges one float with the thread that owns the other half of the row (bounded).
+    auto exchange = [&](float mine, float &theirs) -> bool {
+      sm.xch[pair_n & 1][half][r] = mine;
+      mbar_arrive(&sm.pair[quad]);
+      bool w = mbar_wait(sm, p, &sm.pair[quad], pair_n & 1);
+      w = __all_sync(0xffffffffu, w);
+      if (w) theirs = sm.xch[pair_n & 1][half ^ 1][r];
+      ++pair_n;
+      return w;
+    };
     for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
       const Item it = decode_item(p, item, n_mt);
       if (it.mt * cand_per_tile >= it.n_cand) continue;
@@ -416,14 +467,14 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
       const size_t slot = qrow * p.n_parts + it.sp;
       if (it.lo >= it.hi) {
-        if (row_ok) lse_part[slot] = -INFINITY;
+        if (row_ok && half == 0) lse_part[slot] = -INFINITY;
         continue;
       }
-      float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2)
+      float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2); l: this thread's columns only
       const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
       bool alive = true;
       for (int t = 0; t < n_tiles && alive; ++t, ++kt) {
-        const int t0 = it.lo + t * kTileN;
+        const int t0 = it.lo + t * kTileN, c0 = half * 64;
         alive = mbar_wait(sm, p, &sm.s_full, kt & 1);
         alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
         if (!alive) break;
@@ -431,20 +482,20 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
         const uint32_t page_ok = sm.page_ok[kt & 7];
         const bool full_tile = page_ok == 0xffu && t0 + kTileN <= it.hi;
-        // the whole row of S into registers, then S is free for the next tile's first product
-        uint32_t sv[4][32];
+        // this thread's half row of S into registers, then S is free for the next tile's first product
+        uint32_t sv[2][32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_addr + c * 32, sv[c]);
+        for (int c = 0; c < 2; ++c) tmem_ld32(tmem_s + lane_addr + c0 + c * 32, sv[c]);
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(&sm.s_free);
         if (!full_tile) {   // ragged tail or a bad page: masked scores become -inf (sl2 > 0) / +inf (sl2 < 0)
           const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < 2; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              const int col = c * 32 + i;
+              const int col = c0 + c * 32 + i;
               const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
               if (!ok) sv[c][i] = masked;
             }
@@ -452,23 +503,27 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         // row extremum of the raw scores; times sl2 it is the row maximum of the scaled scores
         float e4[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) e4[c] = __uint_as_float(sv[c][0]);
+        for (int c = 0; c < 4; ++c) e4[c] = __uint_as_float(sv[c & 1][c >> 1]);
         if (sl2 >= 0.f) {
 #pragma unroll
-          for (int i = 1; i < 32; ++i)
+          for (int i = 2; i < 32; i += 2)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) e4[c] = fmaxf(e4[c], __uint_as_float(sv[c][i]));
+            for (int c = 0; c < 4; ++c) e4[c] = fmaxf(e4[c], __uint_as_float(sv[c & 1][i + (c >> 1)]));
         } else {
 #pragma unroll
-          for (int i = 1; i < 32; ++i)
+          for (int i = 2; i < 32; i += 2)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) e4[c] = fminf(e4[c], __uint_as_float(sv[c][i]));
+            for (int c = 0; c < 4; ++c) e4[c] = fminf(e4[c], __uint_as_float(sv[c & 1][i + (c >> 1)]));
         }
-        const float ext = sl2 >= 0.f ? fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]))
-                                     : fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
+        float ext = sl2 >= 0.f ? fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]))
+                               : fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
+        float ext_other = ext;
+        alive = exchange(ext, ext_other);
+        if (!alive) break;
+        ext = sl2 >= 0.f ? fmaxf(ext, ext_other) : fminf(ext, ext_other);
         const float mx = (ext == INFINITY || ext == -INFINITY) ? -INFINITY : ext * sl2;   // all masked -> -inf
         // The running maximum moves only when the new one is clearly larger (2^8): P stays bounded by
-        // 2^8 and the accumulator in TMEM is rescaled rarely.
+        // 2^8 and the accumulator in TMEM is rescaled rarely.  Both threads of a row decide alike.
         float m_use = m;
         bool rescale = false;
         if (mx > m + 8.f) {
@@ -483,13 +538,13 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
           if (!alive) break;
           tc_fence_after();
 #pragma unroll 1
-          for (int c0 = 0; c0 < D; c0 += 32) {
+          for (int c = 0; c < 2; ++c) {   // this thread's 64 columns of O
             uint32_t v[32];
-            tmem_ld32(tmem_o + lane_addr + c0, v);
+            tmem_ld32(tmem_o + lane_addr + c0 + c * 32, v);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-            tmem_st32(tmem_o + lane_addr + c0, v);
+            tmem_st32(tmem_o + lane_addr + c0 + c * 32, v);
           }
           tmem_wait_st();
         }
@@ -504,48 +559,72 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
           if (!alive) break;
           tc_fence_after();
         }
-        const uint32_t p_cols = tmem_p + lane_addr + (kt & 1) * (kTileN / 2);
         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pw[32];                           // 64 tokens -> 32 packed columns
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {     // 64 tokens -> 32 packed columns
-          uint32_t pw[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int c = half * 2 + (j >> 4), i = (2 * j) & 31;
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][i]), sl2, neg_m));       // masked: exp2(-inf) = 0
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][i + 1]), sl2, neg_m));
-            lsum[j & 1] += p0;
-            lsum[2 + (j & 1)] += p1;
-            pw[j] = pack_bf16x2(p0, p1);
-          }
-          tmem_st32(p_cols + half * 32, pw);
+        for (int j = 0; j < 32; ++j) {
+          const int c = j >> 4, i = (2 * j) & 31;
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][i]), sl2, neg_m));       // masked: exp2(-inf) = 0
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][i + 1]), sl2, neg_m));
+          lsum[j & 1] += p0;
+          lsum[2 + (j & 1)] += p1;
+          pw[j] = pack_bf16x2(p0, p1);
         }
+        tmem_st32(tmem_p + lane_addr + (kt & 1) * (kTileN / 2) + half * 32, pw);
         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
         tmem_wait_st();
         tc_fence_before();
+        // p_full counts arrivals, not tiles: nobody may arrive for this tile while the previous tile's phase
+        // is still open (a thread that runs a whole tile ahead would complete it early).  The previous
+        // tile's second product having finished implies that its phase closed; normally it has long finished.
+        if (kt > 0) {
+          alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
+          alive = __all_sync(0xffffffffu, alive);
+          if (!alive) break;
+        }
         mbar_arrive(&sm.p_full);
       }
       if (!alive) break;
-      // epilogue: O / l -> o_part, lse
+      // epilogue: O / l -> o_part, lse (each thread writes its 64 columns; the row sum is the two halves')
+      float l_other = 0.f;
+      alive = exchange(l, l_other);
+      if (!alive) break;
+      const float l_row = l + l_other;
       alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
       if (!__all_sync(0xffffffffu, alive)) break;
       tc_fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      float *dst = o_part + slot * D;
+      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+      // Each thread holds 64 columns of ONE row; a store instruction issued like that touches 32 rows.  The
+      // 32x32 blocks are transposed across the warp first (lane j then holds column j of all 32 rows), so
+      // that every store instruction writes 128 contiguous bytes of one row.
+      const unsigned long long my_off = (unsigned long long)slot * D + half * 64;
+      const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_row > 0.f);
 #pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t v[32];
-        tmem_ld32(tmem_o + lane_addr + c0, v);
+        tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, v);
         tmem_wait_ld();
-        if (row_ok && l > 0.f) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 4)
-            *reinterpret_cast<float4 *>(dst + c0 + i) =
-                make_float4(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv,
-                            __uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * inv);
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) {
+          const bool up = (lane & s) != 0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (i & s) continue;
+            const uint32_t send = up ? v[i] : v[i | s];
+            const uint32_t got = __shfl_xor_sync(0xffffffffu, send, s);
+            if (up) v[i] = got; else v[i | s] = got;
+          }
+        }
+        // v[i] now is element (row i of this warp's 32 rows, column c*32 + lane)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const unsigned long long off = __shfl_sync(0xffffffffu, my_off, i);
+          if ((store_mask >> i) & 1u) o_part[off + c * 32 + lane] = __uint_as_float(v[i]);
         }
       }
-      if (row_ok) lse_part[slot] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+      if (row_ok && half == 0) lse_part[slot] = l_row > 0.f ? (m + log2f(l_row)) * kLn2 : -INFINITY;
       tc_fence_before();
     }
   }
@@ -568,7 +647,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv) {
+bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv, bool whole_page) {
   static EncodeTiledFn fn = nullptr;
   if (!fn) {
     void *sym = nullptr;
@@ -578,15 +657,26 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv)
       return false;
     fn = reinterpret_cast<EncodeTiledFn>(sym);
   }
-  // pool[page][head][token][d]: innermost first
-  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)kPage, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
-  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
-  const cuuint32_t box[4] = {64, (cuuint32_t)kPage, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
+  // pool[page][head][token][d] seen as [page][head][token][d half][64]; dimensions innermost first, with the
+  // half before the token so that a box lands as [d half][16 tokens][64 elements]
+  const cuuint64_t dims[5] = {64, (cuuint64_t)kPage, 2, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, 128, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)kPage, 2, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  if (!whole_page) {   // K: pool[page][head][token][d], one box = 64 elements x 16 tokens
+    const cuuint64_t dims4[4] = {(cuuint64_t)D, (cuuint64_t)kPage, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
+    const cuuint64_t strides4[3] = {(cuuint64_t)D * 2, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
+    const cuuint32_t box4[4] = {64, (cuuint32_t)kPage, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims4, strides4, box4, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(pool), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
 
 }  // namespace
 
@@ -604,8 +694,8 @@ bool prefix_tc_supported(const Params &p, int dtype) {
 // `max_group` is the largest number of candidates in one group.  Returns nullptr when unavailable.
 PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int max_ctas) {
   PrefixTcPlan *plan = new PrefixTcPlan();
-  if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv) ||
-      !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv)) {
+  if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
+      !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true)) {
     delete plan;
     return nullptr;
   }
@@ -619,7 +709,7 @@ PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int m
   if (rounds > 0) grid = (plan->n_items + rounds - 1) / rounds;
   plan->grid = grid < 1 ? 1 : grid;
   if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)(sizeof(Smem) + 1024)) != cudaSuccess) {
+                           (int)sizeof(Smem)) != cudaSuccess) {
     delete plan;
     return nullptr;
   }
@@ -630,7 +720,7 @@ void prefix_tc_plan_free(PrefixTcPlan *plan) { delete plan; }
 
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {
-  prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem) + 1024, stream>>>(
+  prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
       p, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
       plan->n_items, plan->n_mt);
   count_launch();
