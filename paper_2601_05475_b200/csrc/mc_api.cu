@@ -217,7 +217,7 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
     }
   }
   int tp = ((max_p + nsp - 1) / nsp + 127) / 128 * 128;
-  int ts = mc::pow2_floor(max_s / 16 > 256 ? max_s / 16 : 256);
+  int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
   if (ts > 4096) ts = 4096;
   if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0) tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;

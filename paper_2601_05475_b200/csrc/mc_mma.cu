@@ -162,19 +162,29 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
     h = (int)((item / p.B) % p.Hkv);
     part = (int)(item / ((long long)p.B * p.Hkv));
   }
+  // The item's first two page ids do not depend on the sequence length (only on the part index): their
+  // loads, the length's and the queries' are issued together instead of one after the other.  Entries of a
+  // page-table row beyond the sequence are read here but never used as page ids.
+  int pid_first = 0, pid_second = 0;
+  if (MODE == kSuffix) {
+    const int first_pg = part * (p.suffix_part_tokens >> 4);
+    const int32_t *row_pages = p.suffix_pages + (size_t)b * p.max_sp;
+    if (first_pg < p.max_sp) pid_first = __ldg(row_pages + first_pg);
+    if (first_pg + 1 < p.max_sp) pid_second = __ldg(row_pages + first_pg + 1);
+  }
+  uint32_t qf[4][4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (gid < p.g) v = __ldg(reinterpret_cast<const uint4 *>(q + ((size_t)b * p.Hq + (size_t)h * p.g + gid) * D) + tig + 4 * j);
+    qf[j][0] = v.x; qf[j][1] = v.y; qf[j][2] = v.z; qf[j][3] = v.w;
+  }
   const Span sp = resolve_span<MODE>(p, b, part);
   const int g = p.g;
   const size_t row0 = (size_t)b * p.Hq + (size_t)h * g;
   if (sp.lo >= sp.hi) {
     if (lane < g) lse_part[(row0 + lane) * p.n_parts + sp.part] = -INFINITY;
     return;
-  }
-  uint32_t qf[4][4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (gid < g) v = __ldg(reinterpret_cast<const uint4 *>(q + (row0 + gid) * D) + tig + 4 * j);
-    qf[j][0] = v.x; qf[j][1] = v.y; qf[j][2] = v.z; qf[j][3] = v.w;
   }
   State st;
   st.m0 = st.m1 = -INFINITY;
@@ -202,10 +212,11 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
   PageRegs ra, rb;
   int hi_a, hi_b = 0;
   {
-    const size_t s = slab_of(__ldg(sp.pages + pg_first), hi_a);
+    const size_t s = slab_of(MODE == kSuffix ? pid_first : __ldg(sp.pages + pg_first), hi_a);
     issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
   }
-  int pid_next = pg_first + 1 < pg_end ? __ldg(sp.pages + pg_first + 1) : 0;
+  int pid_next = 0;
+  if (pg_first + 1 < pg_end) pid_next = MODE == kSuffix ? pid_second : __ldg(sp.pages + pg_first + 1);
   // The register double buffer covers one page of latency; the stream from HBM is kept kPrefetch pages
   // further ahead by asking L2 for the slabs (lanes 0 and 1, one page each per two-page iteration).
   const int kPrefetch = prefetch_pages;

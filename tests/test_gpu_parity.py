@@ -192,6 +192,40 @@ def test_edge_shapes(case):
     dp.close()
 
 
+def test_rising_scores_force_accumulator_rescale():
+    """Keys whose scores grow by far more than 2^8 from one 128-token tile to the next: the tensor-core prefix
+    pass must rescale its running accumulator (and the other paths their online softmax) and still match."""
+    cfg = wl.Config("rising", "bf16", 1, 16, 64, 8, 128, ("fixed", 0), ("fixed", tuple([40] * 16)), permute_pages=True,
+                    seed=5)
+    hp = wl.make_host_problem(cfg, prefix_len=np.array([1100], dtype=np.int32))
+    # scale the logical keys tile by tile (x1, x6, x1, x14, ...) and rebuild the paged image from them
+    mult = np.ones(1100, dtype=np.float32)
+    for t, f in enumerate([1, 6, 1, 14, 3, 20, 2, 9, 1]):
+        mult[t * 128:(t + 1) * 128] = f
+    hp.k_prefix[0] = wl._round_to_dtype(cfg, hp.k_prefix[0] * mult[:, None, None])
+    wl._scatter(hp.k_pool, hp.tables.prefix_pages[0], hp.k_prefix[0], cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+@pytest.mark.parametrize("scale", [-0.09, 0.0, 0.5])
+def test_other_scales(scale):
+    """Negative scale (the row extremum is then a minimum), zero scale (uniform weights) and a large one."""
+    cfg = SMALL["cfg2s"]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp = DeviceProblem.from_host(hp)
+    o, lse = dp.decode(to_device(cfg, q), scale=scale)
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    o_ref, lse_ref = orc.decode_attention(q, hp.k_prefix, hp.v_prefix, hp.k_suffix, hp.v_suffix,
+                                          hp.tables.group_offsets.tolist(), scale)
+    check_close(cfg, o, lse, o_ref, lse_ref)
+    dp.close()
+
+
 def test_unequal_group_sizes():
     cfg = wl.Config("unequal", "bf16", 2, 2, 8, 2, 128, ("fixed", 0), ("fixed", (5, 40, 0, 100)), seed=4)
     hp = wl.make_host_problem(cfg, prefix_len=np.array([64, 200], dtype=np.int32))
