@@ -141,6 +141,26 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------------
+# multi-process aggregation (replicas only: no data-path collective; ranks only agree on the time)
+# ---------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group (identity when
+    no group is initialised).  The step time of the job is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(bytes_per_replica_step, ms_per_step, world):
+    """Whole-job metric of `world` independent replicas that each move bytes_per_replica_step per step."""
+    return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
+
+
+# ---------------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------------
 class ClockSampler:
@@ -247,7 +267,9 @@ def run_gpu(args):
         # bytes of the average timed step (suffixes grow by one token per step when appending)
         grow = (warmup + (steps + 1) / 2.0) * cfg.B * per_tok if appends else 0.0
         step_bytes = ub0["total"] + grow + (2 * cfg.B * cfg.Hkv * cfg.d * cfg.elem_bytes if appends else 0)
-        res = {"ms": ms, "bytes": step_bytes, "launches": launches, "clocks": clocks, "cfg": cfg}
+        res = {"ms": ms, "bytes": step_bytes, "launches": launches, "clocks": clocks, "cfg": cfg,
+               "prefix_ctas": int(dp.geom.prefix_ctas), "n_parts": int(dp.geom.n_parts),
+               "n_prefix_parts": int(dp.geom.n_prefix_parts)}
 
         # end to end through the host-buffer entry point: pinned host q / k_new / v_new in, o / lse out
         pin = lambda t: t.cpu().pin_memory()
@@ -309,19 +331,24 @@ def run_gpu(args):
                 others[name] = measure(name, args.steps, args.warmup, True)
 
     # max over ranks of the step time
-    ms = main["ms"]
-    e2e_ms = main["e2e_ms"]
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([main["ms"], main["e2e_ms"]], device="cuda")
 
     if rank == 0:
         cfg = main["cfg"]
         peaks, peak_kind = measured_peaks()
         peak = float(peaks["hbm_gbs"])
-        value = world * main["bytes"] / (ms * 1e-3) / 1e9
+        value = aggregate_value(main["bytes"], ms, world)
         suffix_gbs = main["suffix_bytes"] / (main["suffix_ms"] * 1e-3) / 1e9
+
+        def prefix_summary(r, pk):
+            tf = r["prefix_flops"] / (r["prefix_ms"] * 1e-3) / 1e12
+            ctas = r["prefix_ctas"]
+            peak = pk.get("bf16_tflops")
+            return {"kernel": "prefix_tc_kernel (tcgen05)" if ctas else "attn_mma_kernel<prefix>", "ms_alone": r["prefix_ms"],
+                    "ctas": ctas, "tflops": tf, "bf16_peak_tflops": peak,
+                    # the pass deliberately holds only `ctas` of the 148 SMs: utilisation of the SMs it holds
+                    "frac_of_bf16_peak_of_held_sms": (tf / (peak * ctas / 148.0)) if (peak and ctas) else None,
+                    "note": "timed alone; in a step it runs beside the suffix pass and is sized to finish under it"}
 
         def summary(r):
             gbs = r["bytes"] / (r["ms"] * 1e-3) / 1e9
@@ -332,6 +359,7 @@ def run_gpu(args):
                 out["suffix_gbs"] = round(r["suffix_bytes"] / (r["suffix_ms"] * 1e-3) / 1e9, 1)
                 out["prefix_ms"] = round(r["prefix_ms"], 5)
                 out["prefix_tflops"] = round(r["prefix_flops"] / (r["prefix_ms"] * 1e-3) / 1e12, 2)
+                out["prefix_ctas"] = r["prefix_ctas"]
             return out
 
         if args.cpu_baseline:
@@ -355,12 +383,7 @@ def run_gpu(args):
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": suffix_gbs / peak,
                          "frac_of_8tbs": suffix_gbs / NOMINAL_HBM_GBS, "traffic": suffix_traffic(main["suffix_bytes"]),
                          "kernel_ms": main["suffix_ms"], "algorithmic_bytes": main["suffix_bytes"]},
-            "prefix_pass": {"kernel": "prefix_tc_kernel (tcgen05)", "ms_alone": main["prefix_ms"],
-                            "tflops": main["prefix_flops"] / (main["prefix_ms"] * 1e-3) / 1e12,
-                            "bf16_peak_tflops": peaks.get("bf16_tflops"),
-                            "frac_of_bf16_peak": (main["prefix_flops"] / (main["prefix_ms"] * 1e-3) / 1e12 /
-                                                  peaks["bf16_tflops"]) if peaks.get("bf16_tflops") else None,
-                            "note": "runs beside the suffix pass on a CTA count sized to finish under it"},
+            "prefix_pass": prefix_summary(main, peaks),
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": "%d of %d (candidate, head) rows of %s, fp64 numpy, one thread per row"
                                        % (n_rows, cfg.B * cfg.Hq, cfg.name)},

@@ -94,6 +94,7 @@ typedef struct {
   int32_t prefix_part_tokens;    /* tokens per prefix split (multiple of 16) */
   int32_t suffix_part_tokens;    /* tokens per suffix chunk (multiple of 16) */
   int32_t head_dim;
+  int32_t prefix_ctas;           /* persistent CTAs of the tensor-core prefix pass; 0: that kernel is not used */
 } mc_part_geometry_t;
 
 /* Builds the layout object (step 1 of the path, the paged-KV layout): validates the descriptor, fixes

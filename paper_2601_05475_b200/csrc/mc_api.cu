@@ -289,6 +289,7 @@ mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry
   g->prefix_part_tokens = L->p.prefix_part_tokens;
   g->suffix_part_tokens = L->p.suffix_part_tokens;
   g->head_dim = L->p.d;
+  g->prefix_ctas = mc::prefix_tc_grid(L->tc_plan);
   return MC_OK;
 }
 

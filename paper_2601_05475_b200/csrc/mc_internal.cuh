@@ -93,6 +93,7 @@ struct PrefixTcPlan;
 bool prefix_tc_supported(const Params &p, int dtype);
 PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int max_ctas);
 void prefix_tc_plan_free(PrefixTcPlan *plan);
+int prefix_tc_grid(const PrefixTcPlan *plan);
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream);
 

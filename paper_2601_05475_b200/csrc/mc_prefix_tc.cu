@@ -717,6 +717,7 @@ PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int m
 }
 
 void prefix_tc_plan_free(PrefixTcPlan *plan) { delete plan; }
+int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
 
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {
