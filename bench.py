@@ -30,11 +30,11 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the dominant kernel relative to its algorithmic bytes, from the ncu capture summarised in
-# profiles/suffix_kernel_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch on cfg2; the traffic
+# profiles/kernels_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch on cfg2; the traffic
 # grows in proportion to the tokens streamed, so it is scaled by the units of the timed workload).  The ratio
 # is only reported while the kernel source still has the hash it had when the counters were taken.
-SUFFIX_TRAFFIC_RATIO = None
-SUFFIX_KERNEL_SHA1 = None
+SUFFIX_TRAFFIC_RATIO = 1.0208
+SUFFIX_KERNEL_SHA1 = "3395467429623323ca330a89b6fdb8e312fd3a04"
 
 
 def suffix_traffic(algorithmic_bytes):
