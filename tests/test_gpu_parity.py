@@ -334,3 +334,37 @@ def test_launch_counter_counts_kernels():
     dp.decode(to_device(cfg, wl.draw_q(cfg, 0)))
     assert mc.mc_launch_count() - n0 >= 3
     dp.close()
+
+
+def test_step_is_capturable_in_a_cuda_graph_and_replays_with_growing_lengths():
+    """append + decode enqueue only kernels, event records and stream waits, and read the lengths on the device:
+    one captured step can be replayed for consecutive decode steps."""
+    cfg = SMALL["cfg2s"]
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    q_buf = to_device(cfg, wl.draw_q(cfg, 0))
+    k_buf, v_buf = (to_device(cfg, x) for x in wl.draw_append(cfg, 1))
+    stream = torch.cuda.Stream()
+    # one eager step on the capture stream first (lazy module loading must not happen during capture)
+    with torch.cuda.stream(stream):
+        mc.mc_decode_attn(dp.layout, q_buf, cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes, stream.cuda_stream)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        mc.mc_kv_append(dp.layout, k_buf, v_buf, torch.cuda.current_stream().cuda_stream)
+        mc.mc_decode_attn(dp.layout, q_buf, cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes,
+                          torch.cuda.current_stream().cuda_stream)
+    for step in range(1, 4):
+        k_new, v_new = wl.draw_append(cfg, step)
+        q = wl.draw_q(cfg, step)
+        k_buf.copy_(to_device(cfg, k_new))
+        v_buf.copy_(to_device(cfg, v_new))
+        q_buf.copy_(to_device(cfg, q))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        hp.append(k_new, v_new)
+        check_close(cfg, dp.o, dp.lse, *oracle_full(hp, q))
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    np.testing.assert_array_equal(dp.suffix_len.cpu().numpy(), hp.suffix_len)
+    dp.close()
