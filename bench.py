@@ -242,9 +242,8 @@ def run_gpu(args):
         per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
 
         def step(i):
-            if appends:
-                mc.mc_kv_append(dp.layout, kv[i % 4][0], kv[i % 4][1], stream)
-            mc.mc_decode_attn(dp.layout, qs[i % 4], cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes, stream)
+            mc.mc_decode_step(dp.layout, kv[i % 4][0] if appends else None, kv[i % 4][1] if appends else None,
+                              qs[i % 4], cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes, stream)
 
         for i in range(warmup):
             step(i)

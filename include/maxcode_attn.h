@@ -144,6 +144,12 @@ mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const floa
 mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale,
                            void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
 
+/* One whole decode step with device-resident tensors: appends k_new/v_new (as mc_kv_append) and runs
+ * mc_decode_attn, scheduled so that the append, which only the suffix pass depends on, runs beside the start of
+ * the prefix pass.  k_new = v_new = NULL skips the append (then identical to mc_decode_attn). */
+mc_status_t mc_decode_step(mc_kv_layout_t *layout, const void *k_new, const void *v_new, const void *q,
+                           float scale, void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
+
 /* Same step for a caller that keeps its per-step tensors on the HOST: copies q (and, if k_new/v_new are
  * non-NULL, the appended token) host->device into the workspace, appends, runs mc_decode_attn, copies o
  * and lse device->host and synchronises `stream`.  Host pointers should be pinned for the copies to be

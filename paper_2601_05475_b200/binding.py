@@ -41,6 +41,8 @@ EXPORTS = {
     "mc_suffix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
     "mc_merge_lse": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "mc_decode_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "mc_decode_step": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_size_t,
+                                 c_void_p]),
     "mc_decode_step_host": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p,
                                       c_void_p, c_size_t, c_void_p]),
     "mc_decode_attn_static": (c_int32, [POINTER(LayoutDesc), c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -141,6 +143,11 @@ def mc_merge_lse(layout: int, o_part, lse_part, o, lse, stream: int = 0) -> None
 def mc_decode_attn(layout: int, q, scale: float, o, lse, ws, ws_bytes: int, stream: int = 0) -> None:
     _check(lib().mc_decode_attn(layout, _ptr(q), scale, _ptr(o), _ptr(lse), _ptr(ws), ws_bytes, stream),
            "mc_decode_attn")
+
+
+def mc_decode_step(layout: int, k_new, v_new, q, scale: float, o, lse, ws, ws_bytes: int, stream: int = 0) -> None:
+    _check(lib().mc_decode_step(layout, _ptr(k_new), _ptr(v_new), _ptr(q), scale, _ptr(o), _ptr(lse), _ptr(ws),
+                                ws_bytes, stream), "mc_decode_step")
 
 
 def mc_decode_step_host(layout: int, k_new_host, v_new_host, q_host, scale: float, o_host, lse_host, ws,

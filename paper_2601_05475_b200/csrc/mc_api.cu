@@ -358,12 +358,14 @@ mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const floa
   return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, reinterpret_cast<cudaStream_t>(stream));
 }
 
-mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, void *o, float *lse, void *ws,
-                           size_t ws_bytes, void *stream) {
+static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const void *v_new, const void *q,
+                               float scale, void *o, float *lse, void *ws, size_t ws_bytes, void *stream) {
   Layout *L = reinterpret_cast<Layout *>(layout);
   mc_status_t s = mc::check_q(L, q);
   if (s != MC_OK) return s;
   if (!o || !lse || !ws || !mc::aligned16(o)) return MC_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return MC_ERR_INVALID_ARG;
+  if (k_new && (!mc::aligned16(k_new) || !mc::aligned16(v_new))) return MC_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MC_ERR_INVALID_ARG;
   if (ws_bytes < L->ws_bytes) return MC_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -372,16 +374,28 @@ mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, v
   // The two passes write disjoint part slots and run side by side: the prefix pass (tensor-bound, a few
   // persistent CTAs per SM's shared memory) is launched first, on the caller's stream, so that its CTAs are
   // resident before the suffix pass (HBM-bound, thousands of short CTAs) floods the SMs from the handle's
-  // side stream.  The merge joins them.
+  // side stream.  The append touches only suffix pages and lengths, so it goes to the side stream too, in
+  // front of the suffix pass.  The merge joins the streams.
   if (cudaEventRecord(L->fork_ev, st) != cudaSuccess ||
       cudaStreamWaitEvent(L->side_stream, L->fork_ev, 0) != cudaSuccess)
     return MC_ERR_CUDA;
   if ((s = mc::run_pass(L, mc::kPrefix, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+  if (k_new && (s = mc_kv_append(layout, k_new, v_new, L->side_stream)) != MC_OK) return s;
   if ((s = mc::run_pass(L, mc::kSuffix, q, scale, o_part, lse_part, L->side_stream)) != MC_OK) return s;
   if (cudaEventRecord(L->join_ev, L->side_stream) != cudaSuccess ||
       cudaStreamWaitEvent(st, L->join_ev, 0) != cudaSuccess)
     return MC_ERR_CUDA;
   return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
+}
+
+mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, void *o, float *lse, void *ws,
+                           size_t ws_bytes, void *stream) {
+  return decode_impl(layout, nullptr, nullptr, q, scale, o, lse, ws, ws_bytes, stream);
+}
+
+mc_status_t mc_decode_step(mc_kv_layout_t *layout, const void *k_new, const void *v_new, const void *q, float scale,
+                           void *o, float *lse, void *ws, size_t ws_bytes, void *stream) {
+  return decode_impl(layout, k_new, v_new, q, scale, o, lse, ws, ws_bytes, stream);
 }
 
 mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, const void *v_new_host,
@@ -405,9 +419,10 @@ mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, 
     if (cudaMemcpyAsync(k_dev, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(v_dev, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return MC_ERR_CUDA;
-    if ((s = mc_kv_append(layout, k_dev, v_dev, stream)) != MC_OK) return s;
   }
-  if ((s = mc_decode_attn(layout, q_dev, scale, o_dev, lse_dev, ws, ws_bytes, stream)) != MC_OK) return s;
+  if ((s = mc_decode_step(layout, k_new_host ? k_dev : nullptr, k_new_host ? v_dev : nullptr, q_dev, scale, o_dev,
+                          lse_dev, ws, ws_bytes, stream)) != MC_OK)
+    return s;
   if (cudaMemcpyAsync(o_host, o_dev, q_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaMemcpyAsync(lse_host, lse_dev, rows * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess)

@@ -82,10 +82,15 @@ def test_append_sweep_matches_oracle_every_step(name):
     dp = DeviceProblem.from_host(hp)
     for step in range(1, cfg.append_steps + 1):
         k_new, v_new = wl.draw_append(cfg, step)
-        mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
-        hp.append(k_new, v_new)
         q = wl.draw_q(cfg, step)
-        o, lse = dp.decode(to_device(cfg, q))
+        if step % 2:                      # alternate the two ways of taking a step
+            mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
+            o, lse = dp.decode(to_device(cfg, q))
+        else:
+            mc.mc_decode_step(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new), to_device(cfg, q), cfg.scale,
+                              dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes)
+            o, lse = dp.o, dp.lse
+        hp.append(k_new, v_new)
         torch.cuda.synchronize()
         check_close(cfg, o, lse, *oracle_full(hp, q))
     assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
