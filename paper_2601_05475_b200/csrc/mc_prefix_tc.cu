@@ -41,7 +41,7 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint8_t k[kKSlots][kTileBytes];     // [d half][128 tokens][64], 128-byte swizzle
   uint8_t v[kVSlots][kTileBytes];     // [page][d half][16 tokens][64], 128-byte swizzle
   uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
-  uint64_t q_ready[2], q_free[2], s_full, s_free, p_full, pv_done[2];
+  uint64_t q_ready[2], q_free[2], s_full, s_free, p_full[2], pv_done[2];
   uint64_t pair[4];                   // the two warps that share a TMEM lane quadrant meet here
   float xch[2][2][kTileM];            // [tile parity][column half][row]: row extremum / row sum exchange
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
@@ -257,7 +257,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
     }
     mbar_init(&sm.s_full, 1);
     mbar_init(&sm.s_free, kSoftmaxThreads);
-    mbar_init(&sm.p_full, kSoftmaxThreads);
+    mbar_init(&sm.p_full[0], kSoftmaxThreads);
+    mbar_init(&sm.p_full[1], kSoftmaxThreads);
     for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[i], 64);
     mbar_init(&sm.pv_done[0], 1);
     mbar_init(&sm.pv_done[1], 1);
@@ -425,7 +426,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
           if (t > 0) {
             const uint32_t ktp = kt + t - 1;
             const int s = ktp % kVSlots;
-            ok = mbar_wait(sm, p, &sm.p_full, ktp & 1) && mbar_wait(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1);
+            ok = mbar_wait(sm, p, &sm.p_full[ktp & 1], (ktp >> 1) & 1) &&
+                 mbar_wait(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1);
             if (!ok) break;
             tc_fence_after();
             const uint32_t v_addr = smem_u32(sm.v[s]), p_cols = tmem_p + (ktp & 1) * (kTileN / 2);
@@ -552,13 +554,9 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         m = m_use;
         const float neg_m = m == -INFINITY ? 0.f : -m;
         // P goes to TMEM as the A operand of the second product: lane = row, one column per token pair.
-        // The buffer of this tile's parity was last read by the second product of tile kt-2.
-        if (kt >= 2) {
-          alive = mbar_wait(sm, p, &sm.pv_done[kt & 1], ((kt - 2) >> 1) & 1);
-          alive = __all_sync(0xffffffffu, alive);
-          if (!alive) break;
-          tc_fence_after();
-        }
+        // The buffer of this tile's parity was last read by the second product of tile kt-2, which the tensor
+        // pipe finished before this tile's first product (products complete in issue order), i.e. before the
+        // s_full wait above returned.
         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t pw[32];                           // 64 tokens -> 32 packed columns
 #pragma unroll
@@ -574,15 +572,11 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
         tmem_wait_st();
         tc_fence_before();
-        // p_full counts arrivals, not tiles: nobody may arrive for this tile while the previous tile's phase
-        // is still open (a thread that runs a whole tile ahead would complete it early).  The previous
-        // tile's second product having finished implies that its phase closed; normally it has long finished.
-        if (kt > 0) {
-          alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
-          alive = __all_sync(0xffffffffu, alive);
-          if (!alive) break;
-        }
-        mbar_arrive(&sm.p_full);
+        // p_full counts arrivals, not tiles, and a warp may run a whole tile ahead of a slow one: with a single
+        // barrier its arrival for tile t+1 would complete tile t's phase early.  Two barriers alternate by tile
+        // parity; an arrival for tile t+2 presupposes s_full(t+2), hence s_free(t+1) from every thread, and a
+        // thread arrives there only after its p_full arrival for tile t.
+        mbar_arrive(&sm.p_full[kt & 1]);
       }
       if (!alive) break;
       // epilogue: O / l -> o_part, lse (each thread writes its 64 columns; the row sum is the two halves')
