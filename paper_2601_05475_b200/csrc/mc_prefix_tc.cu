@@ -76,6 +76,7 @@ __device__ __forceinline__ bool mbar_wait(Smem &sm, const Params &p, uint64_t *b
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(32);   // a polling warp must not take issue slots from the softmax warps of its scheduler
     if (sm.abort) return false;
     if (clock64() - t0 > kWaitCycles) {
       sm.abort = 1;
