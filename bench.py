@@ -229,17 +229,19 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def measure(name, steps, warmup, want_kernel_split):
+    def measure(name, steps, warmup, want_kernel_split, outer=()):
         cfg = wl.CONFIGS[name]
         appends = cfg.append_steps > 0
         total_steps = 2 * (steps + warmup) + 8
-        dp = make_device_problem(cfg, headroom_tokens=total_steps + 1 if appends else 1)
+        dp = make_device_problem(cfg, headroom_tokens=total_steps + 1 if appends else 1, outer=outer)
         stream = torch.cuda.current_stream().cuda_stream
         qs = [device_q(cfg, i) for i in range(4)]
         kv = [device_append(cfg, i) for i in range(4)] if appends else None
         len0 = dp.suffix_len.clone()
         ub0 = wl.unique_bytes(cfg, dp.prefix_len.cpu().numpy(), len0.cpu().numpy())
         per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+        outer_tokens = sum(int(np.sum(lens)) for (_, lens) in outer)          # each outer token is unique once
+        ub0["total"] += outer_tokens * per_tok
 
         def step(i):
             mc.mc_decode_step(dp.layout, kv[i % 4][0] if appends else None, kv[i % 4][1] if appends else None,
@@ -314,9 +316,11 @@ def run_gpu(args):
                 res[fn_name + "_ms"] = k0.elapsed_time(k1) / steps
             cur = dp.suffix_len.cpu().numpy().astype(np.int64)
             res["suffix_bytes"] = float(cur.sum()) * per_tok
-            res["prefix_bytes"] = float(dp.prefix_len.cpu().numpy().astype(np.int64).sum()) * per_tok
-            res["prefix_flops"] = 4.0 * cfg.Hq * cfg.d * float(
-                (dp.prefix_len.cpu().numpy().astype(np.int64) * cfg.C).sum())
+            res["prefix_bytes"] = (float(dp.prefix_len.cpu().numpy().astype(np.int64).sum()) + outer_tokens) * per_tok
+            res["prefix_flops"] = 4.0 * cfg.Hq * cfg.d * (float(
+                (dp.prefix_len.cpu().numpy().astype(np.int64) * cfg.C).sum()) + sum(
+                float(np.sum(np.asarray(lens, dtype=np.int64) * np.diff(np.asarray(go, dtype=np.int64))))
+                for (go, lens) in outer))
         dp.close()
         del dp
         torch.cuda.empty_cache()
@@ -328,6 +332,9 @@ def run_gpu(args):
         for name in ("cfg2", "cfg3", "cfg4"):
             if name != args.workload:
                 others[name] = measure(name, args.steps, args.warmup, True)
+        # a cascade deeper than two levels: configuration 3 behind a 4096-token prompt shared by all 256 candidates
+        c3 = wl.CONFIGS["cfg3"]
+        others["cfg3+root4096"] = measure("cfg3", args.steps, args.warmup, True, outer=[([0, c3.B], [4096])])
 
     # max over ranks of the step time
     ms, e2e_ms = max_over_ranks([main["ms"], main["e2e_ms"]], device="cuda")

@@ -90,8 +90,8 @@ typedef struct {
 typedef struct {
   int32_t rows;                  /* B*Hq */
   int32_t n_parts;               /* part slots per row */
-  int32_t n_prefix_parts;
-  int32_t prefix_part_tokens;    /* tokens per prefix split (multiple of 16) */
+  int32_t n_prefix_parts;        /* prefix part slots of all cascade levels (base level first) */
+  int32_t prefix_part_tokens;    /* tokens per prefix split of the base level (multiple of 16) */
   int32_t suffix_part_tokens;    /* tokens per suffix chunk (multiple of 16) */
   int32_t head_dim;
   int32_t prefix_ctas;           /* persistent CTAs of the tensor-core prefix pass; 0: that kernel is not used */
@@ -103,6 +103,25 @@ typedef struct {
  * Returns MC_ERR_INVALID_ARG / MC_ERR_UNSUPPORTED / MC_ERR_OUT_OF_MEMORY / MC_ERR_CUDA on failure
  * (*out is then NULL). */
 mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *desc, mc_kv_layout_t **out);
+
+/* An outer level of a prefix cascade: token ranges shared by MORE candidates than the base descriptor's groups
+ * (e.g. a system prompt shared by every prompt group, in front of each group's own prefix).  Same pools, another
+ * group map: candidates group_offsets[j] .. group_offsets[j+1]-1 (contiguous in b) attend to pages[j][0 : len[j]].
+ * All pointers DEVICE memory, borrowed for the life of the handle. */
+typedef struct {
+  int32_t num_groups;            /* groups at this level, 1 <= num_groups <= B */
+  int32_t max_pages;             /* row stride of pages */
+  const int32_t *group_offsets;  /* device, [num_groups+1], increasing, last = B */
+  const int32_t *pages;          /* device, [num_groups][max_pages] */
+  const int32_t *len;            /* device, [num_groups], tokens */
+} mc_prefix_level_t;
+
+/* mc_kv_layout_create for a cascade deeper than two levels: every candidate attends to the tokens of each outer
+ * level's group it belongs to, to its base-level prefix and to its suffix (the order of concatenation does not
+ * change the result).  The prefix pass runs once per level, each level writes part slots of its own, the merge
+ * combines them all.  n_outer <= 3.  With n_outer = 0 this is mc_kv_layout_create. */
+mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *desc, const mc_prefix_level_t *outer,
+                                        int32_t n_outer, mc_kv_layout_t **out);
 
 /* Frees the handle and its device state.  NULL is accepted. */
 mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout);

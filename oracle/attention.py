@@ -132,3 +132,39 @@ def token_range_partial(q_row: np.ndarray, K: np.ndarray, V: np.ndarray, scale: 
     lo = max(0, lo)
     hi = max(lo, min(hi, K.shape[0]))
     return attend(q_row, K[lo:hi], V[lo:hi], scale)
+
+
+def decode_attention_cascade(q: np.ndarray,
+                             levels: Sequence[Tuple[Sequence[np.ndarray], Sequence[np.ndarray], Sequence[int]]],
+                             k_suffix: Sequence[np.ndarray], v_suffix: Sequence[np.ndarray], scale: float,
+                             kv_head_of: Optional[Callable[[int, int, int], int]] = None,
+                             rows: Optional[Sequence[Tuple[int, int]]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """One decode step when the shared history is a cascade of levels (a prefix tree deeper than two).
+
+    levels: list of (k_list, v_list, group_offsets), outermost first; level i gives every candidate of its
+    group j the rows k_list[j] [len][Hkv][d].  Candidate b's history is the concatenation of its group's rows at
+    every level followed by its private suffix; the result is attention over that whole history (the order of
+    concatenation does not matter).  With a single level this is `decode_attention`.
+    """
+    if kv_head_of is None:
+        kv_head_of = contiguous_kv_head
+    q = np.asarray(q)
+    B, Hq, d = q.shape
+    Hkv = k_suffix[0].shape[1]
+    group_of = []
+    for (_, _, go) in levels:
+        g_of = np.zeros(B, dtype=np.int64)
+        for j in range(len(go) - 1):
+            g_of[go[j]:go[j + 1]] = j
+        group_of.append(g_of)
+    o = np.full((B, Hq, d), np.nan, dtype=np.float64)
+    lse = np.full((B, Hq), np.nan, dtype=np.float64)
+    todo = rows if rows is not None else [(b, hq) for b in range(B) for hq in range(Hq)]
+    for (b, hq) in todo:
+        h = kv_head_of(hq, Hq, Hkv)
+        ks = [lv[0][int(group_of[i][b])][:, h, :] for i, lv in enumerate(levels)] + [k_suffix[b][:, h, :]]
+        vs = [lv[1][int(group_of[i][b])][:, h, :] for i, lv in enumerate(levels)] + [v_suffix[b][:, h, :]]
+        K = np.concatenate(ks, axis=0).astype(np.float64)
+        V = np.concatenate(vs, axis=0).astype(np.float64)
+        o[b, hq], lse[b, hq] = attend(q[b, hq], K, V, scale)
+    return o, lse

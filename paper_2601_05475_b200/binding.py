@@ -25,6 +25,11 @@ class LayoutDesc(ctypes.Structure):
                                         "suffix_pages", "suffix_len")]
 
 
+class PrefixLevel(ctypes.Structure):
+    _fields_ = [("num_groups", c_int32), ("max_pages", c_int32), ("group_offsets", c_void_p), ("pages", c_void_p),
+                ("len", c_void_p)]
+
+
 class PartGeometry(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in ("rows", "n_parts", "n_prefix_parts", "prefix_part_tokens",
                                        "suffix_part_tokens", "head_dim", "prefix_ctas")]
@@ -32,6 +37,7 @@ class PartGeometry(ctypes.Structure):
 
 EXPORTS = {
     "mc_kv_layout_create": (c_int32, [POINTER(LayoutDesc), POINTER(c_void_p)]),
+    "mc_kv_layout_create_cascade": (c_int32, [POINTER(LayoutDesc), POINTER(PrefixLevel), c_int32, POINTER(c_void_p)]),
     "mc_kv_layout_destroy": (c_int32, [c_void_p]),
     "mc_kv_layout_validate": (c_int32, [c_void_p, c_void_p, c_size_t, c_void_p]),
     "mc_kv_layout_geometry": (c_int32, [c_void_p, POINTER(PartGeometry)]),
@@ -103,6 +109,14 @@ def mc_launch_count() -> int:
 def mc_kv_layout_create(desc: LayoutDesc) -> int:
     h = c_void_p()
     _check(lib().mc_kv_layout_create(byref(desc), byref(h)), "mc_kv_layout_create")
+    return h.value
+
+
+def mc_kv_layout_create_cascade(desc: LayoutDesc, outer) -> int:
+    """`outer`: sequence of PrefixLevel (outer cascade levels, any order)."""
+    h = c_void_p()
+    arr = (PrefixLevel * max(1, len(outer)))(*outer)
+    _check(lib().mc_kv_layout_create_cascade(byref(desc), arr, len(outer), byref(h)), "mc_kv_layout_create_cascade")
     return h.value
 
 

@@ -9,6 +9,8 @@
 
 namespace mc {
 
+constexpr int kMaxOuterLevels = 3;
+
 struct Layout {
   mc_kv_layout_desc_t desc;
   Params p;
@@ -16,7 +18,10 @@ struct Layout {
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
-  PrefixTcPlan *tc_plan;      // non-null: the prefix pass runs on the tcgen05 kernel
+  PrefixTcPlan *tc_plan;      // non-null: the (innermost) prefix level runs on the tcgen05 kernel
+  int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
+  Params outer_p[kMaxOuterLevels];
+  PrefixTcPlan *outer_plan[kMaxOuterLevels];
   cudaStream_t side_stream;   // the suffix pass of mc_decode_attn runs here, beside the prefix pass
   cudaEvent_t fork_ev, join_ev;
 };
@@ -70,14 +75,14 @@ __global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__re
 // ------------------------------------------------------------------------------------------------
 // validation
 // ------------------------------------------------------------------------------------------------
-__global__ void validate_kernel(Params p, int32_t *refs) {
+__global__ void validate_kernel(Params p, int32_t *refs, int with_suffix) {
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   if (tid == 0) {
     if (__ldg(p.group_offsets) != 0 || __ldg(p.group_offsets + p.G) != p.B) latch(p, kDevBadPage);
     for (int j = 0; j < p.G; ++j)
       if (__ldg(p.group_offsets + j + 1) < __ldg(p.group_offsets + j)) latch(p, kDevBadPage);
   }
-  const long long np = (long long)p.G * p.max_pp, ns = (long long)p.B * p.max_sp;
+  const long long np = (long long)p.G * p.max_pp, ns = with_suffix ? (long long)p.B * p.max_sp : 0;
   for (long long i = tid; i < np + ns; i += nth) {
     int page, used;
     if (i < np) {
@@ -107,11 +112,70 @@ mc_status_t check_q(const Layout *L, const void *q) {
   return MC_OK;
 }
 
+mc_status_t run_level(Layout *L, const Params &p, const PrefixTcPlan *plan, int mode, const void *q, float scale,
+                      float *o_part, float *lse_part, cudaStream_t st) {
+  if (mode == kPrefix && plan && scale != 0.f) return launch_prefix_tc(p, plan, q, scale, o_part, lse_part, st);
+  if (L->use_mma) return launch_mma(p, mode, q, scale, o_part, lse_part, st);
+  return launch_fma(p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
+}
+
+// The prefix pass covers every level of the cascade (outermost first), the suffix pass the private tokens.
 mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t st) {
-  if (mode == kPrefix && L->tc_plan && scale != 0.f) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
-  if (L->use_mma) return launch_mma(L->p, mode, q, scale, o_part, lse_part, st);
-  return launch_fma(L->p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
+  if (mode == kPrefix) {
+    for (int k = L->n_outer - 1; k >= 0; --k) {
+      mc_status_t s = run_level(L, L->outer_p[k], L->outer_plan[k], kPrefix, q, scale, o_part, lse_part, st);
+      if (s != MC_OK) return s;
+    }
+  }
+  return run_level(L, L->p, L->tc_plan, mode, q, scale, o_part, lse_part, st);
+}
+
+// Splits and persistent-CTA count of one prefix level (see the comment in mc_kv_layout_create_cascade).
+struct LevelSizing { int nsp, ctas, max_group; };
+LevelSizing size_level(const Params &p, double suffix_us, int env_ctas) {
+  const int max_p = p.max_pp * kPage;
+  LevelSizing r;
+  r.max_group = (p.B + p.G - 1) / p.G;
+  const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
+  long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
+  double tiles = (double)pairs * ((max_p + 127) / 128);
+  int32_t *go = new (std::nothrow) int32_t[p.G + 1], *pl = new (std::nothrow) int32_t[p.G];
+  if (go && pl && cudaMemcpy(go, p.group_offsets, sizeof(int32_t) * (p.G + 1), cudaMemcpyDeviceToHost) == cudaSuccess &&
+      cudaMemcpy(pl, p.prefix_len, sizeof(int32_t) * p.G, cudaMemcpyDeviceToHost) == cudaSuccess) {
+    pairs = 0;
+    tiles = 0.0;
+    r.max_group = 1;
+    for (int j = 0; j < p.G; ++j) {
+      const int c = go[j + 1] - go[j];
+      if (c > r.max_group) r.max_group = c;
+      const long long pj = (long long)p.Hkv * ((c * p.g + 127) / 128);
+      pairs += pj;
+      tiles += (double)pj * ((pl[j] + 127) / 128);
+    }
+  }
+  (void)cudaGetLastError();
+  delete[] go;
+  delete[] pl;
+  if (pairs < 1) pairs = 1;
+  const double tile_us = 1.6, item_us = 6.0;                      // per 128x128 tile; per item
+  const double budget = suffix_us * 0.9, max_pair_tiles = (max_p + 127) / 128;
+  int nsp;
+  for (nsp = 1; nsp < 8; ++nsp)
+    if ((max_pair_tiles + nsp - 1) / nsp * tile_us + item_us <= budget) break;
+  if (budget < item_us + tile_us) nsp = (int)((160 + pairs - 1) / pairs);   // nothing to hide under: many items
+  if (nsp > 8) nsp = 8;
+  if (nsp < 1) nsp = 1;
+  r.nsp = nsp;
+  r.ctas = env_ctas;
+  if (r.ctas == 0) {
+    const double items = (double)pairs * nsp, avg_item_us = tiles / items * tile_us + item_us;
+    int rounds = (int)(0.7 * budget / avg_item_us);
+    if (rounds < 1) rounds = 1;
+    r.ctas = (int)((items + rounds - 1) / rounds);
+    if (r.ctas < 8) r.ctas = 8;
+  }
+  return r;
 }
 
 }  // namespace
@@ -137,6 +201,11 @@ const char *mc_status_string(mc_status_t s) {
 uint64_t mc_launch_count(void) { return mc::g_launches.load(std::memory_order_relaxed); }
 
 mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **out) {
+  return mc_kv_layout_create_cascade(d, nullptr, 0, out);
+}
+
+mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_prefix_level_t *outer, int32_t n_outer,
+                                        mc_kv_layout_t **out) {
   if (out) *out = nullptr;
   if (!d || !out) return MC_ERR_INVALID_ARG;
   if (d->num_groups < 1 || d->batch < 1 || d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_pages < 1 ||
@@ -147,6 +216,11 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
       !d->suffix_len)
     return MC_ERR_INVALID_ARG;
   if (!mc::aligned16(d->k_pool) || !mc::aligned16(d->v_pool)) return MC_ERR_INVALID_ARG;
+  if (n_outer < 0 || n_outer > mc::kMaxOuterLevels || (n_outer > 0 && !outer)) return MC_ERR_INVALID_ARG;
+  for (int k = 0; k < n_outer; ++k)
+    if (outer[k].num_groups < 1 || outer[k].num_groups > d->batch || outer[k].max_pages < 1 ||
+        !outer[k].group_offsets || !outer[k].pages || !outer[k].len)
+      return MC_ERR_INVALID_ARG;
   if (d->page_size != mc::kPage) return MC_ERR_UNSUPPORTED;
   if (d->dtype != MC_F32 && d->dtype != MC_BF16) return MC_ERR_UNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return MC_ERR_UNSUPPORTED;
@@ -155,6 +229,7 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   Layout *L = new (std::nothrow) Layout();
   if (!L) return MC_ERR_OUT_OF_MEMORY;
   L->desc = *d;
+  L->n_outer = n_outer;
   mc::Params &p = L->p;
   p.k_pool = d->k_pool; p.v_pool = d->v_pool;
   p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
@@ -162,71 +237,60 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   p.G = d->num_groups; p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.d = d->head_dim;
   p.g = d->num_q_heads / d->num_kv_heads;
   p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
+  for (int k = 0; k < n_outer; ++k) {   // an outer level is the same cache seen through another group map
+    mc::Params &po = L->outer_p[k];
+    po = p;
+    po.G = outer[k].num_groups;
+    po.group_offsets = outer[k].group_offsets;
+    po.prefix_pages = outer[k].pages;
+    po.prefix_len = outer[k].len;
+    po.max_pp = outer[k].max_pages;
+  }
 
-  // Part geometry from the table strides (the lengths themselves live on the device and may grow).
-  const int max_p = d->max_prefix_pages * mc::kPage, max_s = d->max_suffix_pages * mc::kPage;
-  // Prefix splits and the number of persistent CTAs of the tensor-core prefix pass are sized together, once,
-  // from the lengths as they are now.  The prefix pass should finish inside the suffix pass's HBM time while
-  // holding as few SMs as possible (an SM it holds runs the suffix pass at half occupancy), and every work
+  // Part geometry.  Suffix chunks come from the table stride (the lengths live on the device and may grow).
+  // Prefix splits and the number of persistent CTAs of the tensor-core prefix pass are sized together, once per
+  // level, from the lengths as they are now.  The prefix pass should finish inside the suffix pass's HBM time
+  // while holding as few SMs as possible (an SM it holds runs the suffix pass at half occupancy), and every work
   // item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be long: as few
   // splits as still let one item fit the time budget.  Constants are measured for this kernel pair.
-  int nsp = 0, tc_ctas = mc::env_int("MC_PREFIX_CTAS", 0), max_group = (p.B + p.G - 1) / p.G;
+  const int max_s = d->max_suffix_pages * mc::kPage;
+  double suffix_us = 0.0;
   {
-    const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
-    long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
-    double tiles = (double)pairs * ((max_p + 127) / 128), suffix_us = 0.0;
-    int32_t *go = new (std::nothrow) int32_t[p.G + 1], *pl = new (std::nothrow) int32_t[p.G];
     int32_t *sl = new (std::nothrow) int32_t[p.B];
-    const size_t eb = d->dtype == MC_F32 ? 4 : 2;
-    if (go && pl && sl &&
-        cudaMemcpy(go, d->group_offsets, sizeof(int32_t) * (p.G + 1), cudaMemcpyDeviceToHost) == cudaSuccess &&
-        cudaMemcpy(pl, d->prefix_len, sizeof(int32_t) * p.G, cudaMemcpyDeviceToHost) == cudaSuccess &&
-        cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
-      pairs = 0;
-      tiles = 0.0;
-      max_group = 1;
-      for (int j = 0; j < p.G; ++j) {
-        const int c = go[j + 1] - go[j];
-        if (c > max_group) max_group = c;
-        const long long pj = (long long)p.Hkv * ((c * p.g + 127) / 128);
-        pairs += pj;
-        tiles += (double)pj * ((pl[j] + 127) / 128);
-      }
+    if (sl && cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
       double suffix_tokens = 0.0;
       for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
-      suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * eb / 6.8e6;   // the stream runs at about 6.8 TB/s
+      suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : 2) / 6.8e6;   // stream at ~6.8 TB/s
     }
     (void)cudaGetLastError();
-    delete[] go;
-    delete[] pl;
     delete[] sl;
-    if (pairs < 1) pairs = 1;
-    const double tile_us = 1.6, item_us = 6.0;                      // per 128x128 tile; per item
-    const double budget = suffix_us * 0.9, max_pair_tiles = (max_p + 127) / 128;
-    for (nsp = 1; nsp < 8; ++nsp)
-      if ((max_pair_tiles + nsp - 1) / nsp * tile_us + item_us <= budget) break;
-    if (budget < item_us + tile_us) nsp = (int)((160 + pairs - 1) / pairs);   // nothing to hide under: many items
-    if (nsp > 8) nsp = 8;
-    if (nsp < 1) nsp = 1;
-    if (tc_ctas == 0) {
-      const double items = (double)pairs * nsp, avg_item_us = tiles / items * tile_us + item_us;
-      int rounds = (int)(0.7 * budget / avg_item_us);
-      if (rounds < 1) rounds = 1;
-      tc_ctas = (int)((items + rounds - 1) / rounds);
-      if (tc_ctas < 8) tc_ctas = 8;
-    }
   }
-  int tp = ((max_p + nsp - 1) / nsp + 127) / 128 * 128;
   int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
   if (ts > 4096) ts = 4096;
-  if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0) tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
-  if (tp < mc::kPage) tp = mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
-  p.prefix_part_tokens = tp;
-  p.suffix_part_tokens = ts;
-  p.n_prefix_parts = (max_p + tp - 1) / tp;
-  p.n_parts = p.n_prefix_parts + (max_s + ts - 1) / ts;
+  mc::LevelSizing sizing[1 + mc::kMaxOuterLevels];
+  int part_base = 0;
+  for (int k = 0; k <= n_outer; ++k) {   // k = 0: the base level; part slots in this order, then the suffix chunks
+    mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
+    sizing[k] = mc::size_level(pk, suffix_us, mc::env_int("MC_PREFIX_CTAS", 0));
+    const int max_p = pk.max_pp * mc::kPage;
+    int tp = ((max_p + sizing[k].nsp - 1) / sizing[k].nsp + 127) / 128 * 128;
+    if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0)
+      tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
+    if (tp < mc::kPage) tp = mc::kPage;
+    pk.prefix_part_tokens = tp;
+    pk.n_prefix_parts = (max_p + tp - 1) / tp;
+    pk.prefix_part_base = part_base;
+    part_base += pk.n_prefix_parts;
+  }
+  const int n_parts = part_base + (max_s + ts - 1) / ts;
+  for (int k = 0; k <= n_outer; ++k) {
+    mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
+    pk.suffix_part_tokens = ts;
+    pk.suffix_part_base = part_base;
+    pk.n_parts = n_parts;
+  }
   L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
 
   const size_t rows = (size_t)p.B * p.Hq, e = d->dtype == MC_F32 ? 4 : 2;
@@ -247,14 +311,22 @@ mc_status_t mc_kv_layout_create(const mc_kv_layout_desc_t *d, mc_kv_layout_t **o
   }
   *L->host_status = 0;
   p.status = L->dev_status;
+  for (int k = 0; k < n_outer; ++k) L->outer_p[k].status = L->dev_status;
 
-  // Tensor-core prefix pass: tensor maps over the pools and the persistent grid.
+  // Tensor-core prefix pass: tensor maps over the pools and the persistent grid of each level.
   L->tc_plan = nullptr;
-  if (mc::prefix_tc_supported(p, d->dtype) && mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0)) {
+  if (mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0)) {
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && max_group <= p.B)
-      L->tc_plan = mc::prefix_tc_plan(p, max_group, sms, tc_ctas > sms ? sms : tc_ctas);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
+      for (int k = 0; k <= n_outer; ++k) {
+        const mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
+        mc::PrefixTcPlan *plan = nullptr;
+        if (mc::prefix_tc_supported(pk, d->dtype) && sizing[k].max_group <= p.B)
+          plan = mc::prefix_tc_plan(pk, sizing[k].max_group, sms, sizing[k].ctas > sms ? sms : sizing[k].ctas);
+        if (k == 0) L->tc_plan = plan; else L->outer_plan[k - 1] = plan;
+      }
+    }
     (void)cudaGetLastError();
   }
   if (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -274,6 +346,7 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   if (L->fork_ev) cudaEventDestroy(L->fork_ev);
   if (L->join_ev) cudaEventDestroy(L->join_ev);
   mc::prefix_tc_plan_free(L->tc_plan);
+  for (int k = 0; k < L->n_outer; ++k) mc::prefix_tc_plan_free(L->outer_plan[k]);
   cudaFree(L->dev_status);
   cudaFreeHost(L->host_status);
   delete L;
@@ -285,7 +358,7 @@ mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry
   if (!L || !g) return MC_ERR_INVALID_ARG;
   g->rows = L->p.B * L->p.Hq;
   g->n_parts = L->p.n_parts;
-  g->n_prefix_parts = L->p.n_prefix_parts;
+  g->n_prefix_parts = L->p.suffix_part_base;   // all prefix levels together (base level first)
   g->prefix_part_tokens = L->p.prefix_part_tokens;
   g->suffix_part_tokens = L->p.suffix_part_tokens;
   g->head_dim = L->p.d;
@@ -316,8 +389,12 @@ mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t 
   if (scratch_bytes < (size_t)L->p.num_pages * sizeof(int32_t)) return MC_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(scratch, 0, (size_t)L->p.num_pages * sizeof(int32_t), st) != cudaSuccess) return MC_ERR_CUDA;
-  mc::validate_kernel<<<148, 256, 0, st>>>(L->p, reinterpret_cast<int32_t *>(scratch));
+  mc::validate_kernel<<<148, 256, 0, st>>>(L->p, reinterpret_cast<int32_t *>(scratch), 1);
   mc::count_launch();
+  for (int k = 0; k < L->n_outer; ++k) {   // outer levels: their own prefix tables, same reference counts
+    mc::validate_kernel<<<148, 256, 0, st>>>(L->outer_p[k], reinterpret_cast<int32_t *>(scratch), 0);
+    mc::count_launch();
+  }
   if (mc::check_launch() != MC_OK) return MC_ERR_CUDA;
   return mc_get_last_status(layout, stream);
 }

@@ -53,7 +53,7 @@ attn_fma_kernel(Params p, const T *__restrict__ q, float scale_log2, float *__re
                 float *__restrict__ lse_part) {
   constexpr int VEC = D / 32;
   const int lane = threadIdx.x & 31;
-  const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.n_prefix_parts;
+  const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hq * nparts_mode;
   const long long item = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
   if (item >= n_items) return;
@@ -141,7 +141,7 @@ attn_fma_kernel(Params p, const T *__restrict__ q, float scale_log2, float *__re
 template <typename T, int D>
 mc_status_t launch_t(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t stream) {
-  const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.n_prefix_parts;
+  const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hq * nparts_mode;
   if (n_items == 0) return MC_OK;
   const unsigned grid = (unsigned)((n_items + kWarpsPerBlock - 1) / kWarpsPerBlock);

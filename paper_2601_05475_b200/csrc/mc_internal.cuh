@@ -23,7 +23,10 @@ struct Params {
   const int32_t *group_offsets, *prefix_pages, *prefix_len, *suffix_pages, *suffix_len;
   int32_t G, B, Hq, Hkv, d, g;
   int32_t num_pages, max_pp, max_sp;
-  int32_t n_parts, n_prefix_parts, prefix_part_tokens, suffix_part_tokens;
+  int32_t n_parts;                                   // part slots per row (all prefix levels + suffix chunks)
+  int32_t n_prefix_parts, prefix_part_base;          // this prefix level's splits and its first part slot
+  int32_t suffix_part_base;                          // first part slot of the suffix chunks
+  int32_t prefix_part_tokens, suffix_part_tokens;
   int32_t *status;
 };
 
@@ -57,13 +60,13 @@ __device__ __forceinline__ Span resolve_span(const Params &p, int b, int part) {
     len = __ldg(p.prefix_len + j);
     cap = p.max_pp * kPage;
     tokens = p.prefix_part_tokens;
-    s.part = part;
+    s.part = p.prefix_part_base + part;
   } else {
     s.pages = p.suffix_pages + (size_t)b * p.max_sp;
     len = __ldg(p.suffix_len + b);
     cap = p.max_sp * kPage;
     tokens = p.suffix_part_tokens;
-    s.part = p.n_prefix_parts + part;
+    s.part = p.suffix_part_base + part;
   }
   if (len > cap || len < 0) {  // a length the table cannot hold: clamp and report
     latch(p, kDevBadPage);

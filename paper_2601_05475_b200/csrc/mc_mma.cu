@@ -148,7 +148,7 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
                 float *__restrict__ lse_part, int prefetch_pages) {
   constexpr bool STREAM = MODE == kSuffix;  // private suffix data is read exactly once
   const int lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
-  const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.n_prefix_parts;
+  const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
   const long long item = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
   if (item >= n_items) return;
@@ -300,7 +300,7 @@ bool mma_supported(const Params &p, int dtype) { return dtype == MC_BF16 && p.d 
 
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
                        cudaStream_t stream) {
-  const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.n_prefix_parts;
+  const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
   if (n_items == 0) return MC_OK;
   const unsigned grid = (unsigned)((n_items + kWarps - 1) / kWarps);

@@ -468,7 +468,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
-      const size_t slot = qrow * p.n_parts + it.sp;
+      const size_t slot = qrow * p.n_parts + p.prefix_part_base + it.sp;
       if (it.lo >= it.hi) {
         if (row_ok && half == 0) lse_part[slot] = -INFINITY;
         continue;

@@ -88,6 +88,8 @@ mc_status_t mc_decode_attn_static(const mc_kv_layout_desc_t *d, const void *q, f
   const size_t l_bytes = mc::align_up((size_t)rows * n_parts * sizeof(float), 256);
   if (mc::kStatusBytes + o_bytes + l_bytes > mc::kStaticScratchBytes) return MC_ERR_WORKSPACE_TOO_SMALL;
   p.n_prefix_parts = (int)n_prefix;
+  p.prefix_part_base = 0;
+  p.suffix_part_base = (int)n_prefix;
   p.n_parts = (int)n_parts;
 
   unsigned char *scratch = nullptr;

@@ -31,7 +31,7 @@ class DeviceProblem:
     """Pools, tables and lengths on the device plus the library's layout handle and workspace."""
 
     def __init__(self, cfg: wl.Config, tables: wl.PageTables, prefix_len: np.ndarray, suffix_len: np.ndarray,
-                 k_pool: torch.Tensor, v_pool: torch.Tensor, device="cuda"):
+                 k_pool: torch.Tensor, v_pool: torch.Tensor, device="cuda", outer=()):
         self.cfg, self.tables, self.device = cfg, tables, device
         self.k_pool, self.v_pool = k_pool, v_pool
         i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
@@ -48,7 +48,16 @@ class DeviceProblem:
         d.prefix_len, d.suffix_pages = self.prefix_len.data_ptr(), self.suffix_pages.data_ptr()
         d.suffix_len = self.suffix_len.data_ptr()
         self.desc = d
-        self.layout = mc.mc_kv_layout_create(d)
+        # outer cascade levels: (group_offsets, lengths, pages) numpy triples
+        self.outer_tensors, levels = [], []
+        for (go, ln, pg) in outer:
+            t = (i32(go), i32(ln), i32(pg))
+            self.outer_tensors.append(t)
+            lv = mc.PrefixLevel()
+            lv.num_groups, lv.max_pages = len(ln), pg.shape[1]
+            lv.group_offsets, lv.len, lv.pages = t[0].data_ptr(), t[1].data_ptr(), t[2].data_ptr()
+            levels.append(lv)
+        self.layout = mc.mc_kv_layout_create_cascade(d, levels) if levels else mc.mc_kv_layout_create(d)
         self.geom = mc.mc_kv_layout_geometry(self.layout)
         self.ws_bytes = mc.mc_workspace_bytes(self.layout)
         self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=device)
@@ -60,7 +69,8 @@ class DeviceProblem:
     @classmethod
     def from_host(cls, hp: wl.HostProblem, device="cuda") -> "DeviceProblem":
         return cls(hp.cfg, hp.tables, hp.prefix_len, hp.suffix_len,
-                   storage_to_device(hp.cfg, hp.k_pool, device), storage_to_device(hp.cfg, hp.v_pool, device), device)
+                   storage_to_device(hp.cfg, hp.k_pool, device), storage_to_device(hp.cfg, hp.v_pool, device), device,
+                   outer=[(lv.group_offsets, lv.length, lv.pages) for lv in hp.outer])
 
     def new_parts(self):
         g = self.geom
@@ -85,12 +95,23 @@ class DeviceProblem:
             pass
 
 
-def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, device="cuda") -> DeviceProblem:
+def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, device="cuda", outer=()
+                        ) -> DeviceProblem:
     """Full-size instance whose pools are drawn on the device (torch's seeded generator) instead of being
     built on the host: lengths and page tables come from `workload`, every slot of both pools is N(0,1)
     rounded to the storage dtype, and K rows are turned into outliers with the configured probability."""
     prefix_len, suffix_len = wl.draw_lengths(cfg)
     tables = wl.build_page_tables(cfg, prefix_len, suffix_len, headroom_tokens)
+    # outer cascade levels ((group_offsets, lengths) pairs) get fresh pages at the end of the pools
+    outer_np = []
+    for (go, lens) in outer:
+        lens = np.asarray(lens, dtype=np.int32)
+        npp = (lens.astype(np.int64) + wl.PAGE - 1) // wl.PAGE
+        pages = np.full((len(lens), max(1, int(npp.max(initial=0)))), -1, dtype=np.int32)
+        for j in range(len(lens)):
+            pages[j, :int(npp[j])] = np.arange(tables.num_pages, tables.num_pages + int(npp[j]), dtype=np.int32)
+            tables.num_pages += int(npp[j])
+        outer_np.append((np.asarray(go, dtype=np.int32), lens, pages))
     tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
     gen = torch.Generator(device=device)
     gen.manual_seed(cfg.seed * 1000003 + 17)
@@ -105,7 +126,9 @@ def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, d
         if cfg.k_outlier_prob > 0.0:
             mask = torch.rand((hi - lo, cfg.Hkv, wl.PAGE, 1), device=device, generator=gen) < cfg.k_outlier_prob
             k_pool[lo:hi] = torch.where(mask, k_pool[lo:hi] * cfg.k_outlier_scale, k_pool[lo:hi])
-    return DeviceProblem(cfg, tables, prefix_len, suffix_len, k_pool, v_pool, device)
+    dp = DeviceProblem(cfg, tables, prefix_len, suffix_len, k_pool, v_pool, device, outer=outer_np)
+    dp.outer_np = outer_np
+    return dp
 
 
 def device_q(cfg: wl.Config, step: int, device="cuda") -> torch.Tensor:
@@ -130,10 +153,15 @@ def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int
     j = int(np.searchsorted(dp.tables.group_offsets, b, side="right") - 1)
     P = int(dp.prefix_len[j].item())
     s = int(dp.suffix_len[b].item()) if suffix_len_now is None else suffix_len_now
+    segments = []
+    for (go, lens, pages) in getattr(dp, "outer_np", []):
+        jo = int(np.searchsorted(go, b, side="right") - 1)
+        segments.append((pages[jo], int(lens[jo])))
+    segments += [(dp.tables.prefix_pages[j], P), (dp.tables.suffix_pages[b], s)]
     out = []
     for pool in (dp.k_pool, dp.v_pool):
         parts = []
-        for pages_row, n in ((dp.tables.prefix_pages[j], P), (dp.tables.suffix_pages[b], s)):
+        for pages_row, n in segments:
             n_pages = (n + wl.PAGE - 1) // wl.PAGE
             if n_pages:
                 ids = torch.from_numpy(np.ascontiguousarray(pages_row[:n_pages], dtype=np.int64)).to(pool.device)

@@ -270,6 +270,7 @@ class HostProblem:
     v_suffix: List[np.ndarray]
     k_pool: np.ndarray              # [num_pages][Hkv][16][d] storage dtype
     v_pool: np.ndarray
+    outer: List["HostLevel"] = dataclasses.field(default_factory=list)   # outer cascade levels, if any
 
     def group_of(self, b: int) -> int:
         return int(np.searchsorted(self.tables.group_offsets, b, side="right") - 1)
@@ -281,6 +282,52 @@ class HostProblem:
             self.k_suffix[b] = np.concatenate([self.k_suffix[b], k_new[b][None]], axis=0)
             self.v_suffix[b] = np.concatenate([self.v_suffix[b], v_new[b][None]], axis=0)
         self.suffix_len = self.suffix_len + 1
+
+
+@dataclasses.dataclass
+class HostLevel:
+    """One outer level of a prefix cascade: token ranges shared by more candidates than the base groups."""
+    group_offsets: np.ndarray       # int32 [n_groups+1], candidates contiguous in b
+    length: np.ndarray              # int32 [n_groups]
+    pages: np.ndarray               # int32 [n_groups][max_pages]
+    k: List[np.ndarray]             # per outer group [len][Hkv][d] float32
+    v: List[np.ndarray]
+
+
+def add_outer_level(hp: "HostProblem", group_offsets: Sequence[int], lengths: Sequence[int], level_index: int = 0
+                    ) -> HostLevel:
+    """Appends an outer cascade level to a host problem: draws its K/V, gives it fresh pages at the end of the
+    pools (permuted among themselves when the configuration permutes pages) and scatters them in."""
+    cfg = hp.cfg
+    lengths = np.asarray(lengths, dtype=np.int32)
+    go = np.asarray(group_offsets, dtype=np.int32)
+    n_groups = len(lengths)
+    npp = (lengths.astype(np.int64) + PAGE - 1) // PAGE
+    first = hp.k_pool.shape[0]
+    extra = int(npp.sum())
+    ids = np.arange(first, first + extra, dtype=np.int32)
+    if cfg.permute_pages:
+        ids = ids[_rng(cfg.seed, _T_PERM, 100 + level_index).permutation(extra)]
+    fill = storage_array(cfg, np.full(1, SENTINEL, dtype=np.float32))[0]
+    pad = np.full((extra,) + hp.k_pool.shape[1:], fill, dtype=hp.k_pool.dtype)
+    hp.k_pool = np.concatenate([hp.k_pool, pad], axis=0)
+    hp.v_pool = np.concatenate([hp.v_pool, pad.copy()], axis=0)
+    hp.tables.num_pages = first + extra
+    max_pages = max(1, int(npp.max(initial=0)))
+    pages = np.full((n_groups, max_pages), -1, dtype=np.int32)
+    ks, vs, cur = [], [], 0
+    for j in range(n_groups):
+        n = int(npp[j])
+        pages[j, :n] = ids[cur:cur + n]
+        cur += n
+        ks.append(_draw_k(cfg, _T_KP, 1000 * (level_index + 1) + j, int(lengths[j])))
+        vs.append(_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_VP, 1000 * (level_index + 1) + j),
+                                               (int(lengths[j]), cfg.Hkv, cfg.d))))
+        _scatter(hp.k_pool, pages[j], ks[j], cfg)
+        _scatter(hp.v_pool, pages[j], vs[j], cfg)
+    lvl = HostLevel(go, lengths, pages, ks, vs)
+    hp.outer.append(lvl)
+    return lvl
 
 
 def _scatter(pool: np.ndarray, pages_row: np.ndarray, tokens: np.ndarray, cfg: Config) -> None:

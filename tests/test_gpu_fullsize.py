@@ -80,3 +80,17 @@ def test_full_size_properties_cfg2():
     torch.cuda.synchronize()
     assert torch.equal(o[0], o[17]) and torch.equal(lse[0], lse[63])
     dp.close()
+
+
+def test_full_size_cascade_cfg3_with_a_root_prompt():
+    """Configuration 3 with a 4096-token prompt shared by all 256 candidates in front of the group prefixes
+    (stacked query tile of 1024 rows per kv head at the root level)."""
+    cfg = wl.CONFIGS["cfg3"]
+    dp = make_device_problem(cfg, outer=[([0, cfg.B], [4096])])
+    assert dp.geom.n_prefix_parts >= 2
+    q = device_q(cfg, 0)
+    o, lse = dp.decode(q)
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    check_rows(dp, q, o, lse, sample_rows(cfg, 16, 3))
+    dp.close()

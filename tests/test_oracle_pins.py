@@ -295,3 +295,35 @@ def test_matches_torch_sdpa_float64():
         Qt = torch.from_numpy(q[b])[None, :, None, :]                            # [1][Hq][1][d]
         ref = torch.nn.functional.scaled_dot_product_attention(Qt, Kt, Vt, scale=scale)[0, :, 0].numpy()
         np.testing.assert_allclose(o[b], ref, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------------
+# cascade (prefix tree deeper than two levels): reduces to the two-level function by concatenation
+# ---------------------------------------------------------------------------------------------------
+def test_cascade_equals_two_level_with_concatenated_prefixes():
+    q, kp, vp, ks, vs, go = _tiny_problem(21, G=2, C=2)
+    rng = np.random.default_rng(22)
+    Hkv, d = kp[0].shape[1], kp[0].shape[2]
+    root_k, root_v = rng.normal(size=(7, Hkv, d)), rng.normal(size=(7, Hkv, d))      # shared by all 4 candidates
+    o, lse = orc.decode_attention_cascade(q, [([root_k], [root_v], [0, 4]), (kp, vp, go)], ks, vs, 0.4)
+    kp2 = [np.concatenate([root_k, k], axis=0) for k in kp]
+    vp2 = [np.concatenate([root_v, v], axis=0) for v in vp]
+    o2, lse2 = orc.decode_attention(q, kp2, vp2, ks, vs, go, 0.4)
+    np.testing.assert_allclose(o, o2, atol=1e-14)
+    np.testing.assert_allclose(lse, lse2, atol=1e-13)
+    # a single level is the two-level function itself, and the level order is irrelevant
+    o3, lse3 = orc.decode_attention_cascade(q, [(kp, vp, go)], ks, vs, 0.4)
+    o4, lse4 = orc.decode_attention(q, kp, vp, ks, vs, go, 0.4)
+    np.testing.assert_array_equal(o3, o4)
+    o5, _ = orc.decode_attention_cascade(q, [(kp, vp, go), ([root_k], [root_v], [0, 4])], ks, vs, 0.4)
+    np.testing.assert_allclose(o5, o, atol=1e-14)
+    # an outer level whose groups cut across differently: 3 + 1 candidates
+    mid_k = [rng.normal(size=(3, Hkv, d)), rng.normal(size=(5, Hkv, d))]
+    mid_v = [rng.normal(size=(3, Hkv, d)), rng.normal(size=(5, Hkv, d))]
+    o6, lse6 = orc.decode_attention_cascade(q, [(mid_k, mid_v, [0, 3, 4]), (kp, vp, go)], ks, vs, 0.4)
+    bo, blse = brute_force_decode(
+        q.tolist(), [np.concatenate([mid_k[0 if b < 3 else 1], kp[b // 2]], axis=0).tolist() for b in range(4)],
+        [np.concatenate([mid_v[0 if b < 3 else 1], vp[b // 2]], axis=0).tolist() for b in range(4)],
+        [x.tolist() for x in ks], [x.tolist() for x in vs], [0, 1, 2, 3, 4], 0.4)
+    np.testing.assert_allclose(o6, np.array(bo), atol=1e-12)
+    np.testing.assert_allclose(lse6, np.array(blse), atol=1e-12)
