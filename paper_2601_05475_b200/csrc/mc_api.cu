@@ -18,10 +18,9 @@ struct Layout {
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
-  PrefixTcPlan *tc_plan;      // non-null: the (innermost) prefix level runs on the tcgen05 kernel
+  PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
   Params outer_p[kMaxOuterLevels];
-  PrefixTcPlan *outer_plan[kMaxOuterLevels];
   cudaStream_t side_stream;   // the suffix pass of mc_decode_attn runs here, beside the prefix pass
   cudaEvent_t fork_ev, join_ev;
 };
@@ -112,9 +111,8 @@ mc_status_t check_q(const Layout *L, const void *q) {
   return MC_OK;
 }
 
-mc_status_t run_level(Layout *L, const Params &p, const PrefixTcPlan *plan, int mode, const void *q, float scale,
-                      float *o_part, float *lse_part, cudaStream_t st) {
-  if (mode == kPrefix && plan && scale != 0.f) return launch_prefix_tc(p, plan, q, scale, o_part, lse_part, st);
+mc_status_t run_level(Layout *L, const Params &p, int mode, const void *q, float scale, float *o_part,
+                      float *lse_part, cudaStream_t st) {
   if (L->use_mma) return launch_mma(p, mode, q, scale, o_part, lse_part, st);
   return launch_fma(p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
 }
@@ -123,19 +121,23 @@ mc_status_t run_level(Layout *L, const Params &p, const PrefixTcPlan *plan, int 
 mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t st) {
   if (mode == kPrefix) {
+    if (L->tc_plan && scale != 0.f) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
     for (int k = L->n_outer - 1; k >= 0; --k) {
-      mc_status_t s = run_level(L, L->outer_p[k], L->outer_plan[k], kPrefix, q, scale, o_part, lse_part, st);
+      mc_status_t s = run_level(L, L->outer_p[k], kPrefix, q, scale, o_part, lse_part, st);
       if (s != MC_OK) return s;
     }
   }
-  return run_level(L, L->p, L->tc_plan, mode, q, scale, o_part, lse_part, st);
+  return run_level(L, L->p, mode, q, scale, o_part, lse_part, st);
 }
 
 // Splits and persistent-CTA count of one prefix level (see the comment in mc_kv_layout_create_cascade).
-struct LevelSizing { int nsp, ctas, max_group; };
-LevelSizing size_level(const Params &p, double suffix_us, int env_ctas) {
+struct LevelWork { long long pairs; double tiles; int max_group; };
+constexpr double kTileUs = 1.6, kItemUs = 6.0;   // measured: per 128x128 tile; per item (prologue + epilogue)
+
+// (group, kv head, 128-row tile) pairs and 128-token tiles of one level, from the lengths as they are now.
+LevelWork level_work(const Params &p) {
   const int max_p = p.max_pp * kPage;
-  LevelSizing r;
+  LevelWork r;
   r.max_group = (p.B + p.G - 1) / p.G;
   const int rows_per_group = (int)(((long long)p.B * p.g + p.G - 1) / p.G);
   long long pairs = (long long)p.G * p.Hkv * ((rows_per_group + 127) / 128);
@@ -157,25 +159,28 @@ LevelSizing size_level(const Params &p, double suffix_us, int env_ctas) {
   (void)cudaGetLastError();
   delete[] go;
   delete[] pl;
-  if (pairs < 1) pairs = 1;
-  const double tile_us = 1.6, item_us = 6.0;                      // per 128x128 tile; per item
-  const double budget = suffix_us * 0.9, max_pair_tiles = (max_p + 127) / 128;
+  r.pairs = pairs < 1 ? 1 : pairs;
+  r.tiles = tiles;
+  return r;
+}
+
+// Splits of one level: as few as let its longest item (plus its fixed cost) end within `budget_us`.
+int choose_splits(const Params &p, const LevelWork &w, double budget_us) {
+  const double max_pair_tiles = (p.max_pp * kPage + 127) / 128;
   int nsp;
   for (nsp = 1; nsp < 8; ++nsp)
-    if ((max_pair_tiles + nsp - 1) / nsp * tile_us + item_us <= budget) break;
-  if (budget < item_us + tile_us) nsp = (int)((160 + pairs - 1) / pairs);   // nothing to hide under: many items
-  if (nsp > 8) nsp = 8;
-  if (nsp < 1) nsp = 1;
-  r.nsp = nsp;
-  r.ctas = env_ctas;
-  if (r.ctas == 0) {
-    const double items = (double)pairs * nsp, avg_item_us = tiles / items * tile_us + item_us;
-    int rounds = (int)(0.7 * budget / avg_item_us);
-    if (rounds < 1) rounds = 1;
-    r.ctas = (int)((items + rounds - 1) / rounds);
-    if (r.ctas < 8) r.ctas = 8;
-  }
-  return r;
+    if ((max_pair_tiles + nsp - 1) / nsp * kTileUs + kItemUs <= budget_us) break;
+  if (budget_us < kItemUs + kTileUs) nsp = (int)((160 + w.pairs - 1) / w.pairs);   // nothing to hide under: many items
+  return nsp > 8 ? 8 : nsp < 1 ? 1 : nsp;
+}
+
+// Persistent CTAs for `items` items of `tiles` tiles in all: the fewest whose rounds still end in the budget.
+int choose_ctas(double items, double tiles, double budget_us) {
+  const double avg_item_us = tiles / items * kTileUs + kItemUs;
+  int rounds = (int)(0.7 * budget_us / avg_item_us);
+  if (rounds < 1) rounds = 1;
+  const int ctas = (int)((items + rounds - 1) / rounds);
+  return ctas < 8 ? 8 : ctas;
 }
 
 }  // namespace
@@ -269,13 +274,20 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   if (ts > 4096) ts = 4096;
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
-  mc::LevelSizing sizing[1 + mc::kMaxOuterLevels];
+  // The levels of the cascade share one persistent grid, so every item has the whole budget.
+  mc::LevelWork work[1 + mc::kMaxOuterLevels];
+  int nsp[1 + mc::kMaxOuterLevels];
+  double all_items = 0.0, all_tiles = 0.0;
+  const double budget_us = suffix_us * 0.9;
   int part_base = 0;
   for (int k = 0; k <= n_outer; ++k) {   // k = 0: the base level; part slots in this order, then the suffix chunks
     mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
-    sizing[k] = mc::size_level(pk, suffix_us, mc::env_int("MC_PREFIX_CTAS", 0));
+    work[k] = mc::level_work(pk);
+    nsp[k] = mc::choose_splits(pk, work[k], budget_us);
+    all_items += (double)work[k].pairs * nsp[k];
+    all_tiles += work[k].tiles;
     const int max_p = pk.max_pp * mc::kPage;
-    int tp = ((max_p + sizing[k].nsp - 1) / sizing[k].nsp + 127) / 128 * 128;
+    int tp = ((max_p + nsp[k] - 1) / nsp[k] + 127) / 128 * 128;
     if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0)
       tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
     if (tp < mc::kPage) tp = mc::kPage;
@@ -319,13 +331,18 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess &&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
-      for (int k = 0; k <= n_outer; ++k) {
-        const mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
-        mc::PrefixTcPlan *plan = nullptr;
-        if (mc::prefix_tc_supported(pk, d->dtype) && sizing[k].max_group <= p.B)
-          plan = mc::prefix_tc_plan(pk, sizing[k].max_group, sms, sizing[k].ctas > sms ? sms : sizing[k].ctas);
-        if (k == 0) L->tc_plan = plan; else L->outer_plan[k - 1] = plan;
+      // outermost level first: its items are the ones with the most rows
+      mc::Params levels[1 + mc::kMaxOuterLevels];
+      int max_group[1 + mc::kMaxOuterLevels];
+      bool all = true;
+      for (int k = n_outer, i = 0; k >= 0; --k, ++i) {
+        levels[i] = k == 0 ? p : L->outer_p[k - 1];
+        max_group[i] = work[k].max_group;
+        all = all && mc::prefix_tc_supported(levels[i], d->dtype) && max_group[i] <= p.B;
       }
+      int ctas = mc::env_int("MC_PREFIX_CTAS", 0);
+      if (ctas <= 0) ctas = mc::choose_ctas(all_items, all_tiles, budget_us);
+      if (all) L->tc_plan = mc::prefix_tc_plan(levels, max_group, n_outer + 1, sms, ctas > sms ? sms : ctas);
     }
     (void)cudaGetLastError();
   }
@@ -346,7 +363,6 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   if (L->fork_ev) cudaEventDestroy(L->fork_ev);
   if (L->join_ev) cudaEventDestroy(L->join_ev);
   mc::prefix_tc_plan_free(L->tc_plan);
-  for (int k = 0; k < L->n_outer; ++k) mc::prefix_tc_plan_free(L->outer_plan[k]);
   cudaFree(L->dev_status);
   cudaFreeHost(L->host_status);
   delete L;

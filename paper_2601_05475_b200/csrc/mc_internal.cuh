@@ -91,10 +91,11 @@ mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const 
                          float *lse, cudaStream_t stream);
 bool mma_supported(const Params &p, int dtype);
 
-// tensor-core (tcgen05) prefix pass
+// tensor-core (tcgen05) prefix pass: one persistent grid over the items of all cascade levels
+constexpr int kMaxTcLevels = 4;
 struct PrefixTcPlan;
 bool prefix_tc_supported(const Params &p, int dtype);
-PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int max_ctas);
+PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int max_ctas);
 void prefix_tc_plan_free(PrefixTcPlan *plan);
 int prefix_tc_grid(const PrefixTcPlan *plan);
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,

@@ -196,32 +196,48 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
+// One level of the prefix cascade as the kernel sees it; the levels' items are numbered one level after another.
+struct TcLevel {
+  const int32_t *group_offsets, *prefix_pages, *prefix_len;
+  int32_t max_pp, n_splits, part_base, part_tokens, n_mt, item_end;
+};
+struct TcLevels {
+  int32_t n;
+  TcLevel lv[kMaxTcLevels];
+};
+
 struct Item {
-  int j, h, sp, mt;      // group, kv head, prefix split, row tile
+  int j, h, mt;          // group, kv head, row tile
+  int part;              // part slot the result goes to
   int b0, n_cand;        // first candidate of the group, candidates in the group
   int lo, hi;            // token range of this split
   const int32_t *pages;
 };
 
-__device__ __forceinline__ Item decode_item(const Params &p, int item, int n_mt) {
+__device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs, int item) {
+  int l = 0;
+  while (l + 1 < lvs.n && item >= lvs.lv[l].item_end) ++l;
+  const TcLevel &L = lvs.lv[l];
+  if (l > 0) item -= lvs.lv[l - 1].item_end;
   Item it;
-  it.mt = item % n_mt;
-  int r = item / n_mt;
-  it.sp = r % p.n_prefix_parts;
-  r /= p.n_prefix_parts;
+  it.mt = item % L.n_mt;
+  int r = item / L.n_mt;
+  const int sp = r % L.n_splits;
+  r /= L.n_splits;
   it.h = r % p.Hkv;
   it.j = r / p.Hkv;
-  it.b0 = __ldg(p.group_offsets + it.j);
-  it.n_cand = __ldg(p.group_offsets + it.j + 1) - it.b0;
-  int len = __ldg(p.prefix_len + it.j);
-  const int cap = p.max_pp * kPage;
+  it.b0 = __ldg(L.group_offsets + it.j);
+  it.n_cand = __ldg(L.group_offsets + it.j + 1) - it.b0;
+  int len = __ldg(L.prefix_len + it.j);
+  const int cap = L.max_pp * kPage;
   if (len < 0 || len > cap) {
     latch(p, kDevBadPage);
     len = len < 0 ? 0 : cap;
   }
-  it.lo = it.sp * p.prefix_part_tokens;
-  it.hi = min(len, it.lo + p.prefix_part_tokens);
-  it.pages = p.prefix_pages + (size_t)it.j * p.max_pp;
+  it.part = L.part_base + sp;
+  it.lo = sp * L.part_tokens;
+  it.hi = min(len, it.lo + L.part_tokens);
+  it.pages = L.prefix_pages + (size_t)it.j * L.max_pp;
   return it;
 }
 
@@ -231,9 +247,9 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
 }
 
 __global__ void __maxnreg__(104)
-prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
-                 const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
-                 float *__restrict__ lse_part, int n_items, int n_mt) {
+prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
+                 const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
+                 float *__restrict__ o_part, float *__restrict__ lse_part, int n_items) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base
@@ -290,7 +306,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
 
     auto next_item = [&](int from, Item &out) -> int {
       for (int i = from; i < n_items; i += gridDim.x) {
-        out = decode_item(p, i, n_mt);
+        out = decode_item(p, lvs, i);
         if (item_has_work(out, cand_per_tile)) return i;
       }
       return n_items;
@@ -393,7 +409,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
-        const Item it = decode_item(p, item, n_mt);
+        const Item it = decode_item(p, lvs, item);
         if (!item_has_work(it, cand_per_tile)) continue;
         const int qb = it_n & 1;
         if (!mbar_wait(sm, p, &sm.q_ready[qb], (it_n >> 1) & 1)) break;
@@ -463,12 +479,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __gr
       return w;
     };
     for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
-      const Item it = decode_item(p, item, n_mt);
+      const Item it = decode_item(p, lvs, item);
       if (it.mt * cand_per_tile >= it.n_cand) continue;
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
-      const size_t slot = qrow * p.n_parts + p.prefix_part_base + it.sp;
+      const size_t slot = qrow * p.n_parts + it.part;
       if (it.lo >= it.hi) {
         if (row_ok && half == 0) lse_part[slot] = -INFINITY;
         continue;
@@ -677,7 +693,8 @@ static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
 
 struct PrefixTcPlan {
   CUtensorMap k_map, v_map;
-  int n_mt, n_items, grid;
+  TcLevels levels;
+  int n_items, grid;
 };
 
 bool prefix_tc_supported(const Params &p, int dtype) {
@@ -685,17 +702,39 @@ bool prefix_tc_supported(const Params &p, int dtype) {
          p.prefix_part_tokens % kTileN == 0;
 }
 
-// Host-side preparation at layout-create time: tensor maps over the two pools and the item count.
-// `max_group` is the largest number of candidates in one group.  Returns nullptr when unavailable.
-PrefixTcPlan *prefix_tc_plan(const Params &p, int max_group, int sm_count, int max_ctas) {
+// Host-side preparation at layout-create time: tensor maps over the two pools and the items of every level
+// (`levels[k]` with at most `max_group[k]` candidates in one group), dealt to one persistent grid in the
+// order given.  Returns nullptr when unavailable.
+PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int max_ctas) {
+  if (n_levels < 1 || n_levels > kMaxTcLevels) return nullptr;
   PrefixTcPlan *plan = new PrefixTcPlan();
+  const Params &p = levels[0];
   if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
       !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true)) {
     delete plan;
     return nullptr;
   }
-  plan->n_mt = (max_group * p.g + kTileM - 1) / kTileM;
-  plan->n_items = p.G * p.Hkv * p.n_prefix_parts * plan->n_mt;
+  long long items = 0;
+  plan->levels.n = n_levels;
+  for (int k = 0; k < n_levels; ++k) {
+    const Params &pk = levels[k];
+    TcLevel &lv = plan->levels.lv[k];
+    lv.group_offsets = pk.group_offsets;
+    lv.prefix_pages = pk.prefix_pages;
+    lv.prefix_len = pk.prefix_len;
+    lv.max_pp = pk.max_pp;
+    lv.n_splits = pk.n_prefix_parts;
+    lv.part_base = pk.prefix_part_base;
+    lv.part_tokens = pk.prefix_part_tokens;
+    lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
+    items += (long long)pk.G * pk.Hkv * pk.n_prefix_parts * lv.n_mt;
+    if (items > 0x7fffffffLL) {
+      delete plan;
+      return nullptr;
+    }
+    lv.item_end = (int32_t)items;
+  }
+  plan->n_items = (int)items;
   int grid = plan->n_items < sm_count ? plan->n_items : sm_count;
   if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
   if (grid < 1) grid = 1;
@@ -717,8 +756,8 @@ int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {
   prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
-      p, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
-      plan->n_items, plan->n_mt);
+      p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part,
+      lse_part, plan->n_items);
   count_launch();
   return check_launch();
 }
