@@ -1,9 +1,11 @@
 // C-ABI entry points: argument checking, layout object, append, validation, status word, and the
 // drivers that enqueue the passes.
+#include <algorithm>
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "mc_internal.cuh"
 
@@ -15,6 +17,7 @@ struct Layout {
   mc_kv_layout_desc_t desc;
   Params p;
   int32_t *dev_status;   // device int
+  int32_t *suffix_order; // device array: launch order of the suffix pass's CTAs, or null
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
@@ -260,15 +263,18 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   // splits as still let one item fit the time budget.  Constants are measured for this kernel pair.
   const int max_s = d->max_suffix_pages * mc::kPage;
   double suffix_us = 0.0;
+  int32_t *sl = nullptr;
   {
-    int32_t *sl = new (std::nothrow) int32_t[p.B];
+    sl = new (std::nothrow) int32_t[p.B];
     if (sl && cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
       double suffix_tokens = 0.0;
       for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
       suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : 2) / 6.8e6;   // stream at ~6.8 TB/s
+    } else {
+      delete[] sl;
+      sl = nullptr;
     }
     (void)cudaGetLastError();
-    delete[] sl;
   }
   int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
   if (ts > 4096) ts = 4096;
@@ -304,6 +310,38 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     pk.n_parts = n_parts;
   }
   L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
+  // Suffix CTAs are launched longest first (by the lengths as they are now; appends change them slowly), so
+  // that the launch ends on short items instead of a few long ones.  Without it the order is as numbered.
+  L->suffix_order = nullptr;
+  if (L->use_mma && sl && mc::env_int("MC_SUFFIX_ORDER", 1)) {
+    const int per = mc::mma_items_per_cta(), n_chunks = n_parts - part_base;
+    const long long n_items = (long long)p.B * p.Hkv * n_chunks, n_ctas = (n_items + per - 1) / per;
+    if (n_ctas > 1 && n_ctas < (1ll << 24)) {
+      std::vector<int32_t> order((size_t)n_ctas), key((size_t)n_ctas);
+      for (long long c = 0; c < n_ctas; ++c) {
+        int longest = 0;
+        for (long long it = c * per; it < (c + 1) * per && it < n_items; ++it) {   // item = (b, chunk, kv head)
+          const int chunk = (int)((it / p.Hkv) % n_chunks), b = (int)(it / ((long long)p.Hkv * n_chunks));
+          int tokens = sl[b] - chunk * ts;
+          tokens = tokens < 0 ? 0 : tokens > ts ? ts : tokens;
+          if (tokens > longest) longest = tokens;
+        }
+        key[(size_t)c] = longest;
+        order[(size_t)c] = (int32_t)c;
+      }
+      std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return key[a] > key[b]; });
+      if (cudaMalloc(&L->suffix_order, sizeof(int32_t) * (size_t)n_ctas) != cudaSuccess ||
+          cudaMemcpy(L->suffix_order, order.data(), sizeof(int32_t) * (size_t)n_ctas, cudaMemcpyHostToDevice) !=
+              cudaSuccess) {
+        cudaFree(L->suffix_order);
+        L->suffix_order = nullptr;
+        (void)cudaGetLastError();
+      }
+    }
+  }
+  delete[] sl;
+  p.suffix_order = L->suffix_order;
+  for (int k = 0; k < n_outer; ++k) L->outer_p[k].suffix_order = L->suffix_order;
 
   const size_t rows = (size_t)p.B * p.Hq, e = d->dtype == MC_F32 ? 4 : 2;
   L->o_part_bytes = mc::align_up(rows * p.n_parts * p.d * sizeof(float), 256);
@@ -314,10 +352,15 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   for (int i = 0; i < 5; ++i) { L->staging_off[i] = off; off += sizes[i]; }
   L->ws_bytes = off;
 
-  if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) { delete L; return MC_ERR_OUT_OF_MEMORY; }
+  if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) {
+    cudaFree(L->suffix_order);
+    delete L;
+    return MC_ERR_OUT_OF_MEMORY;
+  }
   if (cudaMemset(L->dev_status, 0, 256) != cudaSuccess ||
       cudaMallocHost(&L->host_status, sizeof(int32_t)) != cudaSuccess) {
     cudaFree(L->dev_status);
+    cudaFree(L->suffix_order);
     delete L;
     return MC_ERR_CUDA;
   }
@@ -364,6 +407,7 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   if (L->join_ev) cudaEventDestroy(L->join_ev);
   mc::prefix_tc_plan_free(L->tc_plan);
   cudaFree(L->dev_status);
+  cudaFree(L->suffix_order);
   cudaFreeHost(L->host_status);
   delete L;
   return MC_OK;

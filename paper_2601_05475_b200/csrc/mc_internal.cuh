@@ -27,6 +27,7 @@ struct Params {
   int32_t n_prefix_parts, prefix_part_base;          // this prefix level's splits and its first part slot
   int32_t suffix_part_base;                          // first part slot of the suffix chunks
   int32_t prefix_part_tokens, suffix_part_tokens;
+  const int32_t *suffix_order;                       // launch order of the suffix pass's CTAs (null: as numbered)
   int32_t *status;
 };
 
@@ -90,6 +91,7 @@ mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, fl
 mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
                          float *lse, cudaStream_t stream);
 bool mma_supported(const Params &p, int dtype);
+int mma_items_per_cta();
 
 // tensor-core (tcgen05) prefix pass: one persistent grid over the items of all cascade levels
 constexpr int kMaxTcLevels = 4;

@@ -150,7 +150,9 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
   const int lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
   const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
-  const long long item = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+  // the order CTAs are launched in may be given (longest first); every CTA index appears once
+  const long long cta = MODE == kSuffix && p.suffix_order ? __ldg(p.suffix_order + blockIdx.x) : blockIdx.x;
+  const long long item = cta * kWarps + (threadIdx.x >> 5);
   if (item >= n_items) return;
   int b, h, part;
   if (MODE == kSuffix) {  // kv heads of one page are adjacent in the pool: neighbours stream neighbours
@@ -295,6 +297,8 @@ static int suffix_prefetch_pages() {
   }
   return v;
 }
+
+int mma_items_per_cta() { return kWarps; }
 
 bool mma_supported(const Params &p, int dtype) { return dtype == MC_BF16 && p.d == 128 && p.g >= 1 && p.g <= 8; }
 
