@@ -118,7 +118,7 @@ typedef struct {
 
 /* mc_kv_layout_create for a cascade deeper than two levels: every candidate attends to the tokens of each outer
  * level's group it belongs to, to its base-level prefix and to its suffix (the order of concatenation does not
- * change the result).  The prefix pass runs once per level, each level writes part slots of its own, the merge
+ * change the result).  The prefix pass covers every level, each level writes part slots of its own, the merge
  * combines them all.  n_outer <= 3.  With n_outer = 0 this is mc_kv_layout_create. */
 mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *desc, const mc_prefix_level_t *outer,
                                         int32_t n_outer, mc_kv_layout_t **out);
@@ -164,8 +164,10 @@ mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale,
                            void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
 
 /* One whole decode step with device-resident tensors: appends k_new/v_new (as mc_kv_append) and runs
- * mc_decode_attn, scheduled so that the append, which only the suffix pass depends on, runs beside the start of
- * the prefix pass.  k_new = v_new = NULL skips the append (then identical to mc_decode_attn). */
+ * mc_decode_attn.  k_new = v_new = NULL skips the append (then identical to mc_decode_attn).  The suffix pass
+ * is scheduled beside the prefix pass (it starts once the prefix pass's CTAs are running); everything is
+ * enqueued on `stream` or on streams of the handle that fork from and join it, so the call can be captured
+ * into a CUDA graph and replayed: the lengths it depends on are read on the device. */
 mc_status_t mc_decode_step(mc_kv_layout_t *layout, const void *k_new, const void *v_new, const void *q,
                            float scale, void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
 

@@ -26,6 +26,7 @@ struct Layout {
   Params outer_p[kMaxOuterLevels];
   cudaStream_t side_stream;   // the suffix pass of mc_decode_attn runs here, beside the prefix pass
   cudaEvent_t fork_ev, join_ev;
+  bool pdl;                   // suffix pass launched as the prefix pass's programmatic dependent (MC_PDL=0: off)
 };
 
 static std::atomic<uint64_t> g_launches{0};
@@ -262,7 +263,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   // item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be long: as few
   // splits as still let one item fit the time budget.  Constants are measured for this kernel pair.
   const int max_s = d->max_suffix_pages * mc::kPage;
-  double suffix_us = 0.0;
+  double suffix_us = 0.0, suffix_tokens_now = -1.0;
   int32_t *sl = nullptr;
   {
     sl = new (std::nothrow) int32_t[p.B];
@@ -270,6 +271,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
       double suffix_tokens = 0.0;
       for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
       suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : 2) / 6.8e6;   // stream at ~6.8 TB/s
+      suffix_tokens_now = suffix_tokens;
     } else {
       delete[] sl;
       sl = nullptr;
@@ -278,6 +280,18 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   }
   int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
   if (ts > 4096) ts = 4096;
+  if (suffix_tokens_now >= 0.0) {
+    // A small problem is bound by one warp's page-after-page latency, not by HBM: shorter chunks until the
+    // (kv head, chunk) items fill the warps the device holds at once (8 per SM), down to 4 pages a chunk.
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      sms = 148;
+    (void)cudaGetLastError();
+    const double per_warp = suffix_tokens_now * p.Hkv / (8.0 * sms);
+    int tpar = mc::pow2_floor(per_warp < 64.0 ? 64 : per_warp > 4096.0 ? 4096 : (int)per_warp);
+    if (tpar < ts) ts = tpar;
+  }
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
   // The levels of the cascade share one persistent grid, so every item has the whole budget.
@@ -389,6 +403,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     }
     (void)cudaGetLastError();
   }
+  L->pdl = mc::env_int("MC_PDL", 1) != 0;
   if (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&L->fork_ev, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&L->join_ev, cudaEventDisableTiming) != cudaSuccess) {
@@ -508,11 +523,20 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   float *o_part = reinterpret_cast<float *>(ws);
   float *lse_part = reinterpret_cast<float *>(static_cast<char *>(ws) + L->o_part_bytes);
-  // The two passes write disjoint part slots and run side by side: the prefix pass (tensor-bound, a few
-  // persistent CTAs per SM's shared memory) is launched first, on the caller's stream, so that its CTAs are
-  // resident before the suffix pass (HBM-bound, thousands of short CTAs) floods the SMs from the handle's
-  // side stream.  The append touches only suffix pages and lengths, so it goes to the side stream too, in
-  // front of the suffix pass.  The merge joins the streams.
+  // The two passes write disjoint part slots and run side by side.  The prefix pass (tensor-bound, a few
+  // persistent CTAs, each needing an SM's whole shared memory) must get its CTAs placed before the suffix pass
+  // (HBM-bound, thousands of short CTAs) fills every SM.
+  if (L->tc_plan && L->use_mma && scale != 0.f && L->pdl) {
+    // One stream: the suffix pass is launched behind the tensor-core prefix pass as its programmatic
+    // dependent, so it starts once every prefix CTA is running, not when they end.  The order holds when
+    // the step is replayed from a captured graph.  The merge, launched the ordinary way, waits for both.
+    if (k_new && (s = mc_kv_append(layout, k_new, v_new, st)) != MC_OK) return s;
+    if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+    if ((s = mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true)) != MC_OK) return s;
+    return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
+  }
+  // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix
+  // pages and lengths) and the suffix pass on the handle's side stream; the merge joins them.
   if (cudaEventRecord(L->fork_ev, st) != cudaSuccess ||
       cudaStreamWaitEvent(L->side_stream, L->fork_ev, 0) != cudaSuccess)
     return MC_ERR_CUDA;

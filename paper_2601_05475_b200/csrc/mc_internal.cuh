@@ -86,8 +86,10 @@ mc_status_t check_launch();
 // launchers (each enqueues on `stream` and returns the launch status)
 mc_status_t launch_fma(const Params &p, int dtype, int mode, const void *q, float scale, float *o_part,
                        float *lse_part, cudaStream_t stream);
+// `beside_previous`: the launch does not wait for the kernel in front of it on the stream to end, only for
+// that kernel's CTAs to announce that dependents may start (programmatic dependent launch).
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
-                       cudaStream_t stream);
+                       cudaStream_t stream, bool beside_previous = false);
 mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
                          float *lse, cudaStream_t stream);
 bool mma_supported(const Params &p, int dtype);

@@ -303,17 +303,31 @@ int mma_items_per_cta() { return kWarps; }
 bool mma_supported(const Params &p, int dtype) { return dtype == MC_BF16 && p.d == 128 && p.g >= 1 && p.g <= 8; }
 
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
-                       cudaStream_t stream) {
+                       cudaStream_t stream, bool beside_previous) {
   const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
   if (n_items == 0) return MC_OK;
   const unsigned grid = (unsigned)((n_items + kWarps - 1) / kWarps);
   const float sl2 = scale * kLog2e;
   const __nv_bfloat16 *qb = reinterpret_cast<const __nv_bfloat16 *>(q);
-  if (mode == kPrefix)
+  if (mode == kPrefix) {
     attn_mma_kernel<kPrefix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, 0);
-  else
-    attn_mma_kernel<kSuffix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, suffix_prefetch_pages());
+  } else {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kWarps * 32);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = beside_previous ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, attn_mma_kernel<kSuffix>, p, qb, sl2, o_part, lse_part, suffix_prefetch_pages()) !=
+        cudaSuccess) {
+      count_launch();
+      return MC_ERR_CUDA;
+    }
+  }
   count_launch();
   return check_launch();
 }

@@ -260,6 +260,9 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   const int g = p.g, cand_per_tile = kTileM / g;
 
   if (threadIdx.x == 0) {
+    // This CTA holds its SM now: a kernel launched behind this one as its programmatic dependent (the suffix
+    // pass, which needs nothing this kernel writes) may start as soon as every CTA of this grid has said so.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     for (int s = 0; s < kKSlots; ++s) {
       mbar_init(&sm.full_k[s], 1);
       mbar_init(&sm.empty_k[s], 1);

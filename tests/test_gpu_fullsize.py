@@ -94,3 +94,32 @@ def test_full_size_cascade_cfg3_with_a_root_prompt():
     assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
     check_rows(dp, q, o, lse, sample_rows(cfg, 16, 3))
     dp.close()
+
+
+def test_merge_waits_for_a_prefix_pass_that_outlasts_the_suffix_pass(monkeypatch):
+    """The suffix pass starts while the prefix pass is still running; the merge must not.  A long prefix on few
+    CTAs against suffixes of at most one page: the fused call equals the three passes run one after another."""
+    monkeypatch.setenv("MC_PREFIX_CTAS", "8")
+    cfg = wl.Config("long_prefix", "bf16", G=4, C=16, Hq=32, Hkv=8, d=128, prefix=("fixed", 32768),
+                    suffix=("uniform", 0, 16))
+    dp = make_device_problem(cfg, headroom_tokens=4)
+    q = device_q(cfg, 0)
+    g = dp.geom
+    assert g.prefix_ctas == 8
+    lse_off = (g.rows * g.n_parts * g.head_dim * 4 + 255) // 256 * 256
+    o_part, lse_part = dp.ws_ptr, dp.ws_ptr + lse_off
+    o_ref, lse_ref = torch.empty_like(dp.o), torch.empty_like(dp.lse)
+    mc.mc_prefix_attn(dp.layout, q, cfg.scale, o_part, lse_part)
+    mc.mc_suffix_attn(dp.layout, q, cfg.scale, o_part, lse_part)
+    mc.mc_merge_lse(dp.layout, o_part, lse_part, o_ref, lse_ref)
+    torch.cuda.synchronize()
+    check_rows(dp, q, o_ref, lse_ref, sample_rows(cfg, 4, 5))
+    for _ in range(5):
+        dp.ws.zero_()   # a merge that ran early would find empty prefix parts
+        dp.o.zero_()
+        dp.lse.zero_()
+        o, lse = dp.decode(q)
+        torch.cuda.synchronize()
+        assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    dp.close()
