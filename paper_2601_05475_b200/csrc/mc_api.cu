@@ -21,6 +21,7 @@ struct Layout {
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
+  SuffixTmaPlan *sfx_plan;    // non-null: the suffix pass runs on the TMA-fed kernel
   PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
   Params outer_p[kMaxOuterLevels];
@@ -117,6 +118,7 @@ mc_status_t check_q(const Layout *L, const void *q) {
 
 mc_status_t run_level(Layout *L, const Params &p, int mode, const void *q, float scale, float *o_part,
                       float *lse_part, cudaStream_t st) {
+  if (mode == kSuffix && L->sfx_plan) return launch_suffix_tma(p, L->sfx_plan, q, scale, o_part, lse_part, st, false);
   if (L->use_mma) return launch_mma(p, mode, q, scale, o_part, lse_part, st);
   return launch_fma(p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
 }
@@ -324,11 +326,12 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     pk.n_parts = n_parts;
   }
   L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
+  L->sfx_plan = L->use_mma && mc::env_int("MC_SUFFIX_TMA", 1) ? mc::suffix_tma_plan(p, d->dtype) : nullptr;
   // Suffix CTAs are launched longest first (by the lengths as they are now; appends change them slowly), so
   // that the launch ends on short items instead of a few long ones.  Without it the order is as numbered.
   L->suffix_order = nullptr;
   if (L->use_mma && sl && mc::env_int("MC_SUFFIX_ORDER", 1)) {
-    const int per = mc::mma_items_per_cta(), n_chunks = n_parts - part_base;
+    const int per = L->sfx_plan ? mc::suffix_tma_items_per_cta() : mc::mma_items_per_cta(), n_chunks = n_parts - part_base;
     const long long n_items = (long long)p.B * p.Hkv * n_chunks, n_ctas = (n_items + per - 1) / per;
     if (n_ctas > 1 && n_ctas < (1ll << 24)) {
       std::vector<int32_t> order((size_t)n_ctas), key((size_t)n_ctas);
@@ -368,6 +371,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
 
   if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) {
     cudaFree(L->suffix_order);
+    mc::suffix_tma_plan_free(L->sfx_plan);
     delete L;
     return MC_ERR_OUT_OF_MEMORY;
   }
@@ -375,6 +379,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
       cudaMallocHost(&L->host_status, sizeof(int32_t)) != cudaSuccess) {
     cudaFree(L->dev_status);
     cudaFree(L->suffix_order);
+    mc::suffix_tma_plan_free(L->sfx_plan);
     delete L;
     return MC_ERR_CUDA;
   }
@@ -421,6 +426,7 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   if (L->fork_ev) cudaEventDestroy(L->fork_ev);
   if (L->join_ev) cudaEventDestroy(L->join_ev);
   mc::prefix_tc_plan_free(L->tc_plan);
+  mc::suffix_tma_plan_free(L->sfx_plan);
   cudaFree(L->dev_status);
   cudaFree(L->suffix_order);
   cudaFreeHost(L->host_status);
@@ -532,7 +538,9 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
     // the step is replayed from a captured graph.  The merge, launched the ordinary way, waits for both.
     if (k_new && (s = mc_kv_append(layout, k_new, v_new, st)) != MC_OK) return s;
     if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st)) != MC_OK) return s;
-    if ((s = mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true)) != MC_OK) return s;
+    s = L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
+                    : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
+    if (s != MC_OK) return s;
     return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
   }
   // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix

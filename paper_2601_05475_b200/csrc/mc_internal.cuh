@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of the library (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -104,5 +105,19 @@ void prefix_tc_plan_free(PrefixTcPlan *plan);
 int prefix_tc_grid(const PrefixTcPlan *plan);
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream);
+
+
+// Tensor map over a paged pool [page][kv head][16 tokens][128] (bf16) for TMA copies with the 128-byte swizzle:
+// `whole_page`: one 4 KB box per (page, kv head) slab that lands as [d half][16 tokens][64];
+// otherwise one 2 KB box per (page, kv head, d half).
+bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv, bool whole_page);
+
+// suffix pass through TMA-fed shared-memory rings (bf16, d = 128, g <= 8)
+struct SuffixTmaPlan;
+SuffixTmaPlan *suffix_tma_plan(const Params &p, int dtype);
+void suffix_tma_plan_free(SuffixTmaPlan *plan);
+int suffix_tma_items_per_cta();
+mc_status_t launch_suffix_tma(const Params &p, const SuffixTmaPlan *plan, const void *q, float scale, float *o_part,
+                              float *lse_part, cudaStream_t stream, bool beside_previous);
 
 }  // namespace mc

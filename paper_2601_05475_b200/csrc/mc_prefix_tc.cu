@@ -15,8 +15,6 @@
 // 64 of the tile's 128 columns) do the softmax, the rescale and the epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
-#include <cuda.h>
-
 #include "mc_internal.cuh"
 
 namespace mc {
@@ -657,6 +655,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   }
 }
 
+static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
+
+}  // namespace
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -689,10 +691,6 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
-
-}  // namespace
 
 struct PrefixTcPlan {
   CUtensorMap k_map, v_map;

@@ -252,6 +252,31 @@ def test_forced_alu_path_matches_oracle(monkeypatch):
     dp.close()
 
 
+@pytest.mark.parametrize("name", ["cfg2s", "cfg3sp", "cfg4s"])
+def test_warp_level_suffix_kernel_matches_oracle(monkeypatch, name):
+    """The suffix pass on the register-fed warp-level kernel (the default is the TMA-fed one)."""
+    monkeypatch.setenv("MC_SUFFIX_TMA", "0")
+    cfg = SMALL[name]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+@pytest.mark.parametrize("ts", [1024, 4096])
+def test_long_suffix_chunks(monkeypatch, ts):
+    """Chunks of more than 64 pages: the suffix kernel reloads its page-id registers on the way."""
+    monkeypatch.setenv("MC_SUFFIX_PART_TOKENS", str(ts))
+    cfg = SMALL["cfg4s"]
+    hp = wl.make_host_problem(cfg)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    assert dp.geom.suffix_part_tokens == ts
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
 @pytest.mark.parametrize("tp,ts", [(16, 16), (64, 48), (4096, 4096)])
 def test_result_does_not_depend_on_part_geometry(monkeypatch, tp, ts):
     monkeypatch.setenv("MC_PREFIX_PART_TOKENS", str(tp))
