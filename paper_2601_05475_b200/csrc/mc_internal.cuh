@@ -111,6 +111,7 @@ mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const vo
 // `whole_page`: one 4 KB box per (page, kv head) slab that lands as [d half][16 tokens][64];
 // otherwise one 2 KB box per (page, kv head, d half).
 bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv, bool whole_page);
+bool encode_kv_pair_map(CUtensorMap *map, const void *lower_pool, unsigned long long distance, int num_pages, int Hkv);
 
 // suffix pass through TMA-fed shared-memory rings (bf16, d = 128, g <= 8)
 struct SuffixTmaPlan;

@@ -692,6 +692,25 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Both pools in one map: the (page, kv head) slabs of the pool at the lower address and, `distance` bytes above
+// each, the same slab of the other pool.  One 8 KB box = [pool][d half][16 tokens][64] of one (page, kv head).
+bool encode_kv_pair_map(CUtensorMap *map, const void *lower_pool, unsigned long long distance, int num_pages, int Hkv) {
+  if (distance == 0 || (distance & 15ull) != 0 || distance >= (1ull << 40)) return false;
+  void *sym = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !sym)
+    return false;
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(sym);
+  const cuuint64_t dims[5] = {64, (cuuint64_t)kPage, 2, (cuuint64_t)num_pages * (cuuint64_t)Hkv, 2};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, 128, (cuuint64_t)kPage * D * 2, (cuuint64_t)distance};
+  const cuuint32_t box[5] = {64, (cuuint32_t)kPage, 2, 1, 2};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(lower_pool), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct PrefixTcPlan {
   CUtensorMap k_map, v_map;
   TcLevels levels;

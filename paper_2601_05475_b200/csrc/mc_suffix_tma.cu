@@ -6,8 +6,8 @@
 // product) before it can ask for the page after next: measured, that chain and not HBM sets its pace, so the
 // pass needs every warp slot of every SM to reach the memory roofline and loses speed as soon as another
 // kernel holds some of them.  Here the loads are asynchronous copies that cost no registers:
-//   * each warp owns a ring of kStages page stages (K slab 4 KB + V slab 4 KB each); one lane issues the two
-//     TMA copies of a page (128-byte swizzle, so that the fragment loads below are free of bank conflicts)
+//   * each warp owns a ring of kStages page stages (K slab 4 KB + V slab 4 KB each); one lane issues the TMA
+//     copy of a page (128-byte swizzle, so that the fragment loads below are free of bank conflicts)
 //     kStages pages ahead of the page being computed, and an mbarrier per stage counts the bytes in;
 //   * fragments come from shared memory with ldmatrix (K as the A operand of S = K_page Q^T, V transposed
 //     as the A operand of O^T += V_page^T P^T), so nothing is permuted in registers;
@@ -25,7 +25,7 @@ namespace {
 
 constexpr int D = 128;
 constexpr int kW = 2;                      // warps (items) per CTA
-constexpr int kStages = 6;                 // page stages per warp: two being computed, four in flight
+constexpr int kStages = 4;                 // page stages per warp: two being computed, two in flight
 constexpr uint32_t kSlabBytes = kPage * D * 2;       // one (page, kv head) slab of K or of V
 constexpr uint32_t kStageBytes = 2 * kSlabBytes;
 constexpr long long kWaitCycles = 2000000000ll;      // ~1 s
@@ -71,13 +71,14 @@ __device__ __forceinline__ uint64_t l2_stream_policy() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
   return pol;
 }
-// One (page, kv head) slab, 4 KB, as one box: lands as [d half][16 tokens][64 elements], 128-byte swizzle.
-__device__ __forceinline__ void tma_load_slab(uint32_t dst, const CUtensorMap *map, int head, int page, uint64_t *bar,
-                                              uint64_t policy) {
+// The K slab and the V slab of one (page, kv head), 8 KB, as one box: lands as [pool][d half][16 tokens][64 elements]
+// with the 128-byte swizzle.  `slab` = page * Hkv + kv head.
+__device__ __forceinline__ void tma_load_stage(uint32_t dst, const CUtensorMap *map, int slab, uint64_t *bar,
+                                               uint64_t policy) {
   asm volatile(
       "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;\n"
-      ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(0), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
+      ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(0), "r"(slab), "r"(0), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
@@ -112,7 +113,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 __global__ void __launch_bounds__(kW * 32)
-suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t k_off, uint32_t v_off,
                   const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
                   float *__restrict__ lse_part) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -180,20 +181,21 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __g
   const uint64_t pol = l2_stream_policy();
   uint8_t(*ring)[kStageBytes] = sm.ring[warp];
   uint64_t *full = sm.full[warp];
-  // Issued by the lane that holds the page's id.  The pad page and a page with a bad id are loaded from a page
-  // that exists (finite data) and masked when computed.
-  auto issue = [&](int o) {
-    if (lane != (o & 31)) return;
+  // Pages o and o + 1 (o even), each issued by the lane that holds its id, both in one predicated instruction
+  // stream.  The pad page and a page with a bad id are loaded from a page that exists (finite data) and masked
+  // when computed.
+  auto issue_pair = [&](int o) {
+    if ((lane & 30) != (o & 30)) return;
+    o += lane & 1;
     int id = (o >> 5) & 1 ? ids1 : ids0;
     if (o >= n_pages) id = __ldg(row_pages + n_pages - 1);
     if ((unsigned)id >= (unsigned)p.num_pages) id = 0;
     const int s = o % kStages;
     mbar_expect_tx(&full[s], kStageBytes);
-    tma_load_slab(smem_u32(ring[s]), &k_map, h, id, &full[s], pol);
-    tma_load_slab(smem_u32(ring[s]) + kSlabBytes, &v_map, h, id, &full[s], pol);
+    tma_load_stage(smem_u32(ring[s]), &kv_map, id * p.Hkv + h, &full[s], pol);
   };
 #pragma unroll 1
-  for (int o = 0; o < kStages && o < n_ord; ++o) issue(o);
+  for (int o = 0; o < kStages && o < n_ord; o += 2) issue_pair(o);
 
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // heads 2tig and 2tig+1 (l: this lane's share)
   float acc[8][4];   // acc[i]: d tile i; [0],[1]: d = 16i + gid, heads 2tig, 2tig+1; [2],[3]: d = 16i + 8 + gid
@@ -206,7 +208,7 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __g
   const int lm = lane >> 3, lr = lane & 7;
   const int k_tok = lr + 8 * (lm & 1), k_chunk = lm >> 1;
   const int v_tok = lr + 8 * (lm >> 1), v_chunk = lm & 1;
-  const uint32_t k_row = (uint32_t)k_tok * 128u, v_row = kSlabBytes + (uint32_t)v_tok * 128u;
+  const uint32_t k_row = k_off + (uint32_t)k_tok * 128u, v_row = v_off + (uint32_t)v_tok * 128u;
 
   bool alive = true;
 #pragma unroll 1
@@ -216,21 +218,37 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __g
     alive = __all_sync(0xffffffffu, alive);
     if (!alive) break;
     const uint32_t base0 = smem_u32(ring[s0]), base1 = smem_u32(ring[s1]);
-    // ---- scores of both pages: four independent chains (page x even/odd k-step)
+    // ---- scores of both pages: four independent chains (page x even/odd k-step).  Fragment loads run eight
+    // slots ahead of the MMAs that use them (slot j: k-step j / 2 of page j % 2), so that no MMA waits for shared memory.
     float sa[2][4], sb[2][4];
 #pragma unroll
     for (int e = 0; e < 2; ++e)
 #pragma unroll
       for (int c = 0; c < 4; ++c) sa[e][c] = sb[e][c] = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
+    uint32_t f[8][4];
+    auto k_load = [&](int j) {
+      const int kk = j >> 1;
       const uint32_t off = (uint32_t)(kk >> 2) * 2048u + k_row + ((((uint32_t)(2 * (kk & 3) + k_chunk)) ^ (uint32_t)(k_tok & 7)) << 4);
-      uint32_t a0, a1, a2, a3;
-      ldsm_x4(base0 + off, a0, a1, a2, a3);
-      mma16816(sa[kk & 1], a0, a1, a2, a3, qf[kk][0], qf[kk][1]);
-      ldsm_x4(base1 + off, a0, a1, a2, a3);
-      mma16816(sb[kk & 1], a0, a1, a2, a3, qf[kk][0], qf[kk][1]);
+      ldsm_x4(((j & 1) ? base1 : base0) + off, f[j & 7][0], f[j & 7][1], f[j & 7][2], f[j & 7][3]);
+    };
+#pragma unroll
+    for (int j = 0; j < 8; ++j) k_load(j);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int kk = j >> 1;
+      if (j & 1) mma16816(sb[kk & 1], f[j & 7][0], f[j & 7][1], f[j & 7][2], f[j & 7][3], qf[kk][0], qf[kk][1]);
+      else mma16816(sa[kk & 1], f[j & 7][0], f[j & 7][1], f[j & 7][2], f[j & 7][3], qf[kk][0], qf[kk][1]);
+      if (j + 8 < 16) k_load(j + 8);
     }
+    // V fragments of the first four d tiles are requested now and arrive while the softmax below runs.
+    // Slot j: d tile 4 (j / 8) + j % 4 of page (j % 8) / 4; a tile's two MMAs (one per page) are four slots apart.
+    auto v_load = [&](int j) {
+      const int i = 4 * (j >> 3) + (j & 3);
+      const uint32_t off = (uint32_t)(i >> 2) * 2048u + v_row + ((((uint32_t)(2 * (i & 3) + v_chunk)) ^ (uint32_t)(v_tok & 7)) << 4);
+      ldsm_x4_trans((((j & 7) >> 2) ? base1 : base0) + off, f[j & 7][0], f[j & 7][1], f[j & 7][2], f[j & 7][3]);
+    };
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v_load(j);
     // ---- masks: tokens at or beyond the chunk's end, the pad page, pages with a bad id
     const int tok0 = sp.lo + o * kPage;
     const uint32_t gm = (o >> 5) & 1 ? good1 : good0;   // o is even: o and o + 1 lie in the same block of 32
@@ -277,19 +295,13 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __g
       }
     // ---- O^T += V^T P^T for both pages
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t off = (uint32_t)(i >> 2) * 2048u + v_row + ((((uint32_t)(2 * (i & 3) + v_chunk)) ^ (uint32_t)(v_tok & 7)) << 4);
-      uint32_t a0, a1, a2, a3;
-      ldsm_x4_trans(base0 + off, a0, a1, a2, a3);
-      mma16816(acc[i], a0, a1, a2, a3, pb[0][0], pb[0][1]);
-      ldsm_x4_trans(base1 + off, a0, a1, a2, a3);
-      mma16816(acc[i], a0, a1, a2, a3, pb[1][0], pb[1][1]);
+    for (int j = 0; j < 16; ++j) {
+      const int i = 4 * (j >> 3) + (j & 3), pg = (j & 7) >> 2;
+      mma16816(acc[i], f[j & 7][0], f[j & 7][1], f[j & 7][2], f[j & 7][3], pb[pg][0], pb[pg][1]);
+      if (j + 8 < 16) v_load(j + 8);
     }
     __syncwarp();   // every lane has read both stages before they are refilled
-    if (o + kStages < n_ord) {
-      issue(o + kStages);
-      issue(o + kStages + 1);
-    }
+    if (o + kStages < n_ord) issue_pair(o + kStages);
     // Page ids: block k's register is reloaded with block k+2 once block k is consumed; the validity mask of the
     // new ids is taken half a block later, when the load has long returned.
     const int done = o + 2;
@@ -330,17 +342,23 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap k_map, const __g
 }  // namespace
 
 struct SuffixTmaPlan {
-  CUtensorMap k_map, v_map;
+  CUtensorMap kv_map;
+  uint32_t k_off, v_off;   // where a stage holds the K slab and the V slab
 };
 
 int suffix_tma_items_per_cta() { return kW; }
 
-// Tensor maps over the two pools (one 4 KB box per (page, kv head) slab).  nullptr when unavailable.
+// One tensor map over both pools (one 8 KB box per (page, kv head): its K slab and its V slab).  nullptr when
+// unavailable, e.g. when the pools lie 2^40 bytes or more apart.
 SuffixTmaPlan *suffix_tma_plan(const Params &p, int dtype) {
   if (dtype != MC_BF16 || p.d != D || p.g < 1 || p.g > 8) return nullptr;
   SuffixTmaPlan *plan = new SuffixTmaPlan();
-  if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, true) ||
-      !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true) ||
+  const uintptr_t ka = reinterpret_cast<uintptr_t>(p.k_pool), va = reinterpret_cast<uintptr_t>(p.v_pool);
+  plan->k_off = ka < va ? 0u : kSlabBytes;
+  plan->v_off = ka < va ? kSlabBytes : 0u;
+  if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||
+      !encode_kv_pair_map(&plan->kv_map, ka < va ? p.k_pool : p.v_pool, (unsigned long long)(ka < va ? va - ka : ka - va),
+                          p.num_pages, p.Hkv) ||
       cudaFuncSetAttribute(suffix_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem)) !=
           cudaSuccess) {
     (void)cudaGetLastError();
@@ -366,7 +384,7 @@ mc_status_t launch_suffix_tma(const Params &p, const SuffixTmaPlan *plan, const 
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = beside_previous ? 1 : 0;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, suffix_tma_kernel, p, plan->k_map, plan->v_map,
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, suffix_tma_kernel, p, plan->kv_map, plan->k_off, plan->v_off,
                                            reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part);
   count_launch();
   return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
