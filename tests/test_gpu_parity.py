@@ -102,6 +102,28 @@ def test_append_sweep_matches_oracle_every_step(name):
     dp.close()
 
 
+def test_appends_that_open_new_chunks(monkeypatch):
+    """Suffixes that end exactly on a chunk boundary: the appended token opens a chunk that had no tokens when
+    the layout (and the suffix pass's serving order) was made, and later appends fill it."""
+    monkeypatch.setenv("MC_SUFFIX_PART_TOKENS", "32")
+    cfg = wl.scaled_down(wl.CONFIGS["cfg2"], "boundary", C=6, prefix=("fixed", 200),
+                         suffix=("fixed", (0, 32, 64, 31, 96, 33)), append_steps=3)
+    hp = wl.make_host_problem(cfg, headroom_tokens=40)
+    dp = DeviceProblem.from_host(hp)
+    assert dp.geom.suffix_part_tokens == 32
+    for step in range(1, 36):
+        k_new, v_new = wl.draw_append(cfg, step)
+        q = wl.draw_q(cfg, step)
+        mc.mc_decode_step(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new), to_device(cfg, q), cfg.scale,
+                          dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes)
+        hp.append(k_new, v_new)
+        if step in (1, 2, 17, 33, 35):
+            torch.cuda.synchronize()
+            check_close(cfg, dp.o, dp.lse, *oracle_full(hp, q))
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    dp.close()
+
+
 def test_parts_match_oracle_on_their_token_ranges():
     cfg = SMALL["cfg2s"]
     hp = wl.make_host_problem(cfg)
