@@ -41,7 +41,7 @@ def suffix_traffic(algorithmic_bytes):
     import hashlib
     if SUFFIX_TRAFFIC_RATIO is None:
         return None
-    src = os.path.join(ROOT, "paper_2601_05475_b200", "csrc", "mc_mma.cu")
+    src = os.path.join(ROOT, "paper_2601_05475_b200", "csrc", "mc_suffix_tma.cu")
     try:
         if hashlib.sha1(open(src, "rb").read()).hexdigest() != SUFFIX_KERNEL_SHA1:
             return None
@@ -385,7 +385,7 @@ def run_gpu(args):
                        "multi_gpu": "replicas only"},
             "frac_of_8tbs": value / world / NOMINAL_HBM_GBS,
             "candidate_tokens_per_s": world * cfg.B / (ms * 1e-3),
-            "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel<suffix>", "achieved": suffix_gbs, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "suffix_tma_kernel", "achieved": suffix_gbs, "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": suffix_gbs / peak,
                          "frac_of_8tbs": suffix_gbs / NOMINAL_HBM_GBS, "traffic": suffix_traffic(main["suffix_bytes"]),
                          "kernel_ms": main["suffix_ms"], "algorithmic_bytes": main["suffix_bytes"]},

@@ -180,15 +180,6 @@ int choose_splits(const Params &p, const LevelWork &w, double budget_us) {
   return nsp > 8 ? 8 : nsp < 1 ? 1 : nsp;
 }
 
-// Persistent CTAs for `items` items of `tiles` tiles in all: the fewest whose rounds still end in the budget.
-int choose_ctas(double items, double tiles, double budget_us) {
-  const double avg_item_us = tiles / items * kTileUs + kItemUs;
-  int rounds = (int)(0.7 * budget_us / avg_item_us);
-  if (rounds < 1) rounds = 1;
-  const int ctas = (int)((items + rounds - 1) / rounds);
-  return ctas < 8 ? 8 : ctas;
-}
-
 }  // namespace
 }  // namespace mc
 
@@ -259,11 +250,10 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   }
 
   // Part geometry.  Suffix chunks come from the table stride (the lengths live on the device and may grow).
-  // Prefix splits and the number of persistent CTAs of the tensor-core prefix pass are sized together, once per
-  // level, from the lengths as they are now.  The prefix pass should finish inside the suffix pass's HBM time
-  // while holding as few SMs as possible (an SM it holds runs the suffix pass at half occupancy), and every work
-  // item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be long: as few
-  // splits as still let one item fit the time budget.  Constants are measured for this kernel pair.
+  // Prefix splits and the CTAs of the tensor-core prefix pass are sized once per level from the lengths as they
+  // are now.  The prefix pass runs beside the suffix pass and should end well inside the suffix pass's HBM time;
+  // every work item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be
+  // long: as few splits as still let one item fit that time.  Constants are measured for this kernel pair.
   const int max_s = d->max_suffix_pages * mc::kPage;
   double suffix_us = 0.0, suffix_tokens_now = -1.0;
   int32_t *sl = nullptr;
@@ -283,15 +273,16 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
   if (ts > 4096) ts = 4096;
   if (suffix_tokens_now >= 0.0) {
-    // A small problem is bound by one warp's page-after-page latency, not by HBM: shorter chunks until the
-    // (kv head, chunk) items fill the warps the device holds at once (8 per SM), down to 4 pages a chunk.
+    // A small problem cannot keep every warp slot busy with chunks of that size: shorter chunks, about the
+    // tokens one of the device's warp slots (8 per SM) gets, in steps of 128 tokens, down to 4 pages a chunk.
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       sms = 148;
     (void)cudaGetLastError();
     const double per_warp = suffix_tokens_now * p.Hkv / (8.0 * sms);
-    int tpar = mc::pow2_floor(per_warp < 64.0 ? 64 : per_warp > 4096.0 ? 4096 : (int)per_warp);
+    int tpar = per_warp < 128.0 ? mc::pow2_floor(per_warp < 64.0 ? 64 : (int)per_warp)
+                                : per_warp > 4096.0 ? 4096 : (int)per_warp / 128 * 128;
     if (tpar < ts) ts = tpar;
   }
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
@@ -299,15 +290,12 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   // The levels of the cascade share one persistent grid, so every item has the whole budget.
   mc::LevelWork work[1 + mc::kMaxOuterLevels];
   int nsp[1 + mc::kMaxOuterLevels];
-  double all_items = 0.0, all_tiles = 0.0;
   const double budget_us = suffix_us * 0.9;
   int part_base = 0;
   for (int k = 0; k <= n_outer; ++k) {   // k = 0: the base level; part slots in this order, then the suffix chunks
     mc::Params &pk = k == 0 ? p : L->outer_p[k - 1];
     work[k] = mc::level_work(pk);
     nsp[k] = mc::choose_splits(pk, work[k], budget_us);
-    all_items += (double)work[k].pairs * nsp[k];
-    all_tiles += work[k].tiles;
     const int max_p = pk.max_pp * mc::kPage;
     int tp = ((max_p + nsp[k] - 1) / nsp[k] + 127) / 128 * 128;
     if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0)
@@ -402,9 +390,12 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
         max_group[i] = work[k].max_group;
         all = all && mc::prefix_tc_supported(levels[i], d->dtype) && max_group[i] <= p.B;
       }
-      int ctas = mc::env_int("MC_PREFIX_CTAS", 0);
-      if (ctas <= 0) ctas = mc::choose_ctas(all_items, all_tiles, budget_us);
-      if (all) L->tc_plan = mc::prefix_tc_plan(levels, max_group, n_outer + 1, sms, ctas > sms ? sms : ctas);
+      // The suffix pass reaches the memory roofline from little more than half of the SMs and cannot share an SM
+      // with a prefix CTA, so the prefix pass gets enough CTAs to end early (a tenth of the suffix pass's time,
+      // measured alone; beside the suffix stream it runs about a third longer) and frees its SMs for the rest.
+      if (all)
+        L->tc_plan = mc::prefix_tc_plan(levels, max_group, n_outer + 1, sms, mc::env_int("MC_PREFIX_CTAS", 0),
+                                        0.1 * budget_us, mc::kTileUs, mc::kItemUs);
     }
     (void)cudaGetLastError();
   }

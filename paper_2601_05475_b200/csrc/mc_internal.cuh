@@ -100,7 +100,8 @@ int mma_items_per_cta();
 constexpr int kMaxTcLevels = 4;
 struct PrefixTcPlan;
 bool prefix_tc_supported(const Params &p, int dtype);
-PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int max_ctas);
+PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int fixed_ctas,
+                             double target_us, double tile_us, double item_us);
 void prefix_tc_plan_free(PrefixTcPlan *plan);
 int prefix_tc_grid(const PrefixTcPlan *plan);
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,

@@ -15,6 +15,12 @@
 // 64 of the tile's 128 columns) do the softmax, the rescale and the epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
+#include <algorithm>
+#include <functional>
+#include <queue>
+#include <utility>
+#include <vector>
+
 #include "mc_internal.cuh"
 
 namespace mc {
@@ -23,7 +29,6 @@ namespace {
 constexpr int D = 128;
 constexpr int kTileM = 128;      // stacked query rows per tile
 constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
-constexpr int kPagesPerTile = kTileN / kPage;
 constexpr int kKSlots = 3;        // K tiles in flight or in use (TMA, two 2 KB boxes per page: one per d half)
 constexpr int kVSlots = 2;        // V tiles (TMA, one 4 KB box per page)
 constexpr int kSoftmaxThreads = 256;   // two threads per row: columns [0,64) and [64,128)
@@ -244,10 +249,11 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
   return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
 }
 
-__global__ void __maxnreg__(104)
+__global__ void __maxnreg__(160)
 prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
-                 float *__restrict__ o_part, float *__restrict__ lse_part, int n_items) {
+                 float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
+                 const int32_t *__restrict__ cta_begin) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base
@@ -256,6 +262,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = p.g, cand_per_tile = kTileM / g;
+  // this CTA's items: a slice of the list made when the layout was created (balanced by the lengths then)
+  const int k_begin = __ldg(cta_begin + blockIdx.x), k_end = __ldg(cta_begin + blockIdx.x + 1);
 
   if (threadIdx.x == 0) {
     // This CTA holds its SM now: a kernel launched behind this one as its programmatic dependent (the suffix
@@ -306,11 +314,11 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     bool ok = true;
 
     auto next_item = [&](int from, Item &out) -> int {
-      for (int i = from; i < n_items; i += gridDim.x) {
-        out = decode_item(p, lvs, i);
-        if (item_has_work(out, cand_per_tile)) return i;
+      for (int k = from; k < k_end; ++k) {
+        out = decode_item(p, lvs, __ldg(item_list + k));
+        if (item_has_work(out, cand_per_tile)) return k;
       }
-      return n_items;
+      return k_end;
     };
     // Staging of one query tile (128 rows x 16 chunks of 16 bytes) proceeds in 8 rounds of 8 chunks per
     // lane.  Round i's loads are issued in one call and stored (swizzled) in the next, so that their
@@ -354,14 +362,14 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     };
 
     Item it, nxt;
-    int cur = next_item(blockIdx.x, it);
-    if (cur < n_items) {
+    int cur = next_item(k_begin, it);
+    if (cur < k_end) {
       int round = 0;
       while (ok && round <= kQRounds) ok = q_step(it, 0, round);
     }
-    while (ok && cur < n_items && !sm.abort) {
-      const int nxt_idx = next_item(cur + gridDim.x, nxt);
-      int round = nxt_idx < n_items ? 0 : kQRounds + 1;   // staging state of the next item's query tile
+    while (ok && cur < k_end && !sm.abort) {
+      const int nxt_idx = next_item(cur + 1, nxt);
+      int round = nxt_idx < k_end ? 0 : kQRounds + 1;   // staging state of the next item's query tile
       const int last_pg = (it.hi - 1) >> 4;
       for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
         // page ids of the tile's 8 pages (lane pg holds page pg); pages past the end of the prefix repeat the
@@ -409,8 +417,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
-        const Item it = decode_item(p, lvs, item);
+      for (int k = k_begin; k < k_end && !sm.abort; ++k) {
+        const Item it = decode_item(p, lvs, __ldg(item_list + k));
         if (!item_has_work(it, cand_per_tile)) continue;
         const int qb = it_n & 1;
         if (!mbar_wait(sm, p, &sm.q_ready[qb], (it_n >> 1) & 1)) break;
@@ -479,8 +487,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       ++pair_n;
       return w;
     };
-    for (int item = blockIdx.x; item < n_items && !sm.abort; item += gridDim.x) {
-      const Item it = decode_item(p, lvs, item);
+    for (int k = k_begin; k < k_end && !sm.abort; ++k) {
+      const Item it = decode_item(p, lvs, __ldg(item_list + k));
       if (it.mt * cand_per_tile >= it.n_cand) continue;
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
@@ -715,6 +723,7 @@ struct PrefixTcPlan {
   CUtensorMap k_map, v_map;
   TcLevels levels;
   int n_items, grid;
+  int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
 bool prefix_tc_supported(const Params &p, int dtype) {
@@ -722,12 +731,40 @@ bool prefix_tc_supported(const Params &p, int dtype) {
          p.prefix_part_tokens % kTileN == 0;
 }
 
-// Host-side preparation at layout-create time: tensor maps over the two pools and the items of every level
-// (`levels[k]` with at most `max_group[k]` candidates in one group), dealt to one persistent grid in the
-// order given.  Returns nullptr when unavailable.
-PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int max_ctas) {
+namespace {
+
+// Longest-processing-time-first assignment of items (sorted by cost, descending) to `grid` CTAs; returns the
+// largest CTA load and, if asked, which CTA each item went to.
+double lpt_assign(const std::vector<int> &by_cost, const std::vector<double> &cost, int grid, std::vector<int> *owner) {
+  typedef std::pair<double, int> Load;   // (load, CTA); the least loaded CTA on top
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int c = 0; c < grid; ++c) heap.push(Load(0.0, c));
+  double longest = 0.0;
+  for (size_t i = 0; i < by_cost.size(); ++i) {
+    Load l = heap.top();
+    heap.pop();
+    l.first += cost[(size_t)by_cost[i]];
+    if (l.first > longest) longest = l.first;
+    if (owner) (*owner)[(size_t)by_cost[i]] = l.second;
+    heap.push(l);
+  }
+  return longest;
+}
+
+}  // namespace
+
+// Host-side preparation at layout-create time: tensor maps over the two pools, and the items of every level
+// (`levels[k]` with at most `max_group[k]` candidates in one group) dealt to the CTAs of one persistent grid.
+// An item's cost is estimated from the lengths as they are now (`tile_us` per 128 x 128 tile, `item_us` per item);
+// the items are assigned longest first to the least loaded CTA, and the grid is the smallest (at least 8 CTAs, at
+// most 7/16 of the SMs: the suffix pass, which cannot share an SM with this kernel's CTAs, reaches the memory
+// roofline from the rest) whose most loaded CTA stays within `target_us` - or `fixed_ctas` CTAs if that is positive.  The lists stay
+// valid when the lengths change later; only their balance is the create-time one.  nullptr when unavailable.
+PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int fixed_ctas,
+                             double target_us, double tile_us, double item_us) {
   if (n_levels < 1 || n_levels > kMaxTcLevels) return nullptr;
   PrefixTcPlan *plan = new PrefixTcPlan();
+  plan->dev_lists = nullptr;
   const Params &p = levels[0];
   if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
       !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true)) {
@@ -736,6 +773,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   }
   long long items = 0;
   plan->levels.n = n_levels;
+  std::vector<double> cost;
   for (int k = 0; k < n_levels; ++k) {
     const Params &pk = levels[k];
     TcLevel &lv = plan->levels.lv[k];
@@ -747,37 +785,90 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.part_base = pk.prefix_part_base;
     lv.part_tokens = pk.prefix_part_tokens;
     lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
-    items += (long long)pk.G * pk.Hkv * pk.n_prefix_parts * lv.n_mt;
-    if (items > 0x7fffffffLL) {
+    const long long level_items = (long long)pk.G * pk.Hkv * pk.n_prefix_parts * lv.n_mt;
+    items += level_items;
+    if (items > (1ll << 24)) {
       delete plan;
       return nullptr;
     }
     lv.item_end = (int32_t)items;
+    // cost of each item of the level, in the kernel's numbering (row tile fastest, then split, kv head, group)
+    std::vector<int32_t> go((size_t)pk.G + 1), len((size_t)pk.G);
+    const bool known =
+        cudaMemcpy(go.data(), pk.group_offsets, sizeof(int32_t) * go.size(), cudaMemcpyDeviceToHost) == cudaSuccess &&
+        cudaMemcpy(len.data(), pk.prefix_len, sizeof(int32_t) * len.size(), cudaMemcpyDeviceToHost) == cudaSuccess;
+    (void)cudaGetLastError();
+    const int cand_per_tile = kTileM / pk.g;
+    for (long long it = 0; it < level_items; ++it) {
+      const int mt = (int)(it % lv.n_mt);
+      long long r = it / lv.n_mt;
+      const int sp = (int)(r % lv.n_splits);
+      r /= lv.n_splits;
+      const int j = (int)(r / pk.Hkv);
+      const int n_cand = known ? go[(size_t)j + 1] - go[(size_t)j] : max_group[k];
+      const long long cap = (long long)pk.max_pp * kPage;
+      long long l = known ? len[(size_t)j] : cap;
+      l = l < 0 ? 0 : l > cap ? cap : l;
+      const long long lo = (long long)sp * lv.part_tokens;
+      const long long tokens = (l < lo + lv.part_tokens ? l : lo + lv.part_tokens) - lo;
+      double c = 0.0;
+      if (tokens > 0 && mt * cand_per_tile < n_cand) c = (double)((tokens + kTileN - 1) / kTileN) * tile_us + item_us;
+      cost.push_back(c);
+    }
   }
   plan->n_items = (int)items;
-  int grid = plan->n_items < sm_count ? plan->n_items : sm_count;
-  if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;
-  if (grid < 1) grid = 1;
-  // items are dealt round-robin: the fewest CTAs that keep the same number of rounds hold fewer SMs
-  const int rounds = (plan->n_items + grid - 1) / grid;
-  if (rounds > 0) grid = (plan->n_items + rounds - 1) / rounds;
-  plan->grid = grid < 1 ? 1 : grid;
+  std::vector<int> by_cost((size_t)plan->n_items);
+  for (int i = 0; i < plan->n_items; ++i) by_cost[(size_t)i] = i;
+  std::stable_sort(by_cost.begin(), by_cost.end(), [&](int a, int b) { return cost[(size_t)a] > cost[(size_t)b]; });
+  int live = 0;
+  for (int i = 0; i < plan->n_items; ++i) live += cost[(size_t)i] > 0.0;
+  const int most = live < 1 ? 1 : live < sm_count ? live : sm_count;
+  int grid;
+  if (fixed_ctas > 0) {
+    grid = fixed_ctas < most ? fixed_ctas : most;
+  } else {
+    const int cap = sm_count * 7 / 16 > 8 ? sm_count * 7 / 16 : 8;
+    int lo = 8 < most ? 8 : most, hi = most < cap ? most : cap;   // smallest grid in [lo, hi] that meets the target (hi if none does)
+    while (lo < hi) {
+      const int mid = (lo + hi) / 2;
+      if (lpt_assign(by_cost, cost, mid, nullptr) <= target_us) hi = mid; else lo = mid + 1;
+    }
+    grid = lo;
+  }
+  plan->grid = grid;
+  std::vector<int> owner((size_t)plan->n_items, 0);
+  lpt_assign(by_cost, cost, grid, &owner);
+  std::vector<int32_t> lists((size_t)grid + 1 + (size_t)plan->n_items, 0);
+  for (int i = 0; i < plan->n_items; ++i) lists[(size_t)owner[(size_t)i] + 1] += 1;
+  for (int c = 0; c < grid; ++c) lists[(size_t)c + 1] += lists[(size_t)c];
+  std::vector<int32_t> fill(lists.begin(), lists.begin() + grid);
+  for (int i = 0; i < plan->n_items; ++i) {   // costliest first within each CTA
+    const int it = by_cost[(size_t)i];
+    lists[(size_t)grid + 1 + (size_t)fill[(size_t)owner[(size_t)it]]++] = it;
+  }
   if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)sizeof(Smem)) != cudaSuccess) {
-    delete plan;
+                           (int)sizeof(Smem)) != cudaSuccess ||
+      cudaMalloc(&plan->dev_lists, sizeof(int32_t) * lists.size()) != cudaSuccess ||
+      cudaMemcpy(plan->dev_lists, lists.data(), sizeof(int32_t) * lists.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+    (void)cudaGetLastError();
+    prefix_tc_plan_free(plan);
     return nullptr;
   }
   return plan;
 }
 
-void prefix_tc_plan_free(PrefixTcPlan *plan) { delete plan; }
+void prefix_tc_plan_free(PrefixTcPlan *plan) {
+  if (!plan) return;
+  cudaFree(plan->dev_lists);
+  delete plan;
+}
 int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
 
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {
   prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
       p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part,
-      lse_part, plan->n_items);
+      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists);
   count_launch();
   return check_launch();
 }
