@@ -33,8 +33,8 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/kernels_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch on cfg2; the traffic
 # grows in proportion to the tokens streamed, so it is scaled by the units of the timed workload).  The ratio
 # is only reported while the kernel source still has the hash it had when the counters were taken.
-SUFFIX_TRAFFIC_RATIO = 1.0208
-SUFFIX_KERNEL_SHA1 = "3395467429623323ca330a89b6fdb8e312fd3a04"
+SUFFIX_TRAFFIC_RATIO = 1.0145
+SUFFIX_KERNEL_SHA1 = "2ab0fcfbe70b0b84062a61c9673256b55cce990d"
 
 
 def suffix_traffic(algorithmic_bytes):
