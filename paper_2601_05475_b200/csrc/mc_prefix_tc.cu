@@ -4,15 +4,19 @@
 // stacked into dense 128-row tiles (row = candidate * g + head-in-group), so the group's prefix K/V is
 // streamed once for the whole group instead of once per candidate:
 //     S = Q_s K^T          128 x 128 tile, tcgen05.mma, operands in shared memory, accumulator in TMEM
-//     P = exp2(S*c - m)    one thread per row reads its row of S from TMEM, writes bf16 P back to TMEM
+//     P = exp2(S*c - m)    two threads per row read the row of S from TMEM and write bf16 P over it
 //     O += P V             tcgen05.mma, P from TMEM, V in its natural [token][d] layout (MN-major B operand)
 // K/V pages reach shared memory by TMA through tensor maps laid over the paged pools (the page id is a TMA
 // coordinate): V as one 4 KB box per page, K as two 2 KB boxes per page (one per 64-element d half).
 //
-// Work item = (group, kv head, prefix split, 128-row tile); persistent CTAs take items round-robin.
-// Warp roles: warp 0 issues the TMA copies and stages the next item's query tile, warp 1 lane 0 issues
-// the MMAs (warp 1 owns the TMEM allocation), warps 2-9 (256 threads, two per TMEM lane, each owning
-// 64 of the tile's 128 columns) do the softmax, the rescale and the epilogue.
+// Work item = (group, kv head, prefix split, 128-row tile); every CTA has a list of items.  Inside an item the
+// 128-token K/V tiles are dealt alternately to two independent streams ("teams"): each team has its own S and O
+// accumulators in TMEM (S0 O0 S1 O1 = 512 columns), its own 256 softmax threads and its own running maximum and
+// row sum, and writes a part slot of its own - the merge combines the two like any two parts.  While one team
+// computes the exponentials of its tile, the tensor pipe runs the other team's products.
+// Warp roles: warp 0 and warps 18, 19 issue the TMA copies (warp 0 also stages the next item's query tile), warp 1
+// lane 0 issues the MMAs (warp 1 owns the TMEM allocation), warps 2-9 are team 0 and warps 10-17 team 1 (two
+// threads per TMEM lane, each owning 64 of the tile's 128 columns): softmax, rescale, epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
 #include <algorithm>
@@ -31,12 +35,15 @@ constexpr int kTileM = 128;      // stacked query rows per tile
 constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
 constexpr int kKSlots = 3;        // K tiles in flight or in use (TMA, two 2 KB boxes per page: one per d half)
 constexpr int kVSlots = 2;        // V tiles (TMA, one 4 KB box per page)
-constexpr int kSoftmaxThreads = 256;   // two threads per row: columns [0,64) and [64,128)
-constexpr int kThreads = 64 + kSoftmaxThreads;
+constexpr int kTeams = 2;              // independent tile streams: tile t of an item belongs to team t & 1
+constexpr int kSoftmaxThreads = 256;   // per team, two threads per row: columns [0,64) and [64,128)
+constexpr int kProducers = 3;          // copy-issuing warps: K d-half 0 (+ query staging), K d-half 1, V
+constexpr int kThreads = 64 + kTeams * kSoftmaxThreads + (kProducers - 1) * 32;
 constexpr uint32_t kHalfBytes = kTileN * 64 * 2;        // one head-dim (or token) half of a 128x128 bf16 tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;         // 32 KB
 constexpr uint32_t kPageBytes = kPage * D * 2;          // one (page, kv head) slab; one TMA box for V
-constexpr uint32_t kTmemCols = 512;                     // S: [0,128)  O: [128,256)  P (bf16 pairs): [256,320), [320,384)
+constexpr uint32_t kTmemCols = 512;                     // team T: S at 256 T, O at 256 T + 128; P (bf16 pairs) over S:
+                                                        // the thread that owns S columns [64 h, 64 h + 64) writes [64 h, 64 h + 32)
 constexpr long long kWaitCycles = 2000000000ll;         // ~1 s
 
 struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
@@ -44,9 +51,9 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint8_t k[kKSlots][kTileBytes];     // [d half][128 tokens][64], 128-byte swizzle
   uint8_t v[kVSlots][kTileBytes];     // [page][d half][16 tokens][64], 128-byte swizzle
   uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
-  uint64_t q_ready[2], q_free[2], s_full, s_free, p_full[2], pv_done[2];
-  uint64_t pair[4];                   // the two warps that share a TMEM lane quadrant meet here
-  float xch[2][2][kTileM];            // [tile parity][column half][row]: row extremum / row sum exchange
+  uint64_t q_ready[2], q_free[2], s_full[kTeams], p_full[kTeams], pv_done[kTeams];
+  uint64_t pair[kTeams][4];           // the two warps of a team that share a TMEM lane quadrant meet here
+  float xch[kTeams][2][kTileM];       // [team][column half][row]: row extremum / row sum exchange
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
   volatile int abort;
@@ -185,6 +192,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 
@@ -237,7 +252,7 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
     latch(p, kDevBadPage);
     len = len < 0 ? 0 : cap;
   }
-  it.part = L.part_base + sp;
+  it.part = L.part_base + kTeams * sp;   // team T writes slot it.part + T
   it.lo = sp * L.part_tokens;
   it.hi = min(len, it.lo + L.part_tokens);
   it.pages = L.prefix_pages + (size_t)it.j * L.max_pp;
@@ -249,7 +264,7 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
   return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
 }
 
-__global__ void __maxnreg__(160)
+__global__ void __maxnreg__(96)
 prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
                  float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
@@ -270,7 +285,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     // pass, which needs nothing this kernel writes) may start as soon as every CTA of this grid has said so.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     for (int s = 0; s < kKSlots; ++s) {
-      mbar_init(&sm.full_k[s], 1);
+      mbar_init(&sm.full_k[s], 2);   // one arrival per K d half
       mbar_init(&sm.empty_k[s], 1);
     }
     for (int s = 0; s < kVSlots; ++s) {
@@ -281,13 +296,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       mbar_init(&sm.q_ready[b], 32);
       mbar_init(&sm.q_free[b], 1);
     }
-    mbar_init(&sm.s_full, 1);
-    mbar_init(&sm.s_free, kSoftmaxThreads);
-    mbar_init(&sm.p_full[0], kSoftmaxThreads);
-    mbar_init(&sm.p_full[1], kSoftmaxThreads);
-    for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[i], 64);
-    mbar_init(&sm.pv_done[0], 1);
-    mbar_init(&sm.pv_done[1], 1);
+    for (int t = 0; t < kTeams; ++t) {
+      mbar_init(&sm.s_full[t], 1);
+      mbar_init(&sm.p_full[t], kSoftmaxThreads);
+      mbar_init(&sm.pv_done[t], 1);
+      for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[t][i], 64);
+    }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -300,16 +314,19 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tmem_s = tmem, tmem_o = tmem + kTileN, tmem_p = tmem + 2 * kTileN;
+  // team T: S at columns [256 T, 256 T + 128), O at [256 T + 128, 256 T + 256)
 
   // Counters advance identically in every role: `kt` counts K/V tiles, `it_n` counts items with work.
   uint32_t kt = 0, it_n = 0;
 
-  if (warp == 0) {
-    // ---------------------------------------------------------------- producer (all 32 lanes)
-    // K/V: a tile is 32 TMA boxes (K and V, 8 pages, 2 head-dim halves), one per lane.
-    // Q:   the stacked query tile of the NEXT item is staged (plain loads, swizzled stores) into the
+  if (warp == 0 || warp >= 2 + kTeams * (kSoftmaxThreads / 32)) {
+    // ---------------------------------------------------------------- producers (three warps, all 32 lanes)
+    // K/V: a tile is 24 TMA boxes (K: 8 pages x 2 head-dim halves of 2 KB, V: 8 pages of 4 KB).  Issuing a box
+    //      costs the issuing warp well over a hundred cycles (measured), so the boxes of a tile are shared out:
+    //      warp 0 takes K's first d half, the two extra warps K's second d half and V; 8 boxes from 8 lanes each.
+    // Q:   warp 0 also stages the stacked query tile of the NEXT item (plain loads, swizzled stores) into the
     //      other Q buffer while the current item is being computed.
+    const int prole = warp == 0 ? 0 : warp - (1 + kTeams * (kSoftmaxThreads / 32));   // 0, 1: K d half; 2: V
     const uint64_t policy = l2_keep_policy();
     bool ok = true;
 
@@ -363,47 +380,57 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 
     Item it, nxt;
     int cur = next_item(k_begin, it);
-    if (cur < k_end) {
+    if (cur < k_end && prole == 0) {
       int round = 0;
       while (ok && round <= kQRounds) ok = q_step(it, 0, round);
     }
     while (ok && cur < k_end && !sm.abort) {
       const int nxt_idx = next_item(cur + 1, nxt);
-      int round = nxt_idx < k_end ? 0 : kQRounds + 1;   // staging state of the next item's query tile
+      int round = nxt_idx < k_end && prole == 0 ? 0 : kQRounds + 1;   // staging state of the next item's query tile
       const int last_pg = (it.hi - 1) >> 4;
-      for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt) {
-        // page ids of the tile's 8 pages (lane pg holds page pg); pages past the end of the prefix repeat the
-        // last valid page: finite data, masked later
-        int pid = __ldg(it.pages + min((t0 >> 4) + (lane & 7), last_pg));
+      // Page ids are read 32 at a time (four tiles' worth, one per lane) a block ahead of their use, so that no
+      // tile waits for a table look-up.  Pages past the end of the prefix repeat the last valid page: finite
+      // data, masked later.
+      auto load_ids = [&](int blk) -> int { return __ldg(it.pages + min((it.lo >> 4) + blk * 32 + lane, last_pg)); };
+      int ids_cur = load_ids(0), ids_next = load_ids(1);
+      int tile = 0;
+      for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt, ++tile) {
+        // lane pg (and every lane with the same low three bits) gets the id of the tile's page pg
+        int pid = __shfl_sync(0xffffffffu, ids_cur, (tile & 3) * 8 + (lane & 7));
+        if ((tile & 3) == 3) {
+          ids_cur = ids_next;
+          ids_next = load_ids((tile >> 2) + 2);
+        }
         const bool in_range = t0 + (lane & 7) * kPage < it.hi, good = (unsigned)pid < (unsigned)p.num_pages;
-        if (lane < 8 && in_range && !good) latch(p, kDevBadPage);
+        if (lane < 8 && in_range && !good && prole == 0) latch(p, kDevBadPage);
         if (!good) pid = 0;   // a bad page id is replaced by page 0 and its 16 columns are masked
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range && good) & 0xffu;
-        // ---- K(t): 16 boxes of 2 KB (lanes 0-15: page = lane & 7, d half = lane >> 3)
-        const int sk = kt % kKSlots;
-        ok = mbar_wait(sm, p, &sm.empty_k[sk], ((kt / kKSlots) & 1) ^ 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane == 0) mbar_expect_tx(&sm.full_k[sk], kTileBytes);
-        __syncwarp();
-        if (lane < 16)
-          tma_load_half_page(sm.k[sk] + (lane >> 3) * kHalfBytes + (lane & 7) * (kPageBytes / 2), &k_map, (lane >> 3) * 64,
-                             it.h, pid, &sm.full_k[sk], policy);
-        // ---- V(t): 8 boxes of 4 KB
-        const int sv = kt % kVSlots;
-        ok = mbar_wait(sm, p, &sm.empty_v[sv], ((kt / kVSlots) & 1) ^ 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // published before the arrive below; the softmax role reads it after the chain of barrier waits
-        // (full -> second/first product -> s_full of a later tile is not enough: it is read after s_full of
-        // THIS tile, which follows full_k of this tile, announced by this warp after this store)
-        if (lane == 0) {
-          sm.page_ok[kt & 7] = okmask;
-          mbar_expect_tx(&sm.full_v[sv], kTileBytes);
+        if (prole < 2) {
+          // ---- K(t), d half `prole`: 8 boxes of 2 KB (lanes 0-7: page = lane)
+          const int sk = kt % kKSlots;
+          ok = mbar_wait(sm, p, &sm.empty_k[sk], ((kt / kKSlots) & 1) ^ 1);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          // page_ok is published before this warp's arrive on full_k; the softmax role reads it after s_full of
+          // THIS tile, which follows full_k of this tile
+          if (lane == 0) {
+            if (prole == 0) sm.page_ok[kt & 7] = okmask;
+            mbar_expect_tx(&sm.full_k[sk], kHalfBytes);
+          }
+          __syncwarp();
+          if (lane < 8)
+            tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64, it.h, pid,
+                               &sm.full_k[sk], policy);
+        } else {
+          // ---- V(t): 8 boxes of 4 KB
+          const int sv = kt % kVSlots;
+          ok = mbar_wait(sm, p, &sm.empty_v[sv], ((kt / kVSlots) & 1) ^ 1);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (lane == 0) mbar_expect_tx(&sm.full_v[sv], kTileBytes);
+          __syncwarp();
+          if (lane < 8) tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, it.h, pid, &sm.full_v[sv], policy);
         }
-        __syncwarp();
-        if (lane >= 16 && lane < 24)
-          tma_load_page(sm.v[sv] + (lane & 7) * kPageBytes, &v_map, it.h, pid, &sm.full_v[sv], policy);
         if (round <= kQRounds) {
           ok = q_step(nxt, it_n + 1, round);
           if (!ok) break;
@@ -417,6 +444,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
+      uint32_t team_tiles[kTeams] = {0u, 0u};   // tiles of each team whose P has been taken (all items)
       for (int k = k_begin; k < k_end && !sm.abort; ++k) {
         const Item it = decode_item(p, lvs, __ldg(item_list + k));
         if (!item_has_work(it, cand_per_tile)) continue;
@@ -426,65 +454,77 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         tc_fence_after();
         const uint32_t q_addr = smem_u32(sm.q[qb]);
         const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
-        // Iteration t issues S(t) = Q K(t)^T as soon as the softmax role holds S(t-1) in registers, then
-        // O += P(t-1) V(t-1) once P(t-1) is staged: the exponentials of tile t-1 overlap the first
-        // product, the row maxima of tile t overlap the second.  The first product of the next item
-        // follows the last second product directly and runs under this item's epilogue.
+        // Tile t belongs to team t & 1.  Per team the order on the tensor pipe is S(t), O += P(t) V(t), S(t+2), ...:
+        // P(t) lies over S(t), so S(t+2) may only follow the second product of tile t; the other team's products
+        // fill the gaps.  Products complete in issue order.  The first product of the next item follows this item's
+        // last second product directly and runs under this item's epilogue.
         bool ok = true;
-        for (int t = 0; t <= n_tiles && ok; ++t) {
-          if (t < n_tiles) {
-            const uint32_t ktq = kt + t;
-            const int s = ktq % kKSlots;
-            if (ktq > 0) ok = mbar_wait(sm, p, &sm.s_free, (ktq - 1) & 1);
-            ok = ok && mbar_wait(sm, p, &sm.full_k[s], (ktq / kKSlots) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_addr = smem_u32(sm.k[s]);
+        auto issue_qk = [&](int t) -> bool {
+          const uint32_t ktq = kt + t;
+          const int s = ktq % kKSlots;
+          if (!mbar_wait(sm, p, &sm.full_k[s], (ktq / kKSlots) & 1)) return false;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(sm.k[s]), tmem_s = tmem + (uint32_t)(t & 1) * 256u;
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-              umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
-            }
-            umma_commit(&sm.empty_k[s]);   // K(t) is free as soon as the first product has read it
-            umma_commit(&sm.s_full);
-            if (t == n_tiles - 1) umma_commit(&sm.q_free[qb]);   // last reader of this item's Q tile
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+            umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
           }
-          if (t > 0) {
-            const uint32_t ktp = kt + t - 1;
-            const int s = ktp % kVSlots;
-            ok = mbar_wait(sm, p, &sm.p_full[ktp & 1], (ktp >> 1) & 1) &&
-                 mbar_wait(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t v_addr = smem_u32(sm.v[s]), p_cols = tmem_p + (ktp & 1) * (kTileN / 2);
-            // one k-step per page: its 16 token rows x both 64-element halves (2 KB apart) are one 4 KB box
+          umma_commit(&sm.empty_k[s]);   // K(t) is free as soon as the first product has read it
+          umma_commit(&sm.s_full[t & 1]);
+          if (t == n_tiles - 1) umma_commit(&sm.q_free[qb]);   // last reader of this item's Q tile
+          return true;
+        };
+        ok = issue_qk(0) && (n_tiles < 2 || issue_qk(1));
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int team = t & 1;
+          const uint32_t ktp = kt + t;
+          const int s = ktp % kVSlots;
+          ok = mbar_wait(sm, p, &sm.p_full[team], team_tiles[team] & 1) &&
+               mbar_wait(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1);
+          if (!ok) break;
+          ++team_tiles[team];
+          tc_fence_after();
+          const uint32_t v_addr = smem_u32(sm.v[s]), tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
+          // one k-step per page: its 16 token rows x both 64-element halves (2 KB apart) are one 4 KB box;
+          // the P columns of tokens [64 h, 64 h + 64) start at S column 64 h
 #pragma unroll
-            for (int kk = 0; kk < kTileN / 16; ++kk)
-              umma_ts(tmem_o, p_cols + kk * 8, smem_desc(v_addr + kk * kPageBytes, kPageBytes / 2, 1024), kIdescPV,
-                      (t > 1) || (kk > 0));
-            umma_commit(&sm.empty_v[s]);
-            umma_commit(&sm.pv_done[ktp & 1]);
-          }
+          for (int kk = 0; kk < kTileN / 16; ++kk)
+            umma_ts(tmem_o, tmem_s + (kk >> 2) * 64 + (kk & 3) * 8, smem_desc(v_addr + kk * kPageBytes, kPageBytes / 2, 1024),
+                    kIdescPV, (t >= kTeams) || (kk > 0));
+          umma_commit(&sm.empty_v[s]);
+          umma_commit(&sm.pv_done[team]);
+          if (t + kTeams < n_tiles) ok = issue_qk(t + kTeams);
         }
         if (!ok) break;
         kt += n_tiles;
       }
     }
   } else {
-    // ---------------------------------------------------------------- softmax / epilogue (256 threads)
+    // ---------------------------------------------------------------- softmax / epilogue (two teams of 256 threads)
+    const int team = (warp - 2) >> 3;          // which of the item's two tile streams
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may access
-    const int half = (warp - 2) >> 2;          // which 64 of the tile's 128 columns this thread owns
+    const int half = ((warp - 2) >> 2) & 1;    // which 64 of the tile's 128 columns this thread owns
     const int r = quad * 32 + lane;            // row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
     uint32_t pair_n = 0;                       // completed meetings of this warp pair
-    // Exchanges one float with the thread that owns the other half of the row (bounded).
-    auto exchange = [&](float mine, float &theirs) -> bool {
-      sm.xch[pair_n & 1][half][r] = mine;
-      mbar_arrive(&sm.pair[quad]);
-      bool w = mbar_wait(sm, p, &sm.pair[quad], pair_n & 1);
-      w = __all_sync(0xffffffffu, w);
-      if (w) theirs = sm.xch[pair_n & 1][half ^ 1][r];
+    uint32_t team_tiles = 0;                   // tiles this team has taken so far (all items)
+    // The two threads of a row meet (bounded).
+    auto meet = [&]() -> bool {
+      mbar_arrive(&sm.pair[team][quad]);
+      bool w = mbar_wait(sm, p, &sm.pair[team][quad], pair_n & 1);
       ++pair_n;
+      return __all_sync(0xffffffffu, w);
+    };
+    // Exchanges one float with the thread that owns the other half of the row.  The slot is reused: between the
+    // exchanges of two tiles lies a barrier round of the whole team (every thread announces its P after reading
+    // here, and the next tile's S follows the product that waited for all of them); around the epilogue's
+    // exchange, which has no such round on either side, the pair meets once more.
+    auto exchange = [&](float mine, float &theirs) -> bool {
+      sm.xch[team][half][r] = mine;
+      const bool w = meet();
+      if (w) theirs = sm.xch[team][half ^ 1][r];
       return w;
     };
     for (int k = k_begin; k < k_end && !sm.abort; ++k) {
@@ -493,58 +533,58 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
-      const size_t slot = qrow * p.n_parts + it.part;
-      if (it.lo >= it.hi) {
+      const size_t slot = qrow * p.n_parts + it.part + team;
+      const int n_tiles = it.lo < it.hi ? (it.hi - it.lo + kTileN - 1) / kTileN : 0;
+      if (team >= n_tiles) {   // no tokens in this split, or a single tile: it is the other team's
         if (row_ok && half == 0) lse_part[slot] = -INFINITY;
+        kt += n_tiles;
         continue;
       }
       float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2); l: this thread's columns only
-      const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
       bool alive = true;
-      for (int t = 0; t < n_tiles && alive; ++t, ++kt) {
+      for (int t = team; t < n_tiles && alive; t += kTeams, ++team_tiles) {
         const int t0 = it.lo + t * kTileN, c0 = half * 64;
-        alive = mbar_wait(sm, p, &sm.s_full, kt & 1);
+        alive = mbar_wait(sm, p, &sm.s_full[team], team_tiles & 1);
         alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
         if (!alive) break;
         tc_fence_after();
         // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
-        const uint32_t page_ok = sm.page_ok[kt & 7];
+        const uint32_t page_ok = sm.page_ok[(kt + t) & 7];
         const bool full_tile = page_ok == 0xffu && t0 + kTileN <= it.hi;
-        // this thread's half row of S into registers, then S is free for the next tile's first product
-        uint32_t sv[2][32];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) tmem_ld32(tmem_s + lane_addr + c0 + c * 32, sv[c]);
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&sm.s_free);
-        if (!full_tile) {   // ragged tail or a bad page: masked scores become -inf (sl2 > 0) / +inf (sl2 < 0)
-          const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
-#pragma unroll
-          for (int c = 0; c < 2; ++c)
+        // This thread's half row of S is read twice, 32 columns at a time - once for the row extremum, once for the
+        // exponentials - so that no more than 32 scores are held in registers at any time.
+        auto load_chunk = [&](int c, uint32_t (&sv)[32]) {
+          tmem_ld32(tmem_s + lane_addr + c0 + c * 32, sv);
+          tmem_wait_ld();
+          if (!full_tile) {   // ragged tail or a bad page: masked scores become -inf (sl2 > 0) / +inf (sl2 < 0)
+            const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int col = c0 + c * 32 + i;
               const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
-              if (!ok) sv[c][i] = masked;
+              if (!ok) sv[i] = masked;
             }
-        }
+          }
+        };
         // row extremum of the raw scores; times sl2 it is the row maximum of the scaled scores
-        float e4[4];
+        float ext = sl2 >= 0.f ? -INFINITY : INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sv[32];
+          load_chunk(c, sv);
+          float e4[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) e4[c] = __uint_as_float(sv[c & 1][c >> 1]);
-        if (sl2 >= 0.f) {
+          for (int i = 0; i < 4; ++i) e4[i] = __uint_as_float(sv[i]);
+          if (sl2 >= 0.f) {
 #pragma unroll
-          for (int i = 2; i < 32; i += 2)
+            for (int i = 4; i < 32; ++i) e4[i & 3] = fmaxf(e4[i & 3], __uint_as_float(sv[i]));
+            ext = fmaxf(ext, fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3])));
+          } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) e4[c] = fmaxf(e4[c], __uint_as_float(sv[c & 1][i + (c >> 1)]));
-        } else {
-#pragma unroll
-          for (int i = 2; i < 32; i += 2)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) e4[c] = fminf(e4[c], __uint_as_float(sv[c & 1][i + (c >> 1)]));
+            for (int i = 4; i < 32; ++i) e4[i & 3] = fminf(e4[i & 3], __uint_as_float(sv[i]));
+            ext = fminf(ext, fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3])));
+          }
         }
-        float ext = sl2 >= 0.f ? fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]))
-                               : fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
         float ext_other = ext;
         alive = exchange(ext, ext_other);
         if (!alive) break;
@@ -556,12 +596,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         bool rescale = false;
         if (mx > m + 8.f) {
           m_use = mx;
-          rescale = t > 0 && m > -INFINITY;
+          rescale = t >= kTeams && m > -INFINITY;
         }
         const float alpha = rescale ? fast_exp2(m - m_use) : 1.f;
         if (__any_sync(0xffffffffu, rescale)) {
-          // every earlier product into O must have completed before O is rescaled in place
-          alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
+          // every earlier product into this team's O must have completed before O is rescaled in place
+          alive = mbar_wait(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
           alive = __all_sync(0xffffffffu, alive);
           if (!alive) break;
           tc_fence_after();
@@ -579,38 +619,41 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         l *= alpha;
         m = m_use;
         const float neg_m = m == -INFINITY ? 0.f : -m;
-        // P goes to TMEM as the A operand of the second product: lane = row, one column per token pair.
-        // The buffer of this tile's parity was last read by the second product of tile kt-2, which the tensor
-        // pipe finished before this tile's first product (products complete in issue order), i.e. before the
-        // s_full wait above returned.
+        // P goes to TMEM as the A operand of the second product: lane = row, one column per token pair, written
+        // over the first half of the S columns this thread has read (the team's next first product, which
+        // overwrites S, is issued after the second product that reads this P).
         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t pw[32];                           // 64 tokens -> 32 packed columns
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sv[32], pw[16];                 // 32 tokens -> 16 packed columns
+          load_chunk(c, sv);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int c = j >> 4, i = (2 * j) & 31;
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c][i]), sl2, neg_m));       // masked: exp2(-inf) = 0
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c][i + 1]), sl2, neg_m));
-          lsum[j & 1] += p0;
-          lsum[2 + (j & 1)] += p1;
-          pw[j] = pack_bf16x2(p0, p1);
+          for (int j = 0; j < 16; ++j) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * j]), sl2, neg_m));       // masked: exp2(-inf) = 0
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * j + 1]), sl2, neg_m));
+            lsum[j & 1] += p0;
+            lsum[2 + (j & 1)] += p1;
+            pw[j] = pack_bf16x2(p0, p1);
+          }
+          // columns [c0 + 16 c, c0 + 16 c + 16): inside S columns [c0, c0 + 32), which this thread is done with
+          // (chunk 1 is re-read from [c0 + 32, c0 + 64) after chunk 0's P has been written)
+          tmem_st16(tmem_s + lane_addr + c0 + c * 16, pw);
         }
-        tmem_st32(tmem_p + lane_addr + (kt & 1) * (kTileN / 2) + half * 32, pw);
         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
         tmem_wait_st();
         tc_fence_before();
-        // p_full counts arrivals, not tiles, and a warp may run a whole tile ahead of a slow one: with a single
-        // barrier its arrival for tile t+1 would complete tile t's phase early.  Two barriers alternate by tile
-        // parity; an arrival for tile t+2 presupposes s_full(t+2), hence s_free(t+1) from every thread, and a
-        // thread arrives there only after its p_full arrival for tile t.
-        mbar_arrive(&sm.p_full[kt & 1]);
+        // p_full counts arrivals, not tiles; no thread can arrive for the team's next tile before this phase
+        // closes, because that tile's S follows the product that waits for this phase.
+        mbar_arrive(&sm.p_full[team]);
       }
+      kt += n_tiles;
       if (!alive) break;
       // epilogue: O / l -> o_part, lse (each thread writes its 64 columns; the row sum is the two halves')
       float l_other = 0.f;
-      alive = exchange(l, l_other);
+      alive = meet() && exchange(l, l_other) && meet();
       if (!alive) break;
       const float l_row = l + l_other;
-      alive = mbar_wait(sm, p, &sm.pv_done[(kt - 1) & 1], ((kt - 1) >> 1) & 1);
+      alive = mbar_wait(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
       if (!__all_sync(0xffffffffu, alive)) break;
       tc_fence_after();
       const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
@@ -726,9 +769,14 @@ struct PrefixTcPlan {
   int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
+bool prefix_tc_shape_supported(const Params &p, int dtype) {
+  return dtype == MC_BF16 && p.d == D && p.g >= 1 && p.g <= kTileM && kTileM % p.g == 0;
+}
+
 bool prefix_tc_supported(const Params &p, int dtype) {
-  return dtype == MC_BF16 && p.d == D && p.g >= 1 && p.g <= kTileM && kTileM % p.g == 0 &&
-         p.prefix_part_tokens % kTileN == 0;
+  // a split is a pair of part slots, one per team, and a whole number of 128-token tiles
+  return prefix_tc_shape_supported(p, dtype) && p.n_prefix_parts % kTeams == 0 &&
+         (p.prefix_part_tokens * kTeams) % kTileN == 0;
 }
 
 namespace {
@@ -781,11 +829,11 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.prefix_pages = pk.prefix_pages;
     lv.prefix_len = pk.prefix_len;
     lv.max_pp = pk.max_pp;
-    lv.n_splits = pk.n_prefix_parts;
+    lv.n_splits = pk.n_prefix_parts / kTeams;
     lv.part_base = pk.prefix_part_base;
-    lv.part_tokens = pk.prefix_part_tokens;
+    lv.part_tokens = pk.prefix_part_tokens * kTeams;
     lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
-    const long long level_items = (long long)pk.G * pk.Hkv * pk.n_prefix_parts * lv.n_mt;
+    const long long level_items = (long long)pk.G * pk.Hkv * lv.n_splits * lv.n_mt;
     items += level_items;
     if (items > (1ll << 24)) {
       delete plan;
@@ -863,6 +911,8 @@ void prefix_tc_plan_free(PrefixTcPlan *plan) {
   delete plan;
 }
 int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
+int prefix_tc_tile_tokens() { return kTileN; }
+int prefix_tc_teams() { return kTeams; }
 
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {

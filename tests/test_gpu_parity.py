@@ -144,13 +144,21 @@ def test_parts_match_oracle_on_their_token_ranges():
         for part in range(g.n_parts):
             if part < g.n_prefix_parts:
                 K, V = hp.k_prefix[0][:, h], hp.v_prefix[0][:, h]
-                lo = part * g.prefix_part_tokens
-                hi = lo + g.prefix_part_tokens
+                T, W = g.prefix_part_tokens, g.prefix_interleave
+                if W == 0:                             # part k = tokens [kT, (k+1)T)
+                    idx = np.arange(part * T, min((part + 1) * T, K.shape[0]))
+                else:                                  # parts 2s, 2s+1 = even / odd W-token tiles of [2sT, 2(s+1)T)
+                    lo = (part // 2) * 2 * T
+                    idx = np.arange(lo, min(lo + 2 * T, K.shape[0]))
+                    idx = idx[((idx - lo) // W) % 2 == part % 2]
             else:
                 K, V = hp.k_suffix[b][:, h], hp.v_suffix[b][:, h]
                 lo = (part - g.n_prefix_parts) * g.suffix_part_tokens
-                hi = lo + g.suffix_part_tokens
-            o_ref, lse_ref = orc.token_range_partial(q[b, hq], K, V, cfg.scale, lo, hi)
+                idx = np.arange(lo, min(lo + g.suffix_part_tokens, K.shape[0]))
+            if len(idx):
+                o_ref, lse_ref = orc.attend(q[b, hq], K[idx], V[idx], cfg.scale)
+            else:
+                o_ref, lse_ref = np.zeros(cfg.d), -np.inf
             if lse_ref == -np.inf:
                 assert lp[row, part] == -np.inf
             else:
