@@ -380,10 +380,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 
     Item it, nxt;
     int cur = next_item(k_begin, it);
-    if (cur < k_end && prole == 0) {
-      int round = 0;
-      while (ok && round <= kQRounds) ok = q_step(it, 0, round);
-    }
+    // (the query tile of the CTA's first item is staged by the softmax warps, which have nothing else to do yet)
     while (ok && cur < k_end && !sm.abort) {
       const int nxt_idx = next_item(cur + 1, nxt);
       int round = nxt_idx < k_end && prole == 0 ? 0 : kQRounds + 1;   // staging state of the next item's query tile
@@ -452,7 +449,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         if (!mbar_wait(sm, p, &sm.q_ready[qb], (it_n >> 1) & 1)) break;
         ++it_n;
         tc_fence_after();
-        const uint32_t q_addr = smem_u32(sm.q[qb]);
+        const uint64_t q_desc = smem_desc(smem_u32(sm.q[qb]), 16, 1024);
         const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
         // Tile t belongs to team t & 1.  Per team the order on the tensor pipe is S(t), O += P(t) V(t), S(t+2), ...:
         // P(t) lies over S(t), so S(t+2) may only follow the second product of tile t; the other team's products
@@ -464,11 +461,14 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           const int s = ktq % kKSlots;
           if (!mbar_wait(sm, p, &sm.full_k[s], (ktq / kKSlots) & 1)) return false;
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(sm.k[s]), tmem_s = tmem + (uint32_t)(t & 1) * 256u;
+          const uint32_t tmem_s = tmem + (uint32_t)(t & 1) * 256u;
+          // the descriptors of the eight k-steps differ only in the start address field (bytes >> 4, no carry out
+          // of its 14 bits: shared memory ends below 256 KB)
+          const uint64_t k_desc = smem_desc(smem_u32(sm.k[s]), 16, 1024);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            umma_ss(tmem_s, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), kIdescQK, kk > 0);
+            const uint64_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+            umma_ss(tmem_s, q_desc + off, k_desc + off, kIdescQK, kk > 0);
           }
           umma_commit(&sm.empty_k[s]);   // K(t) is free as soon as the first product has read it
           umma_commit(&sm.s_full[t & 1]);
@@ -485,13 +485,14 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if (!ok) break;
           ++team_tiles[team];
           tc_fence_after();
-          const uint32_t v_addr = smem_u32(sm.v[s]), tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
+          const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
+          const uint64_t v_desc = smem_desc(smem_u32(sm.v[s]), kPageBytes / 2, 1024);
           // one k-step per page: its 16 token rows x both 64-element halves (2 KB apart) are one 4 KB box;
           // the P columns of tokens [64 h, 64 h + 64) start at S column 64 h
 #pragma unroll
           for (int kk = 0; kk < kTileN / 16; ++kk)
-            umma_ts(tmem_o, tmem_s + (kk >> 2) * 64 + (kk & 3) * 8, smem_desc(v_addr + kk * kPageBytes, kPageBytes / 2, 1024),
-                    kIdescPV, (t >= kTeams) || (kk > 0));
+            umma_ts(tmem_o, tmem_s + (kk >> 2) * 64 + (kk & 3) * 8, v_desc + (uint64_t)((kk * kPageBytes) >> 4), kIdescPV,
+                    (t >= kTeams) || (kk > 0));
           umma_commit(&sm.empty_v[s]);
           umma_commit(&sm.pv_done[team]);
           if (t + kTeams < n_tiles) ok = issue_qk(t + kTeams);
@@ -510,6 +511,39 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
     uint32_t pair_n = 0;                       // completed meetings of this warp pair
     uint32_t team_tiles = 0;                   // tiles this team has taken so far (all items)
+    // The CTA's first item with work: its stacked query tile (128 rows x 16 chunks of 16 bytes) is staged here by
+    // all 512 softmax threads at once, four chunks each, instead of by the one producer warp in eight rounds -
+    // nothing can start before it is in place.  Later items are staged by the producer under the item before.
+    {
+      int k0 = k_begin;
+      Item qi;
+      for (; k0 < k_end; ++k0) {
+        qi = decode_item(p, lvs, __ldg(item_list + k0));
+        if (item_has_work(qi, cand_per_tile)) break;
+      }
+      if (k0 < k_end) {
+        const int tid = threadIdx.x - 64;
+        uint4 qv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int idx = i * (kTeams * kSoftmaxThreads) + tid, row = idx >> 4, c = idx & 15;
+          const int cand = qi.mt * cand_per_tile + row / g;
+          qv[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (cand < qi.n_cand) {
+            const size_t qrow = (size_t)(qi.b0 + cand) * p.Hq + (size_t)qi.h * g + (row % g);
+            qv[i] = __ldg(reinterpret_cast<const uint4 *>(q + qrow * D) + c);
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int idx = i * (kTeams * kSoftmaxThreads) + tid, row = idx >> 4, c = idx & 15;
+          *reinterpret_cast<uint4 *>(sm.q[0] + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = qv[i];
+        }
+        fence_async_proxy();
+        asm volatile("bar.sync 1, %0;\n" ::"n"(kTeams * kSoftmaxThreads) : "memory");   // the softmax warps only
+        if (warp == 2) mbar_arrive(&sm.q_ready[0]);                                       // its 32 arrivals
+      }
+    }
     // The two threads of a row meet (bounded).
     auto meet = [&]() -> bool {
       mbar_arrive(&sm.pair[team][quad]);
