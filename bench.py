@@ -336,6 +336,47 @@ def run_gpu(args):
         c3 = wl.CONFIGS["cfg3"]
         others["cfg3+root4096"] = measure("cfg3", args.steps, args.warmup, True, outer=[([0, c3.B], [4096])])
 
+    def measure_search():
+        """The search bookkeeping on 2^17 problems x 8 trajectories x 8 steps (Section 3.1: K = 8, depth 8): one pass
+        = rewards / best-so-far / value targets / labels / returns, value head, selection of tau* and of the state
+        to expand.  Algorithmic bytes per (trajectory, step): 5 read + 10 written; per trajectory 4 (length) +
+        4 (return) + 20 (logits) + 4 (expected) + 2 x 4 re-read by the two selections."""
+        b = wl.draw_search_batch(problems=1 << 17, K=8, T=8, seed=0)
+        N, T, P = b["N"], b["T"], b["P"]
+        dev = lambda a: torch.from_numpy(a).cuda()
+        sp, ok, ln, lg, go = dev(b["speedup"]), dev(b["correct"]), dev(b["len"]), dev(b["logits"]), dev(b["group_offsets"])
+        r = torch.empty((T, N), dtype=torch.uint8, device="cuda")
+        lab = torch.empty_like(r)
+        u, v = torch.empty((T, N), device="cuda"), torch.empty((T, N), device="cuda")
+        G, ev = torch.empty(N, device="cuda"), torch.empty(N, device="cuda")
+        best_t, best_s = (torch.empty(P, dtype=torch.int32, device="cuda") for _ in range(2))
+        s1, s2, s3 = wl.SEARCH_THRESHOLDS
+        stream = torch.cuda.current_stream().cuda_stream
+
+        def one():
+            mc.mc_search_returns(sp, ok, ln, N, T, s1, s2, s3, 0.95, r, u, v, lab, G, stream)
+            mc.mc_search_value_head(lg, N, None, ev, stream)
+            mc.mc_search_group_argmax(G, go, P, best_t, stream)
+            mc.mc_search_group_argmax(ev, go, P, best_s, stream)
+
+        for _ in range(3):
+            one()
+        total, reps = 0.0, 10
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            one()
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1)
+        ms = total / reps
+        nbytes = N * T * 15 + N * (4 + 4 + 20 + 4 + 8) + 2 * P * 8
+        return {"trajectories": N, "steps": T, "ms": round(ms, 5), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                "algorithmic_bytes": nbytes, "trajectory_steps_per_s": round(N * T / (ms * 1e-3), 1),
+                "l2": "arrays of one pass (220 MB) larger than L2, no flush"}
+
+    search = measure_search() if args.all_configs else None
+
     # max over ranks of the step time
     ms, e2e_ms = max_over_ranks([main["ms"], main["e2e_ms"]], device="cuda")
 
@@ -398,6 +439,7 @@ def run_gpu(args):
             "gpu_launches": int(main["launches"]),
             "clocks": main["clocks"],
             "per_config": {**{cfg.name: summary(main)}, **{k: summary(v) for k, v in others.items()}},
+            "search_bookkeeping": (dict(search, frac_of_measured_hbm=round(search["gbs"] / peak, 4)) if search else None),
         }
         print(json.dumps(line))
     if world > 1:

@@ -56,6 +56,10 @@ EXPORTS = {
     "mc_get_last_status": (c_int32, [c_void_p, c_void_p]),
     "mc_launch_count": (c_uint64, []),
     "mc_status_string": (c_char_p, [c_int32]),
+    "mc_search_returns": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_float, c_float, c_float, c_float,
+                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "mc_search_value_head": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p, c_void_p]),
+    "mc_search_group_argmax": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
 }
 
 
@@ -183,3 +187,20 @@ def mc_static_scratch_bytes() -> int:
 
 def mc_get_last_status(layout: int, stream: int = 0) -> int:
     return lib().mc_get_last_status(layout, stream)
+
+
+def mc_search_returns(speedup_pct, correct, length, N: int, T: int, s1: float, s2: float, s3: float, gamma: float,
+                      reward=None, best_so_far=None, value_target=None, label=None, traj_return=None,
+                      stream: int = 0) -> None:
+    _check(lib().mc_search_returns(_ptr(speedup_pct), _ptr(correct), _ptr(length), N, T, s1, s2, s3, gamma, _ptr(reward),
+                                   _ptr(best_so_far), _ptr(value_target), _ptr(label), _ptr(traj_return), stream),
+           "mc_search_returns")
+
+
+def mc_search_value_head(logits, N: int, prob, expected, stream: int = 0) -> None:
+    _check(lib().mc_search_value_head(_ptr(logits), N, _ptr(prob), _ptr(expected), stream), "mc_search_value_head")
+
+
+def mc_search_group_argmax(values, group_offsets, P: int, best, stream: int = 0) -> None:
+    _check(lib().mc_search_group_argmax(_ptr(values), _ptr(group_offsets), P, _ptr(best), stream),
+           "mc_search_group_argmax")

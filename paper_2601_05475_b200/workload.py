@@ -393,3 +393,25 @@ def gather_logical(pool: np.ndarray, pages_row: Sequence[int], n_tokens: int, h:
         return np.zeros((0, pool.shape[-1]), dtype=pool.dtype)
     ids = np.asarray(pages_row[:n_pages], dtype=np.int64)
     return pool[ids, h].reshape(n_pages * PAGE, pool.shape[-1])[:n_tokens]
+
+
+# ----------------------------------------------------------------------------
+# search bookkeeping: a batch of trajectories
+# ----------------------------------------------------------------------------
+SEARCH_THRESHOLDS = (120.0, 200.0, 300.0)      # s1, s2, s3 in percent (the paper leaves them open)
+
+
+def draw_search_batch(problems: int, K: int = 8, T: int = 8, seed: int = 0, ragged: bool = True):
+    """`problems` optimisation problems with K trajectories of at most T steps each (Section 3.1: K = 8, depth 8).
+    Returns a dict of step-major float32 / uint8 / int32 arrays: speed-ups in percent (log-normal around 100,
+    heavy right tail like measured kernel speed-ups), correctness (70 % pass), lengths (uniform 1..T when ragged),
+    value-head logits N(0, 2) for the last state of every trajectory, and the group offsets of the problems."""
+    N = problems * K
+    rng = np.random.Generator(np.random.Philox(np.random.SeedSequence([seed, 77, N, T])))
+    speedup = (100.0 * np.exp(rng.normal(0.1, 0.6, size=(T, N)))).astype(np.float32)
+    correct = (rng.random((T, N)) < 0.7).astype(np.uint8)
+    length = rng.integers(1, T + 1, size=N).astype(np.int32) if ragged else np.full(N, T, dtype=np.int32)
+    logits = rng.normal(0.0, 2.0, size=(N, 5)).astype(np.float32)
+    group_offsets = (np.arange(problems + 1) * K).astype(np.int32)
+    return {"speedup": speedup, "correct": correct, "len": length, "logits": logits, "group_offsets": group_offsets,
+            "N": N, "T": T, "P": problems}

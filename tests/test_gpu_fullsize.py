@@ -123,3 +123,35 @@ def test_merge_waits_for_a_prefix_pass_that_outlasts_the_suffix_pass(monkeypatch
         assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)
     assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
     dp.close()
+
+
+def test_search_bookkeeping_at_bench_size_sampled_rows():
+    """2^20 trajectories x 8 steps, the launch configuration bench.py times; 300 sampled trajectories and every
+    problem's selection are checked against the oracle."""
+    from oracle import search as sorc
+    b = wl.draw_search_batch(problems=1 << 17, K=8, T=8, seed=0)
+    N, T, P = b["N"], b["T"], b["P"]
+    dev = lambda a: torch.from_numpy(a).cuda()
+    r = torch.empty((T, N), dtype=torch.uint8, device="cuda")
+    lab = torch.empty_like(r)
+    u, v = torch.empty((T, N), device="cuda"), torch.empty((T, N), device="cuda")
+    G = torch.empty(N, device="cuda")
+    best = torch.empty(P, dtype=torch.int32, device="cuda")
+    s1, s2, s3 = wl.SEARCH_THRESHOLDS
+    mc.mc_search_returns(dev(b["speedup"]), dev(b["correct"]), dev(b["len"]), N, T, s1, s2, s3, 0.95, r, u, v, lab, G)
+    mc.mc_search_group_argmax(G, dev(b["group_offsets"]), P, best)
+    torch.cuda.synchronize()
+    r, u, v, lab, G, best = (x.cpu().numpy() for x in (r, u, v, lab, G, best))
+    rng = np.random.default_rng(0)
+    for n in [0, N - 1] + [int(x) for x in rng.integers(N, size=300)]:
+        L = int(b["len"][n])
+        sp, ok = b["speedup"][:L, n].astype(np.float64), b["correct"][:L, n] != 0
+        rr = [sorc.categorical_reward(s, c, s1, s2, s3) for s, c in zip(sp, ok)]
+        assert r[:L, n].tolist() == rr
+        np.testing.assert_allclose(u[:L, n], sorc.best_so_far(rr, 0.95), rtol=1e-5)
+        np.testing.assert_allclose(v[:L, n], sorc.value_targets(rr, 0.95), rtol=1e-5)
+        l_ref, m = sorc.future_labels(sp, ok, 0.95, s1, s2, s3)
+        clear = np.abs(m[:, None] - np.array([100.0, s1, s2, s3])[None, :]).min(axis=1) > 1e-3
+        assert (lab[:L, n][clear] == l_ref[clear]).all()
+        assert abs(G[n] - sorc.trajectory_return(rr, 0.95)) <= 1e-5
+    assert best.tolist() == sorc.group_argmax(G, b["group_offsets"]).tolist()   # fp32 values, exact decision

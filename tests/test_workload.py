@@ -101,3 +101,13 @@ def test_unique_bytes_accounting():
     assert ub["kv_prefix"] == 8192 * 4096
     assert ub["kv_suffix"] == int(sl.sum()) * 4096
     assert ub["q_o"] == 2 * 64 * 64 * 128 * 2 and ub["lse"] == 64 * 64 * 4
+
+
+def test_search_batch_is_seeded_and_shaped():
+    a, b = wl.draw_search_batch(5, K=8, T=8, seed=1), wl.draw_search_batch(5, K=8, T=8, seed=1)
+    assert a["N"] == 40 and a["speedup"].shape == (8, 40) and a["correct"].dtype == np.uint8
+    for k in ("speedup", "correct", "len", "logits", "group_offsets"):
+        np.testing.assert_array_equal(a[k], b[k])
+    assert a["len"].min() >= 1 and a["len"].max() <= 8 and a["group_offsets"].tolist() == list(range(0, 41, 8))
+    assert 0.5 < a["correct"].mean() < 0.9 and (a["speedup"] > 0).all()
+    assert not np.array_equal(a["speedup"], wl.draw_search_batch(5, K=8, T=8, seed=2)["speedup"])
