@@ -168,3 +168,38 @@ def decode_attention_cascade(q: np.ndarray,
         V = np.concatenate(vs, axis=0).astype(np.float64)
         o[b, hq], lse[b, hq] = attend(q[b, hq], K, V, scale)
     return o, lse
+
+
+def scoring_attention(q: Sequence[np.ndarray],
+                      k_prefix: Sequence[np.ndarray], v_prefix: Sequence[np.ndarray],
+                      k_seq: Sequence[np.ndarray], v_seq: Sequence[np.ndarray],
+                      group_offsets: Sequence[int], scale: float,
+                      kv_head_of: Optional[Callable[[int, int, int], int]] = None
+                      ) -> Tuple[List[np.ndarray], List[np.ndarray]]:
+    """Causal attention of whole sequences behind a shared prompt (scoring / prefill of candidates).
+
+    Sequence b (in prompt group j) has n_b tokens with keys/values k_seq[b], v_seq[b] [n_b][Hkv][d] and one query
+    per token, q[b] [n_b][Hq][d].  The query at position i attends to the group's whole prompt and to the
+    sequence's own tokens 0..i (itself included):  K = concat(Kprefix_j, Kseq_b[0 : i+1]),  o = softmax(scale q K^T) V.
+    This is `attend` applied row by row, nothing else.  Returns per sequence (o [n_b][Hq][d], lse [n_b][Hq]).
+    """
+    if kv_head_of is None:
+        kv_head_of = contiguous_kv_head
+    outs, lses = [], []
+    for b in range(len(k_seq)):
+        j = 0
+        while not (group_offsets[j] <= b < group_offsets[j + 1]):
+            j += 1
+        n_b, Hq, d = np.asarray(q[b]).shape
+        Hkv = k_seq[b].shape[1]
+        o = np.zeros((n_b, Hq, d), dtype=np.float64)
+        lse = np.zeros((n_b, Hq), dtype=np.float64)
+        for i in range(n_b):
+            for hq in range(Hq):
+                h = kv_head_of(hq, Hq, Hkv)
+                K = np.concatenate([k_prefix[j][:, h, :], k_seq[b][:i + 1, h, :]], axis=0).astype(np.float64)
+                V = np.concatenate([v_prefix[j][:, h, :], v_seq[b][:i + 1, h, :]], axis=0).astype(np.float64)
+                o[i, hq], lse[i, hq] = attend(q[b][i, hq], K, V, scale)
+        outs.append(o)
+        lses.append(lse)
+    return outs, lses

@@ -327,3 +327,65 @@ def test_cascade_equals_two_level_with_concatenated_prefixes():
         [x.tolist() for x in ks], [x.tolist() for x in vs], [0, 1, 2, 3, 4], 0.4)
     np.testing.assert_allclose(o6, np.array(bo), atol=1e-12)
     np.testing.assert_allclose(lse6, np.array(blse), atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------------------------------
+# scoring (causal attention of whole sequences behind a shared prompt)
+# ------------------------------------------------------------------------------------------------------------
+def _scoring_case(seed=0, G=2, C=2, Hq=4, Hkv=2, d=8):
+    rng = np.random.default_rng(seed)
+    go = [0, C, 2 * C][:G + 1]
+    kp = [rng.normal(size=(int(rng.integers(3, 9)), Hkv, d)) for _ in range(G)]
+    vp = [rng.normal(size=k.shape) for k in kp]
+    ks = [rng.normal(size=(int(rng.integers(1, 7)), Hkv, d)) for _ in range(G * C)]
+    vs = [rng.normal(size=k.shape) for k in ks]
+    q = [rng.normal(size=(k.shape[0], Hq, d)) for k in ks]
+    return q, kp, vp, ks, vs, go
+
+
+def test_scoring_last_position_is_the_decode_step():
+    """The query at a sequence's last position sees the prompt and the whole sequence: exactly one decode step."""
+    q, kp, vp, ks, vs, go = _scoring_case(1)
+    o, lse = orc.scoring_attention(q, kp, vp, ks, vs, go, 0.3)
+    q_last = np.stack([qb[-1] for qb in q])
+    o_ref, lse_ref = orc.decode_attention(q_last, kp, vp, ks, vs, go, 0.3)
+    for b in range(len(ks)):
+        np.testing.assert_allclose(o[b][-1], o_ref[b], atol=1e-14)
+        np.testing.assert_allclose(lse[b][-1], lse_ref[b], atol=1e-14)
+
+
+def test_scoring_is_causal_and_positions_are_decode_steps_of_truncated_sequences():
+    q, kp, vp, ks, vs, go = _scoring_case(2)
+    o, lse = orc.scoring_attention(q, kp, vp, ks, vs, go, 0.5)
+    # changing the tokens after position i changes nothing at or before i
+    ks2 = [k.copy() for k in ks]
+    vs2 = [v.copy() for v in vs]
+    for b in range(len(ks)):
+        ks2[b][2:] += 7.0
+        vs2[b][2:] -= 3.0
+    o2, lse2 = orc.scoring_attention(q, kp, vp, ks2, vs2, go, 0.5)
+    for b in range(len(ks)):
+        np.testing.assert_array_equal(o[b][:2], o2[b][:2])
+        np.testing.assert_array_equal(lse[b][:2], lse2[b][:2])
+        if ks[b].shape[0] > 2:
+            assert np.abs(o[b][2:] - o2[b][2:]).max() > 1e-3
+    # position i of sequence b = a decode step of the sequence cut after token i
+    b, i = 1, min(1, ks[1].shape[0] - 1)
+    cut_k = [k[:i + 1] if n == b else k for n, k in enumerate(ks)]
+    cut_v = [v[:i + 1] if n == b else v for n, v in enumerate(vs)]
+    qq = np.stack([q[n][min(i, q[n].shape[0] - 1)] if n == b else q[n][-1] for n in range(len(ks))])
+    o_ref, lse_ref = orc.decode_attention(qq, kp, vp, cut_k, cut_v, go, 0.5)
+    np.testing.assert_allclose(o[b][i], o_ref[b], atol=1e-14)
+    np.testing.assert_allclose(lse[b][i], lse_ref[b], atol=1e-14)
+
+
+def test_scoring_without_prompt_is_library_causal_attention():
+    """With an empty prompt and MHA heads it is plain causal self-attention: torch's float64 routine."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(3)
+    n, H, d = 6, 2, 4
+    k, v, q = (rng.normal(size=(n, H, d)) for _ in range(3))
+    o, _ = orc.scoring_attention([q], [np.zeros((0, H, d))], [np.zeros((0, H, d))], [k], [v], [0, 1], 0.7)
+    t = lambda a: torch.from_numpy(np.transpose(a, (1, 0, 2))[None].copy())       # [1][H][n][d]
+    ref = torch.nn.functional.scaled_dot_product_attention(t(q), t(k), t(v), is_causal=True, scale=0.7)
+    np.testing.assert_allclose(o[0], np.transpose(ref[0].numpy(), (1, 0, 2)), atol=1e-12)
