@@ -119,12 +119,21 @@ typedef struct {
   const int32_t *group_offsets;  /* device, [num_groups+1], increasing, last = B */
   const int32_t *pages;          /* device, [num_groups][max_pages] */
   const int32_t *len;            /* device, [num_groups], tokens */
+  const int32_t *row_limit;      /* device, [B], or NULL.  Candidate b sees only the first row_limit[b] tokens of its
+                                    group at this level (a causal mask when the candidates of a group are the query
+                                    positions of one sequence and the level holds that sequence's own tokens).  Must not
+                                    decrease from one candidate of a group to the next; values above len are the same as
+                                    len, 0 hides the level from that candidate. */
 } mc_prefix_level_t;
 
 /* mc_kv_layout_create for a cascade deeper than two levels: every candidate attends to the tokens of each outer
  * level's group it belongs to, to its base-level prefix and to its suffix (the order of concatenation does not
  * change the result).  The prefix pass covers every level, each level writes part slots of its own, the merge
- * combines them all.  n_outer <= 3.  With n_outer = 0 this is mc_kv_layout_create. */
+ * combines them all.  n_outer <= 3.  With n_outer = 0 this is mc_kv_layout_create.
+ * Scoring / prefill of whole sequences uses the same call: make every (sequence, query position) a candidate, give
+ * the base descriptor the shared prompt (its groups then hold all positions of all sequences of a prompt group) and
+ * empty suffixes, and add one outer level whose groups are the sequences, whose pages are each sequence's own
+ * tokens and whose row_limit is position + 1. */
 mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *desc, const mc_prefix_level_t *outer,
                                         int32_t n_outer, mc_kv_layout_t **out);
 

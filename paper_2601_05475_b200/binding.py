@@ -27,7 +27,7 @@ class LayoutDesc(ctypes.Structure):
 
 class PrefixLevel(ctypes.Structure):
     _fields_ = [("num_groups", c_int32), ("max_pages", c_int32), ("group_offsets", c_void_p), ("pages", c_void_p),
-                ("len", c_void_p)]
+                ("len", c_void_p), ("row_limit", c_void_p)]
 
 
 class PartGeometry(ctypes.Structure):

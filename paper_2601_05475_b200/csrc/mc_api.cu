@@ -81,6 +81,10 @@ __global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__re
 // ------------------------------------------------------------------------------------------------
 __global__ void validate_kernel(Params p, int32_t *refs, int with_suffix) {
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  if (p.row_limit)   // per-candidate limits must not decrease inside a group
+    for (int j = tid; j < p.G; j += nth)
+      for (int b = __ldg(p.group_offsets + j) + 1; b < __ldg(p.group_offsets + j + 1); ++b)
+        if (__ldg(p.row_limit + b) < __ldg(p.row_limit + b - 1)) latch(p, kDevBadPage);
   if (tid == 0) {
     if (__ldg(p.group_offsets) != 0 || __ldg(p.group_offsets + p.G) != p.B) latch(p, kDevBadPage);
     for (int j = 0; j < p.G; ++j)
@@ -239,6 +243,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   p.G = d->num_groups; p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.d = d->head_dim;
   p.g = d->num_q_heads / d->num_kv_heads;
   p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
+  p.row_limit = nullptr;
   for (int k = 0; k < n_outer; ++k) {   // an outer level is the same cache seen through another group map
     mc::Params &po = L->outer_p[k];
     po = p;
@@ -247,6 +252,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     po.prefix_pages = outer[k].pages;
     po.prefix_len = outer[k].len;
     po.max_pp = outer[k].max_pages;
+    po.row_limit = outer[k].row_limit;
   }
 
   // Part geometry.  Suffix chunks come from the table stride (the lengths live on the device and may grow).

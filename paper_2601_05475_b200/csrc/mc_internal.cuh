@@ -28,6 +28,7 @@ struct Params {
   int32_t n_prefix_parts, prefix_part_base;          // this prefix level's splits and its first part slot
   int32_t suffix_part_base;                          // first part slot of the suffix chunks
   int32_t prefix_part_tokens, suffix_part_tokens;
+  const int32_t *row_limit;                          // per candidate: tokens of this prefix level it may see (null: all)
   const int32_t *suffix_order;                       // launch order of the suffix pass's CTAs (null: as numbered)
   int32_t *status;
 };
@@ -60,6 +61,7 @@ __device__ __forceinline__ Span resolve_span(const Params &p, int b, int part) {
     int j = group_of(p, b);
     s.pages = p.prefix_pages + (size_t)j * p.max_pp;
     len = __ldg(p.prefix_len + j);
+    if (p.row_limit) len = min(len, max(__ldg(p.row_limit + b), 0));
     cap = p.max_pp * kPage;
     tokens = p.prefix_part_tokens;
     s.part = p.prefix_part_base + part;

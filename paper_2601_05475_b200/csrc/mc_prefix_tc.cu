@@ -217,6 +217,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // One level of the prefix cascade as the kernel sees it; the levels' items are numbered one level after another.
 struct TcLevel {
   const int32_t *group_offsets, *prefix_pages, *prefix_len;
+  const int32_t *row_limit;   // per candidate: tokens of this level it may see (non-decreasing within a group), or null
   int32_t max_pp, n_splits, part_base, part_tokens, n_mt, item_end;
 };
 struct TcLevels {
@@ -230,6 +231,7 @@ struct Item {
   int b0, n_cand;        // first candidate of the group, candidates in the group
   int lo, hi;            // token range of this split
   const int32_t *pages;
+  const int32_t *limits; // per-candidate token limits of the group (indexed from its first candidate), or null
 };
 
 __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs, int item) {
@@ -256,6 +258,14 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
   it.lo = sp * L.part_tokens;
   it.hi = min(len, it.lo + L.part_tokens);
   it.pages = L.prefix_pages + (size_t)it.j * L.max_pp;
+  it.limits = nullptr;
+  if (L.row_limit) {
+    // the limits do not decrease inside a group: no row of this tile sees beyond the limit of its last candidate
+    it.limits = L.row_limit + it.b0;
+    const int cand_per_tile = kTileM / p.g;
+    const int last = min((it.mt + 1) * cand_per_tile, it.n_cand) - 1;
+    if (last >= it.mt * cand_per_tile) it.hi = min(it.hi, max(__ldg(it.limits + last), 0));
+  }
   return it;
 }
 
@@ -575,6 +585,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         continue;
       }
       float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2); l: this thread's columns only
+      // tokens of the item this row may see: the split's end, or less under a per-candidate limit (causal mask)
+      const int hi_row = it.limits && row_ok ? min(it.hi, __ldg(it.limits + cand)) : it.hi;
       bool alive = true;
       for (int t = team; t < n_tiles && alive; t += kTeams, ++team_tiles) {
         const int t0 = it.lo + t * kTileN, c0 = half * 64;
@@ -584,7 +596,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         tc_fence_after();
         // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
         const uint32_t page_ok = sm.page_ok[(kt + t) & 7];
-        const bool full_tile = page_ok == 0xffu && t0 + kTileN <= it.hi;
+        const bool full_tile = page_ok == 0xffu && t0 + kTileN <= hi_row;
         // This thread's half row of S is read twice, 32 columns at a time - once for the row extremum, once for the
         // exponentials - so that no more than 32 scores are held in registers at any time.
         auto load_chunk = [&](int c, uint32_t (&sv)[32]) {
@@ -595,7 +607,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int col = c0 + c * 32 + i;
-              const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < it.hi);
+              const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < hi_row);
               if (!ok) sv[i] = masked;
             }
           }
@@ -862,6 +874,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.group_offsets = pk.group_offsets;
     lv.prefix_pages = pk.prefix_pages;
     lv.prefix_len = pk.prefix_len;
+    lv.row_limit = pk.row_limit;
     lv.max_pp = pk.max_pp;
     lv.n_splits = pk.n_prefix_parts / kTeams;
     lv.part_base = pk.prefix_part_base;
@@ -909,7 +922,8 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   if (fixed_ctas > 0) {
     grid = fixed_ctas < most ? fixed_ctas : most;
   } else {
-    const int cap = sm_count * 7 / 16 > 8 ? sm_count * 7 / 16 : 8;
+    // (with nothing to run beside - no suffix tokens, as in scoring - the pass may have every SM)
+    const int cap = target_us <= 0.0 ? sm_count : sm_count * 7 / 16 > 8 ? sm_count * 7 / 16 : 8;
     int lo = 8 < most ? 8 : most, hi = most < cap ? most : cap;   // smallest grid in [lo, hi] that meets the target (hi if none does)
     while (lo < hi) {
       const int mid = (lo + hi) / 2;

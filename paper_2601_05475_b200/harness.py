@@ -168,3 +168,56 @@ def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int
                 parts.append(pool[ids, h].reshape(n_pages * wl.PAGE, -1)[:n].float().cpu().numpy())
         out.append(np.concatenate(parts, axis=0) if parts else np.zeros((0, dp.cfg.d), dtype=np.float32))
     return out[0], out[1]
+
+
+class ScoringDeviceProblem:
+    """A scoring problem on the device: every (sequence, position) is a candidate of a cascade layout whose base
+    level is the shared prompts and whose one outer level is each sequence's own tokens under a causal row limit.
+    Memory and marshalling only."""
+
+    def __init__(self, hp: "wl.ScoringHostProblem", device="cuda"):
+        cfg = hp.cfg
+        self.cfg, self.hp = cfg, hp
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        self.k_pool, self.v_pool = storage_to_device(cfg, hp.k_pool, device), storage_to_device(cfg, hp.v_pool, device)
+        self.n_virtual = int(hp.seq_offsets[-1])
+        Bv = max(1, self.n_virtual)
+        self.t = {"go": i32(hp.group_offsets), "pp": i32(hp.prefix_pages), "pl": i32(hp.prefix_len),
+                  "sp": i32(np.full((Bv, 1), -1)), "sl": i32(np.zeros(Bv)), "so": i32(hp.seq_offsets),
+                  "qp": i32(hp.seq_pages), "ql": i32(hp.seq_len), "rl": i32(hp.row_limit)}
+        d = mc.LayoutDesc()
+        d.num_groups, d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = cfg.G, Bv, cfg.Hq, cfg.Hkv, cfg.d
+        d.page_size, d.num_pages = wl.PAGE, hp.k_pool.shape[0]
+        d.max_prefix_pages, d.max_suffix_pages = hp.prefix_pages.shape[1], 1
+        d.dtype = mc.MC_F32 if cfg.dtype == "f32" else mc.MC_BF16
+        d.k_pool, d.v_pool = self.k_pool.data_ptr(), self.v_pool.data_ptr()
+        d.group_offsets, d.prefix_pages, d.prefix_len = (self.t[k].data_ptr() for k in ("go", "pp", "pl"))
+        d.suffix_pages, d.suffix_len = self.t["sp"].data_ptr(), self.t["sl"].data_ptr()
+        lv = mc.PrefixLevel()
+        lv.num_groups, lv.max_pages = cfg.B, hp.seq_pages.shape[1]
+        lv.group_offsets, lv.pages, lv.len = (self.t[k].data_ptr() for k in ("so", "qp", "ql"))
+        lv.row_limit = self.t["rl"].data_ptr()
+        self.desc = d
+        self.layout = mc.mc_kv_layout_create_cascade(d, [lv])
+        self.geom = mc.mc_kv_layout_geometry(self.layout)
+        self.ws_bytes = mc.mc_workspace_bytes(self.layout)
+        self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=device)
+        self.ws_ptr = (self.ws.data_ptr() + 255) // 256 * 256
+        tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+        self.o = torch.empty(Bv, cfg.Hq, cfg.d, dtype=tdtype, device=device)
+        self.lse = torch.empty(Bv, cfg.Hq, dtype=torch.float32, device=device)
+
+    def score(self, q: torch.Tensor, stream: int = 0):
+        mc.mc_decode_attn(self.layout, q, self.cfg.scale, self.o, self.lse, self.ws_ptr, self.ws_bytes, stream)
+        return self.o, self.lse
+
+    def close(self):
+        if self.layout:
+            mc.mc_kv_layout_destroy(self.layout)
+            self.layout = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -415,3 +415,75 @@ def draw_search_batch(problems: int, K: int = 8, T: int = 8, seed: int = 0, ragg
     group_offsets = (np.arange(problems + 1) * K).astype(np.int32)
     return {"speedup": speedup, "correct": correct, "len": length, "logits": logits, "group_offsets": group_offsets,
             "N": N, "T": T, "P": problems}
+
+
+# ----------------------------------------------------------------------------
+# scoring: whole sequences behind a shared prompt, one query per token
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class ScoringHostProblem:
+    """G prompt groups x C sequences; every token of every sequence is a query (a "virtual candidate", numbered
+    sequence by sequence, position by position).  Logical K/V plus the paged pool image and the tables that describe
+    it to the library as a cascade: base level = the prompts, one outer level = each sequence's own tokens."""
+    cfg: Config                       # dtype / heads / d; G, C as given
+    prefix_len: np.ndarray            # int32 [G]
+    seq_len: np.ndarray               # int32 [G*C]
+    k_prefix: List[np.ndarray]
+    v_prefix: List[np.ndarray]
+    k_seq: List[np.ndarray]           # per sequence [n_b][Hkv][d] float32
+    v_seq: List[np.ndarray]
+    k_pool: np.ndarray
+    v_pool: np.ndarray
+    prefix_pages: np.ndarray          # int32 [G][max_prefix_pages]
+    seq_pages: np.ndarray             # int32 [G*C][max_seq_pages]
+    group_offsets: np.ndarray         # int32 [G+1] over virtual candidates (base level)
+    seq_offsets: np.ndarray           # int32 [G*C+1] over virtual candidates (outer level)
+    row_limit: np.ndarray             # int32 [B']: position + 1
+
+
+def make_scoring_host_problem(cfg: Config, prefix_len: Sequence[int], seq_len: Sequence[int]) -> ScoringHostProblem:
+    prefix_len = np.asarray(prefix_len, dtype=np.int32)
+    seq_len = np.asarray(seq_len, dtype=np.int32)
+    assert len(prefix_len) == cfg.G and len(seq_len) == cfg.B
+    npp = (prefix_len.astype(np.int64) + PAGE - 1) // PAGE
+    nsp = (seq_len.astype(np.int64) + PAGE - 1) // PAGE
+    num_pages = int(npp.sum() + nsp.sum()) + 1                        # one spare page so that the pool is never empty
+    ids = np.arange(num_pages, dtype=np.int32)
+    if cfg.permute_pages:
+        ids = ids[_rng(cfg.seed, _T_PERM, 500).permutation(num_pages)]
+    prefix_pages = np.full((cfg.G, max(1, int(npp.max(initial=0)))), -1, dtype=np.int32)
+    seq_pages = np.full((cfg.B, max(1, int(nsp.max(initial=0)))), -1, dtype=np.int32)
+    cur = 0
+    for j in range(cfg.G):
+        prefix_pages[j, :int(npp[j])] = ids[cur:cur + int(npp[j])]
+        cur += int(npp[j])
+    for b in range(cfg.B):
+        seq_pages[b, :int(nsp[b])] = ids[cur:cur + int(nsp[b])]
+        cur += int(nsp[b])
+    k_prefix = [_draw_k(cfg, _T_KP, 5000 + j, int(prefix_len[j])) for j in range(cfg.G)]
+    v_prefix = [_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_VP, 5000 + j), (int(prefix_len[j]), cfg.Hkv, cfg.d)))
+                for j in range(cfg.G)]
+    k_seq = [_draw_k(cfg, _T_KS, 5000 + b, int(seq_len[b])) for b in range(cfg.B)]
+    v_seq = [_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_VS, 5000 + b), (int(seq_len[b]), cfg.Hkv, cfg.d)))
+             for b in range(cfg.B)]
+    shape = (num_pages, cfg.Hkv, PAGE, cfg.d)
+    fill = storage_array(cfg, np.full(1, SENTINEL, dtype=np.float32))[0]
+    k_pool = np.full(shape, fill, dtype=fill.dtype)
+    v_pool = np.full(shape, fill, dtype=fill.dtype)
+    for j in range(cfg.G):
+        _scatter(k_pool, prefix_pages[j], k_prefix[j], cfg)
+        _scatter(v_pool, prefix_pages[j], v_prefix[j], cfg)
+    for b in range(cfg.B):
+        _scatter(k_pool, seq_pages[b], k_seq[b], cfg)
+        _scatter(v_pool, seq_pages[b], v_seq[b], cfg)
+    seq_offsets = np.concatenate([[0], np.cumsum(seq_len)]).astype(np.int32)
+    group_offsets = seq_offsets[::cfg.C].copy()
+    row_limit = np.concatenate([np.arange(1, n + 1) for n in seq_len] + [np.zeros(0)]).astype(np.int32)
+    return ScoringHostProblem(cfg, prefix_len, seq_len, k_prefix, v_prefix, k_seq, v_seq, k_pool, v_pool, prefix_pages,
+                              seq_pages, group_offsets, seq_offsets, row_limit)
+
+
+def draw_scoring_q(cfg: Config, seq_len: Sequence[int], step: int = 0) -> List[np.ndarray]:
+    """One query per token of every sequence: list of [n_b][Hq][d] float32 (storage-representable)."""
+    return [_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_Q, 9000 + 100 * step + b), (int(n), cfg.Hq, cfg.d)))
+            for b, n in enumerate(seq_len)]

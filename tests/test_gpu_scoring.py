@@ -1,0 +1,58 @@
+"""Scoring / prefill of whole sequences behind a shared prompt (every token a query, causal inside the sequence),
+run through the cascade layout with per-candidate row limits, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as orc
+from paper_2601_05475_b200 import binding as mc
+from paper_2601_05475_b200 import workload as wl
+from paper_2601_05475_b200.harness import ScoringDeviceProblem, to_device
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+CASES = {
+    # bf16, tcgen05 kernel: g = 4 -> 32 positions per 128-row tile; sequences longer than a tile, ragged prompts,
+    # a one-token and an empty sequence
+    "bf16": (wl.Config("score", "bf16", 2, 3, 16, 4, 128, ("fixed", 0), ("fixed", (0,)), permute_pages=True, seed=11),
+             [300, 77], [70, 1, 40, 0, 133, 33]),
+    # g = 8, a prompt shorter than a page and sequences that end inside a K/V tile
+    "bf16-g8": (wl.Config("score8", "bf16", 1, 2, 16, 2, 128, ("fixed", 0), ("fixed", (0,)), seed=12), [9], [150, 260]),
+    # fp32: the plain-ALU kernels honour the limits too
+    "f32": (wl.Config("scoref", "f32", 2, 2, 4, 2, 64, ("fixed", 0), ("fixed", (0,)), seed=13), [40, 17], [20, 5, 33, 18]),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_scoring_matches_oracle(name):
+    cfg, prefix_len, seq_len = CASES[name]
+    hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
+    q = wl.draw_scoring_q(cfg, seq_len)
+    dp = ScoringDeviceProblem(hp)
+    assert (dp.geom.prefix_ctas > 0) == (cfg.dtype == "bf16")      # bf16 cases run on the tcgen05 kernel
+    scratch = torch.empty(hp.k_pool.shape[0], dtype=torch.int32, device="cuda")
+    assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_OK
+    o, lse = dp.score(to_device(cfg, np.concatenate(q, axis=0)))
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    o_ref, lse_ref = orc.scoring_attention(q, hp.k_prefix, hp.v_prefix, hp.k_seq, hp.v_seq,
+                                           [0, cfg.C, 2 * cfg.C][:cfg.G + 1], cfg.scale)
+    o_ref, lse_ref = np.concatenate(o_ref, axis=0), np.concatenate(lse_ref, axis=0)
+    err = np.abs(o.float().cpu().numpy().astype(np.float64) - o_ref)
+    tol = (1e-5, 1e-5) if cfg.dtype == "f32" else (2e-2, 2e-3)
+    assert err.max() <= tol[0] and err.mean() <= tol[1], (err.max(), err.mean())
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    dp.close()
+
+
+def test_decreasing_row_limits_are_reported_by_validate():
+    cfg, prefix_len, seq_len = CASES["f32"]
+    hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
+    hp.row_limit[3] = 1          # positions 1, 2, 3, 1, ... inside the first sequence
+    dp = ScoringDeviceProblem(hp)
+    scratch = torch.empty(hp.k_pool.shape[0], dtype=torch.int32, device="cuda")
+    assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_ERR_INVALID_ARG
+    dp.close()
