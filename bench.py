@@ -373,9 +373,42 @@ def run_gpu(args):
         nbytes = N * T * 15 + N * (4 + 4 + 20 + 4 + 8) + 2 * P * 8
         return {"trajectories": N, "steps": T, "ms": round(ms, 5), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                 "algorithmic_bytes": nbytes, "trajectory_steps_per_s": round(N * T / (ms * 1e-3), 1),
-                "l2": "arrays of one pass (220 MB) larger than L2, no flush"}
+                "l2": "arrays of one pass (170 MB) larger than L2, no flush"}
 
     search = measure_search() if args.all_configs else None
+
+    def measure_scoring():
+        """Scoring of whole candidates by the value model's attention (Section 2.3): 4 problems x 8 candidates x 512
+        tokens behind a 4096-token prompt, every token a query, causal inside the candidate; Hq 32 / Hkv 8 / d 128.
+        One pass = mc_decode_attn on the cascade layout (prompt level + own-token level with row limits)."""
+        from paper_2601_05475_b200.harness import ScoringDeviceProblem, to_device
+        scfg = wl.Config("scoring", "bf16", 4, 8, 32, 8, 128, ("fixed", 4096), ("fixed", (0,)), permute_pages=True)
+        seq_len = [512] * scfg.B
+        hp = wl.make_scoring_host_problem(scfg, [4096] * scfg.G, seq_len)
+        dp = ScoringDeviceProblem(hp)
+        q = to_device(scfg, np.concatenate(wl.draw_scoring_q(scfg, seq_len), axis=0))
+        stream = torch.cuda.current_stream().cuda_stream
+        for _ in range(3):
+            dp.score(q, stream)
+        torch.cuda.synchronize()
+        reps = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            dp.score(q, stream)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        ok = mc.mc_get_last_status(dp.layout) == mc.MC_OK
+        seen = sum(n * 4096 + n * (n + 1) // 2 for n in seq_len)               # (query, key) pairs that are not masked
+        flops = 4.0 * scfg.Hq * scfg.d * seen
+        ctas, n_parts, nv = int(dp.geom.prefix_ctas), int(dp.geom.n_parts), dp.n_virtual
+        dp.close()
+        return {"sequences": scfg.B, "tokens_per_sequence": 512, "prompt_tokens": 4096, "queries": nv, "ms": round(ms, 4),
+                "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "flops": flops, "prefix_ctas": ctas, "n_parts": n_parts,
+                "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
+
+    scoring = measure_scoring() if args.all_configs else None
 
     # max over ranks of the step time
     ms, e2e_ms = max_over_ranks([main["ms"], main["e2e_ms"]], device="cuda")
@@ -440,6 +473,8 @@ def run_gpu(args):
             "clocks": main["clocks"],
             "per_config": {**{cfg.name: summary(main)}, **{k: summary(v) for k, v in others.items()}},
             "search_bookkeeping": (dict(search, frac_of_measured_hbm=round(search["gbs"] / peak, 4)) if search else None),
+            "scoring_attention": (dict(scoring, bound="tensor", frac_of_measured_bf16=(
+                round(scoring["tflops"] / peaks["bf16_tflops"], 4) if peaks.get("bf16_tflops") else None)) if scoring else None),
         }
         print(json.dumps(line))
     if world > 1:

@@ -155,3 +155,34 @@ def test_search_bookkeeping_at_bench_size_sampled_rows():
         assert (lab[:L, n][clear] == l_ref[clear]).all()
         assert abs(G[n] - sorc.trajectory_return(rr, 0.95)) <= 1e-5
     assert best.tolist() == sorc.group_argmax(G, b["group_offsets"]).tolist()   # fp32 values, exact decision
+
+
+def test_scoring_at_bench_size_sampled_rows():
+    """32 sequences x 512 tokens behind 4096-token prompts (the configuration bench.py times): 48 sampled
+    (sequence, position, head) rows, among them first and last positions, against the oracle's row-by-row definition."""
+    from paper_2601_05475_b200.harness import ScoringDeviceProblem, to_device
+    scfg = wl.Config("scoring", "bf16", 4, 8, 32, 8, 128, ("fixed", 4096), ("fixed", (0,)), permute_pages=True)
+    seq_len = [512] * scfg.B
+    hp = wl.make_scoring_host_problem(scfg, [4096] * scfg.G, seq_len)
+    q = wl.draw_scoring_q(scfg, seq_len)
+    dp = ScoringDeviceProblem(hp)
+    assert dp.geom.prefix_ctas > 0
+    o, lse = dp.score(to_device(scfg, np.concatenate(q, axis=0)))
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    o, lse = o.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(0)
+    rows = [(0, 0, 0), (31, 511, 31), (5, 127, 3), (5, 128, 3)] + \
+           [(int(rng.integers(32)), int(rng.integers(512)), int(rng.integers(32))) for _ in range(44)]
+    errs = []
+    for (b, i, hq) in rows:
+        j, h = b // scfg.C, hq // scfg.g
+        K = np.concatenate([hp.k_prefix[j][:, h], hp.k_seq[b][:i + 1, h]], axis=0)
+        V = np.concatenate([hp.v_prefix[j][:, h], hp.v_seq[b][:i + 1, h]], axis=0)
+        o_ref, lse_ref = orc.attend(q[b][i, hq], K, V, scfg.scale)
+        v = int(hp.seq_offsets[b]) + i
+        errs.append(np.abs(o[v, hq] - o_ref))
+        assert abs(lse[v, hq] - lse_ref) <= 1e-3
+    errs = np.concatenate(errs)
+    assert errs.max() <= 2e-2 and errs.mean() <= 2e-3
+    dp.close()
