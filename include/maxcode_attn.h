@@ -33,8 +33,7 @@
  * that page and latch MC_ERR_INVALID_ARG in the device status word (see mc_get_last_status).
  *
  * Partial results ("parts").  rows = B*Hq, row = b*Hq + hq.  Each row has n_parts slots:
- *   parts [0, n_prefix_parts)            prefix parts of prefix_part_tokens tokens each (which tokens: see
- *                                        mc_part_geometry_t.prefix_interleave)
+ *   parts [0, n_prefix_parts)            prefix splits of prefix_part_tokens tokens each
  *   parts [n_prefix_parts, n_parts)      suffix chunks of suffix_part_tokens tokens each
  *   o_part   float [rows][n_parts][d]    normalised partial output of that token range
  *   lse_part float [rows][n_parts]       its log-sum-exp; -inf marks an empty part (o_part undefined)
@@ -96,10 +95,6 @@ typedef struct {
   int32_t suffix_part_tokens;    /* tokens per suffix chunk (multiple of 16) */
   int32_t head_dim;
   int32_t prefix_ctas;           /* persistent CTAs of the tensor-core prefix pass; 0: that kernel is not used */
-  int32_t prefix_interleave;     /* 0: prefix part k of a level covers its tokens [k*T, (k+1)*T), T = prefix_part_tokens.
-                                    W > 0 (the tensor-core prefix pass, for every scale but 0): parts 2s and 2s+1 share the
-                                    tokens [2sT, 2(s+1)T); counting that range in tiles of W tokens, part 2s holds the tiles
-                                    with an even index and part 2s+1 those with an odd index. */
 } mc_part_geometry_t;
 
 /* Builds the layout object (step 1 of the path, the paged-KV layout): validates the descriptor, fixes

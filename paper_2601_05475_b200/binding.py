@@ -32,7 +32,7 @@ class PrefixLevel(ctypes.Structure):
 
 class PartGeometry(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in ("rows", "n_parts", "n_prefix_parts", "prefix_part_tokens",
-                                       "suffix_part_tokens", "head_dim", "prefix_ctas", "prefix_interleave")]
+                                       "suffix_part_tokens", "head_dim", "prefix_ctas")]
 
 
 EXPORTS = {

@@ -305,16 +305,11 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     nsp[k] = mc::choose_splits(pk, work[k], budget_us);
     const int max_p = pk.max_pp * mc::kPage;
     int tp = ((max_p + nsp[k] - 1) / nsp[k] + 127) / 128 * 128;
-    // The tensor-core prefix pass deals the 128-token tiles of a split alternately to two streams, each with a
-    // part slot of its own: a split is then a pair of slots, and a slot stands for half a split's tokens.
-    const bool two_streams = want_tc && mc::prefix_tc_shape_supported(pk, d->dtype);
-    const int streams = two_streams ? mc::prefix_tc_teams() : 1;
-    tp /= streams;
     if (mc::env_int("MC_PREFIX_PART_TOKENS", 0) > 0)
       tp = mc::env_int("MC_PREFIX_PART_TOKENS", tp) / mc::kPage * mc::kPage;
     if (tp < mc::kPage) tp = mc::kPage;
     pk.prefix_part_tokens = tp;
-    pk.n_prefix_parts = (max_p + tp * streams - 1) / (tp * streams) * streams;
+    pk.n_prefix_parts = (max_p + tp - 1) / tp;
     pk.prefix_part_base = part_base;
     part_base += pk.n_prefix_parts;
   }
@@ -447,7 +442,6 @@ mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry
   g->suffix_part_tokens = L->p.suffix_part_tokens;
   g->head_dim = L->p.d;
   g->prefix_ctas = mc::prefix_tc_grid(L->tc_plan);
-  g->prefix_interleave = L->tc_plan ? mc::prefix_tc_tile_tokens() : 0;
   return MC_OK;
 }
 

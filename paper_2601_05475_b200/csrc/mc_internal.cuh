@@ -106,8 +106,6 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
                              double target_us, double tile_us, double item_us);
 void prefix_tc_plan_free(PrefixTcPlan *plan);
 int prefix_tc_grid(const PrefixTcPlan *plan);
-int prefix_tc_tile_tokens();   // tokens per K/V tile
-int prefix_tc_teams();         // tile streams (= part slots) per prefix split
 bool prefix_tc_shape_supported(const Params &p, int dtype);   // everything but the part geometry
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream);

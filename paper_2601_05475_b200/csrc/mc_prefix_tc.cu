@@ -12,7 +12,7 @@
 // Work item = (group, kv head, prefix split, 128-row tile); every CTA has a list of items.  Inside an item the
 // 128-token K/V tiles are dealt alternately to two independent streams ("teams"): each team has its own S and O
 // accumulators in TMEM (S0 O0 S1 O1 = 512 columns), its own 256 softmax threads and its own running maximum and
-// row sum, and writes a part slot of its own - the merge combines the two like any two parts.  While one team
+// row sum; the two are merged in the item's epilogue.  While one team
 // computes the exponentials of its tile, the tensor pipe runs the other team's products.
 // Warp roles: warp 0 and warps 18, 19 issue the TMA copies (warp 0 also stages the next item's query tile), warp 1
 // lane 0 issues the MMAs (warp 1 owns the TMEM allocation), warps 2-9 are team 0 and warps 10-17 team 1 (two
@@ -53,6 +53,7 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
   uint64_t q_ready[2], q_free[2], s_full[kTeams], p_full[kTeams], pv_done[kTeams];
   uint64_t pair[kTeams][4];           // the two warps of a team that share a TMEM lane quadrant meet here
+  uint64_t both;                      // the two teams meet here around an item's epilogue
   float xch[kTeams][2][kTileM];       // [team][column half][row]: row extremum / row sum exchange
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
@@ -254,7 +255,7 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
     latch(p, kDevBadPage);
     len = len < 0 ? 0 : cap;
   }
-  it.part = L.part_base + kTeams * sp;   // team T writes slot it.part + T
+  it.part = L.part_base + sp;
   it.lo = sp * L.part_tokens;
   it.hi = min(len, it.lo + L.part_tokens);
   it.pages = L.prefix_pages + (size_t)it.j * L.max_pp;
@@ -306,6 +307,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       mbar_init(&sm.q_ready[b], 32);
       mbar_init(&sm.q_free[b], 1);
     }
+    mbar_init(&sm.both, kTeams * kSoftmaxThreads);
     for (int t = 0; t < kTeams; ++t) {
       mbar_init(&sm.s_full[t], 1);
       mbar_init(&sm.p_full[t], kSoftmaxThreads);
@@ -521,6 +523,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
     uint32_t pair_n = 0;                       // completed meetings of this warp pair
     uint32_t team_tiles = 0;                   // tiles this team has taken so far (all items)
+    uint32_t other_tiles = 0;                  // ... and the other team
+    uint32_t both_n = 0;                       // completed meetings of the two teams
     // The CTA's first item with work: its stacked query tile (128 rows x 16 chunks of 16 bytes) is staged here by
     // all 512 softmax threads at once, four chunks each, instead of by the one producer warp in eight rounds -
     // nothing can start before it is in place.  Later items are staged by the producer under the item before.
@@ -577,13 +581,13 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
-      const size_t slot = qrow * p.n_parts + it.part + team;
+      const size_t slot = qrow * p.n_parts + it.part;
       const int n_tiles = it.lo < it.hi ? (it.hi - it.lo + kTileN - 1) / kTileN : 0;
-      if (team >= n_tiles) {   // no tokens in this split, or a single tile: it is the other team's
-        if (row_ok && half == 0) lse_part[slot] = -INFINITY;
-        kt += n_tiles;
+      if (n_tiles == 0) {   // no tokens in this split
+        if (row_ok && half == 0 && team == 0) lse_part[slot] = -INFINITY;
         continue;
       }
+      const int my_tiles = (n_tiles - team + 1) / kTeams, ot_tiles = n_tiles - my_tiles;   // tiles team, team + 2, ...
       float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2); l: this thread's columns only
       // tokens of the item this row may see: the split's end, or less under a per-candidate limit (causal mask)
       const int hi_row = it.limits && row_ok ? min(it.hi, __ldg(it.limits + cand)) : it.hi;
@@ -693,28 +697,65 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         mbar_arrive(&sm.p_full[team]);
       }
       kt += n_tiles;
+      other_tiles += ot_tiles;
       if (!alive) break;
-      // epilogue: O / l -> o_part, lse (each thread writes its 64 columns; the row sum is the two halves')
+      // ---- epilogue: the two streams of the item are merged here, so the item writes one part.
+      // Row sum of this team (the two halves'), then both teams publish (m, l) of every row and meet.
       float l_other = 0.f;
       alive = meet() && exchange(l, l_other) && meet();
       if (!alive) break;
       const float l_row = l + l_other;
-      alive = mbar_wait(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
+      if (half == 0) {   // the pair is past its last read of the exchange slots (second meeting above)
+        sm.xch[team][0][r] = m;
+        sm.xch[team][1][r] = l_row;
+      }
+      auto teams_meet = [&]() -> bool {
+        mbar_arrive(&sm.both);
+        bool w = mbar_wait(sm, p, &sm.both, both_n & 1);
+        ++both_n;
+        return __all_sync(0xffffffffu, w);
+      };
+      alive = teams_meet();
+      if (!alive) break;
+      const float m_o = sm.xch[team ^ 1][0][r], l_o = sm.xch[team ^ 1][1][r];
+      // weights of the two streams in log2 units: exp2(m_T - max) l_T; a stream without tiles or without an
+      // unmasked token in this row has weight 0 and its accumulator is not read
+      const bool have_me = my_tiles > 0, have_ot = ot_tiles > 0;
+      const float m_all = fmaxf(have_me && l_row > 0.f ? m : -INFINITY, have_ot && l_o > 0.f ? m_o : -INFINITY);
+      const float a_me = have_me && l_row > 0.f ? fast_exp2(m - m_all) : 0.f;
+      const float a_ot = have_ot && l_o > 0.f ? fast_exp2(m_o - m_all) : 0.f;
+      const float l_all = a_me * l_row + a_ot * l_o;
+      if (have_me) alive = mbar_wait(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
+      if (have_ot) alive = alive && mbar_wait(sm, p, &sm.pv_done[team ^ 1], (other_tiles - 1) & 1);
       if (!__all_sync(0xffffffffu, alive)) break;
       tc_fence_after();
-      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-      // Each thread holds 64 columns of ONE row; a store instruction issued like that touches 32 rows.  The
-      // 32x32 blocks are transposed across the warp first (lane j then holds column j of all 32 rows), so
-      // that every store instruction writes 128 contiguous bytes of one row.
-      const unsigned long long my_off = (unsigned long long)slot * D + half * 64;
-      const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_row > 0.f);
-#pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
+      const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+      // Each of the row's four threads takes 32 of the 128 output columns: [64 half + 32 team, +32).  A thread holds
+      // 32 columns of ONE row; a store instruction issued like that touches 32 rows, so the 32x32 block is
+      // transposed across the warp first (lane j then holds column j of all 32 rows) and every store instruction
+      // writes 128 contiguous bytes of one row.
+      const int col0 = half * 64 + team * 32;
+      const unsigned long long my_off = (unsigned long long)slot * D + col0;
+      const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_all > 0.f);
+      {
         uint32_t v[32];
-        tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, v);
-        tmem_wait_ld();
+        const float w_me = a_me * inv, w_ot = a_ot * inv;
+        if (have_me) {
+          tmem_ld32(tmem_o + lane_addr + col0, v);
+          tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * inv);
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * w_me);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0u;
+        }
+        if (have_ot) {
+          uint32_t w[32];
+          tmem_ld32(tmem + (uint32_t)(team ^ 1) * 256u + kTileN + lane_addr + col0, w);   // the other team's accumulator
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaf(__uint_as_float(w[i]), w_ot, __uint_as_float(v[i])));
+        }
 #pragma unroll
         for (int s = 16; s >= 1; s >>= 1) {
           const bool up = (lane & s) != 0;
@@ -726,15 +767,18 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
             if (up) v[i] = got; else v[i | s] = got;
           }
         }
-        // v[i] now is element (row i of this warp's 32 rows, column c*32 + lane)
+        // v[i] now is element (row i of this warp's 32 rows, column col0 + lane)
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const unsigned long long off = __shfl_sync(0xffffffffu, my_off, i);
-          if ((store_mask >> i) & 1u) o_part[off + c * 32 + lane] = __uint_as_float(v[i]);
+          if ((store_mask >> i) & 1u) o_part[off + lane] = __uint_as_float(v[i]);
         }
       }
-      if (row_ok && half == 0) lse_part[slot] = l_row > 0.f ? (m + log2f(l_row)) * kLn2 : -INFINITY;
+      if (row_ok && half == 0 && team == 0) lse_part[slot] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
       tc_fence_before();
+      // nobody goes on (to overwrite an accumulator or an exchange slot) before everybody has read both
+      alive = teams_meet();
+      if (!alive) break;
     }
   }
 
@@ -820,9 +864,7 @@ bool prefix_tc_shape_supported(const Params &p, int dtype) {
 }
 
 bool prefix_tc_supported(const Params &p, int dtype) {
-  // a split is a pair of part slots, one per team, and a whole number of 128-token tiles
-  return prefix_tc_shape_supported(p, dtype) && p.n_prefix_parts % kTeams == 0 &&
-         (p.prefix_part_tokens * kTeams) % kTileN == 0;
+  return prefix_tc_shape_supported(p, dtype) && p.prefix_part_tokens % kTileN == 0;
 }
 
 namespace {
@@ -876,9 +918,9 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.prefix_len = pk.prefix_len;
     lv.row_limit = pk.row_limit;
     lv.max_pp = pk.max_pp;
-    lv.n_splits = pk.n_prefix_parts / kTeams;
+    lv.n_splits = pk.n_prefix_parts;
     lv.part_base = pk.prefix_part_base;
-    lv.part_tokens = pk.prefix_part_tokens * kTeams;
+    lv.part_tokens = pk.prefix_part_tokens;
     lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
     const long long level_items = (long long)pk.G * pk.Hkv * lv.n_splits * lv.n_mt;
     items += level_items;
@@ -959,8 +1001,7 @@ void prefix_tc_plan_free(PrefixTcPlan *plan) {
   delete plan;
 }
 int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
-int prefix_tc_tile_tokens() { return kTileN; }
-int prefix_tc_teams() { return kTeams; }
+
 
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
                              float *lse_part, cudaStream_t stream) {

@@ -144,13 +144,8 @@ def test_parts_match_oracle_on_their_token_ranges():
         for part in range(g.n_parts):
             if part < g.n_prefix_parts:
                 K, V = hp.k_prefix[0][:, h], hp.v_prefix[0][:, h]
-                T, W = g.prefix_part_tokens, g.prefix_interleave
-                if W == 0:                             # part k = tokens [kT, (k+1)T)
-                    idx = np.arange(part * T, min((part + 1) * T, K.shape[0]))
-                else:                                  # parts 2s, 2s+1 = even / odd W-token tiles of [2sT, 2(s+1)T)
-                    lo = (part // 2) * 2 * T
-                    idx = np.arange(lo, min(lo + 2 * T, K.shape[0]))
-                    idx = idx[((idx - lo) // W) % 2 == part % 2]
+                T = g.prefix_part_tokens              # part k = tokens [kT, (k+1)T)
+                idx = np.arange(part * T, min((part + 1) * T, K.shape[0]))
             else:
                 K, V = hp.k_suffix[b][:, h], hp.v_suffix[b][:, h]
                 lo = (part - g.n_prefix_parts) * g.suffix_part_tokens
@@ -291,6 +286,31 @@ def test_warp_level_suffix_kernel_matches_oracle(monkeypatch, name):
     q = wl.draw_q(cfg, 0)
     dp, o, lse = run_decode(hp, q)
     check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
+@pytest.mark.parametrize("env", [{"MC_PDL": "0"}, {"MC_PREFIX_TC": "0"}, {"MC_SUFFIX_ORDER": "0"},
+                                 {"MC_PREFIX_TC": "0", "MC_SUFFIX_TMA": "0"}, {"MC_PREFIX_CTAS": "3"}])
+@pytest.mark.parametrize("name", ["cfg2s", "cfg3sp"])
+def test_alternative_schedules_match_oracle(monkeypatch, env, name):
+    """The same step on the library's other schedules: two streams instead of a programmatic dependent launch, the
+    warp-level prefix pass, suffix items in plain order, both warp-level passes, a prefix grid of three CTAs (several
+    items per CTA).  A decode step and an append step each."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    cfg = SMALL[name]
+    hp = wl.make_host_problem(cfg, headroom_tokens=4)
+    q = wl.draw_q(cfg, 0)
+    dp, o, lse = run_decode(hp, q)
+    check_close(cfg, o, lse, *oracle_full(hp, q))
+    k_new, v_new = wl.draw_append(cfg, 1)
+    q = wl.draw_q(cfg, 1)
+    mc.mc_decode_step(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new), to_device(cfg, q), cfg.scale, dp.o,
+                      dp.lse, dp.ws_ptr, dp.ws_bytes)
+    torch.cuda.synchronize()
+    hp.append(k_new, v_new)
+    check_close(cfg, dp.o, dp.lse, *oracle_full(hp, q))
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
     dp.close()
 
 
