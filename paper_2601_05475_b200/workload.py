@@ -441,7 +441,11 @@ class ScoringHostProblem:
     row_limit: np.ndarray             # int32 [B']: position + 1
 
 
-def make_scoring_host_problem(cfg: Config, prefix_len: Sequence[int], seq_len: Sequence[int]) -> ScoringHostProblem:
+def make_scoring_host_problem(cfg: Config, prefix_len: Sequence[int], seq_len: Sequence[int],
+                              last_queries: Optional[int] = None) -> ScoringHostProblem:
+    """`last_queries` = None: every token of a sequence is a query (scoring).  `last_queries` = n: only the last n
+    tokens of every sequence are queries (a decode step that verifies n speculated tokens at once); the virtual
+    candidates of sequence b are then its positions max(0, n_b - n) .. n_b - 1."""
     prefix_len = np.asarray(prefix_len, dtype=np.int32)
     seq_len = np.asarray(seq_len, dtype=np.int32)
     assert len(prefix_len) == cfg.G and len(seq_len) == cfg.B
@@ -476,14 +480,17 @@ def make_scoring_host_problem(cfg: Config, prefix_len: Sequence[int], seq_len: S
     for b in range(cfg.B):
         _scatter(k_pool, seq_pages[b], k_seq[b], cfg)
         _scatter(v_pool, seq_pages[b], v_seq[b], cfg)
-    seq_offsets = np.concatenate([[0], np.cumsum(seq_len)]).astype(np.int32)
+    n_query = seq_len if last_queries is None else np.minimum(seq_len, last_queries)
+    seq_offsets = np.concatenate([[0], np.cumsum(n_query)]).astype(np.int32)
     group_offsets = seq_offsets[::cfg.C].copy()
-    row_limit = np.concatenate([np.arange(1, n + 1) for n in seq_len] + [np.zeros(0)]).astype(np.int32)
+    row_limit = np.concatenate([np.arange(n - nq + 1, n + 1) for n, nq in zip(seq_len, n_query)] +
+                               [np.zeros(0)]).astype(np.int32)
     return ScoringHostProblem(cfg, prefix_len, seq_len, k_prefix, v_prefix, k_seq, v_seq, k_pool, v_pool, prefix_pages,
                               seq_pages, group_offsets, seq_offsets, row_limit)
 
 
 def draw_scoring_q(cfg: Config, seq_len: Sequence[int], step: int = 0) -> List[np.ndarray]:
-    """One query per token of every sequence: list of [n_b][Hq][d] float32 (storage-representable)."""
+    """One query per token of every sequence: list of [n_b][Hq][d] float32 (storage-representable).  (When only the
+    last n tokens are queries, take the last n rows of each.)"""
     return [_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_Q, 9000 + 100 * step + b), (int(n), cfg.Hq, cfg.d)))
             for b, n in enumerate(seq_len)]

@@ -48,6 +48,28 @@ def test_scoring_matches_oracle(name):
     dp.close()
 
 
+@pytest.mark.parametrize("n_spec", [1, 4])
+def test_multi_token_decode_step(n_spec):
+    """A decode step that checks several speculated tokens per candidate at once: the last n_spec tokens of every
+    sequence are queries, each seeing the prompt and its sequence up to itself (n_spec = 1 is the ordinary step)."""
+    cfg = wl.Config("spec", "bf16", 2, 4, 16, 4, 128, ("fixed", 0), ("fixed", (0,)), permute_pages=True, seed=21)
+    prefix_len, seq_len = [200, 50], [90, 3, 40, 17, 64, 1, 130, 33]
+    hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len, last_queries=n_spec)
+    q_all = wl.draw_scoring_q(cfg, seq_len)
+    q = [x[-n_spec:] for x in q_all]
+    dp = ScoringDeviceProblem(hp)
+    o, lse = dp.score(to_device(cfg, np.concatenate(q, axis=0)))
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    o_ref, lse_ref = orc.scoring_attention(q_all, hp.k_prefix, hp.v_prefix, hp.k_seq, hp.v_seq, [0, 4, 8], cfg.scale)
+    o_ref = np.concatenate([x[-n_spec:] for x in o_ref], axis=0)
+    lse_ref = np.concatenate([x[-n_spec:] for x in lse_ref], axis=0)
+    err = np.abs(o.float().cpu().numpy().astype(np.float64) - o_ref)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    dp.close()
+
+
 def test_decreasing_row_limits_are_reported_by_validate():
     cfg, prefix_len, seq_len = CASES["f32"]
     hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
