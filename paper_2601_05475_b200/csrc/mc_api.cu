@@ -142,7 +142,7 @@ mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_p
 
 // Splits and persistent-CTA count of one prefix level (see the comment in mc_kv_layout_create_cascade).
 struct LevelWork { long long pairs; double tiles; int max_group; };
-constexpr double kTileUs = 1.6, kItemUs = 6.0;   // measured: per 128x128 tile; per item (prologue + epilogue)
+constexpr double kTileUs = 1.3, kItemUs = 8.0;   // measured: per 128x128 tile; per item (prologue + epilogue)
 
 // (group, kv head, 128-row tile) pairs and 128-token tiles of one level, from the lengths as they are now.
 LevelWork level_work(const Params &p) {
