@@ -276,19 +276,22 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     }
     (void)cudaGetLastError();
   }
-  int ts = mc::pow2_floor(max_s / 16 > 512 ? max_s / 16 : 512);   // about 16 chunks per row, 512..4096 tokens
+  // A chunk costs its warp about 4 us of start-up and wind-down besides its pages (measured), so chunks are long:
+  // about 4 per row, 512..4096 tokens (cfg3: 8.7 % faster with 2048-token chunks than with 512)
+  int ts = mc::pow2_floor(max_s / 4 > 512 ? max_s / 4 : 512);
   if (ts > 4096) ts = 4096;
   if (suffix_tokens_now >= 0.0) {
-    // A small problem cannot keep every warp slot busy with chunks of that size: shorter chunks, about the
-    // tokens one of the device's warp slots (8 per SM) gets, in steps of 128 tokens, down to 4 pages a chunk.
+    // A small problem cannot keep every warp slot (6 per SM) busy with chunks of that size: shorter chunks, so that
+    // a slot gets about 1.6 full chunks and the partial chunks of the rows fill the end of the launch - to the nearest
+    // 128 tokens, down to 4 pages a chunk.
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       sms = 148;
     (void)cudaGetLastError();
-    const double per_warp = suffix_tokens_now * p.Hkv / (8.0 * sms);
-    int tpar = per_warp < 128.0 ? mc::pow2_floor(per_warp < 64.0 ? 64 : (int)per_warp)
-                                : per_warp > 4096.0 ? 4096 : (int)per_warp / 128 * 128;
+    const double per_chunk = suffix_tokens_now * p.Hkv / (6.0 * sms) / 1.6;
+    int tpar = per_chunk < 128.0 ? mc::pow2_floor(per_chunk < 64.0 ? 64 : (int)per_chunk)
+                                 : per_chunk > 4096.0 ? 4096 : ((int)per_chunk + 64) / 128 * 128;
     if (tpar < ts) ts = tpar;
   }
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
