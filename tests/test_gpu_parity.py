@@ -124,6 +124,48 @@ def test_appends_that_open_new_chunks(monkeypatch):
     dp.close()
 
 
+def test_many_consecutive_steps_stay_correct():
+    """240 decode steps in a row on one layout (appends cross page, tile and chunk boundaries many times; every
+    barrier of the persistent prefix kernel goes through hundreds of phases); the oracle checks a step now and then
+    and the status word stays clean."""
+    cfg = wl.scaled_down(wl.CONFIGS["cfg2"], "soak", C=16, prefix=("fixed", 777), suffix=("uniform", 0, 300),
+                         append_steps=240)
+    hp = wl.make_host_problem(cfg, headroom_tokens=250)
+    dp = DeviceProblem.from_host(hp)
+    assert dp.geom.prefix_ctas > 0
+    for step in range(1, 241):
+        k_new, v_new = wl.draw_append(cfg, step)
+        q = wl.draw_q(cfg, step)
+        mc.mc_decode_step(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new), to_device(cfg, q), cfg.scale,
+                          dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes)
+        hp.append(k_new, v_new)
+        if step % 60 == 0 or step in (1, 17, 239):
+            torch.cuda.synchronize()
+            rows = [(b, hq) for b in (0, 7, 15) for hq in (0, 31, 63)]
+            o_ref, lse_ref = oracle_full(hp, q, rows=rows)
+            check_close(cfg, dp.o, dp.lse, o_ref, lse_ref, rows=rows)
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    assert torch.isfinite(dp.o.float()).all()
+    dp.close()
+
+
+def test_layouts_can_be_created_and_destroyed_repeatedly():
+    cfg = SMALL["cfg3s"]
+    hp = wl.make_host_problem(cfg)
+    q = to_device(cfg, wl.draw_q(cfg, 0))
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(40):
+        dp = DeviceProblem.from_host(hp)
+        dp.decode(q)
+        torch.cuda.synchronize()
+        dp.close()
+        del dp
+    torch.cuda.empty_cache()
+    assert free0 - torch.cuda.mem_get_info()[0] < (64 << 20)      # nothing of the 40 handles is left behind
+
+
 def test_parts_match_oracle_on_their_token_ranges():
     cfg = SMALL["cfg2s"]
     hp = wl.make_host_problem(cfg)
