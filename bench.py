@@ -326,16 +326,6 @@ def run_gpu(args):
         torch.cuda.empty_cache()
         return res
 
-    main = measure(args.workload, args.steps, args.warmup, True)
-    others = {}
-    if args.all_configs:
-        for name in ("cfg2", "cfg3", "cfg4"):
-            if name != args.workload:
-                others[name] = measure(name, args.steps, args.warmup, True)
-        # a cascade deeper than two levels: configuration 3 behind a 4096-token prompt shared by all 256 candidates
-        c3 = wl.CONFIGS["cfg3"]
-        others["cfg3+root4096"] = measure("cfg3", args.steps, args.warmup, True, outer=[([0, c3.B], [4096])])
-
     def measure_search():
         """The search bookkeeping on 2^17 problems x 8 trajectories x 8 steps (Section 3.1: K = 8, depth 8): one pass
         = rewards / best-so-far / value targets / labels / returns, value head, selection of tau* and of the state
@@ -375,8 +365,6 @@ def run_gpu(args):
                 "algorithmic_bytes": nbytes, "trajectory_steps_per_s": round(N * T / (ms * 1e-3), 1),
                 "l2": "arrays of one pass (170 MB) larger than L2, no flush"}
 
-    search = measure_search() if args.all_configs else None
-
     def measure_scoring():
         """Scoring of whole candidates by the value model's attention (Section 2.3): 4 problems x 8 candidates x 512
         tokens behind a 4096-token prompt, every token a query, causal inside the candidate; Hq 32 / Hkv 8 / d 128.
@@ -407,6 +395,23 @@ def run_gpu(args):
         return {"sequences": scfg.B, "tokens_per_sequence": 512, "prompt_tokens": 4096, "queries": nv, "ms": round(ms, 4),
                 "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "flops": flops, "prefix_ctas": ctas, "n_parts": n_parts,
                 "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
+
+    if args.scoring_only:      # profiling aid: only the scoring pass, one small JSON line
+        if rank == 0:
+            print(json.dumps({"scoring_attention": measure_scoring()}))
+        return 0
+
+    main = measure(args.workload, args.steps, args.warmup, True)
+    others = {}
+    if args.all_configs:
+        for name in ("cfg2", "cfg3", "cfg4"):
+            if name != args.workload:
+                others[name] = measure(name, args.steps, args.warmup, True)
+        # a cascade deeper than two levels: configuration 3 behind a 4096-token prompt shared by all 256 candidates
+        c3 = wl.CONFIGS["cfg3"]
+        others["cfg3+root4096"] = measure("cfg3", args.steps, args.warmup, True, outer=[([0, c3.B], [4096])])
+
+    search = measure_search() if args.all_configs else None
 
     scoring = measure_scoring() if args.all_configs else None
 
@@ -491,6 +496,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false",
                     help="skip the CPU-oracle leg (profiling runs only; the default run reports it)")
+    ap.add_argument("--scoring-only", action="store_true", help="run only the scoring pass (profiling aid)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
                     help="time only --workload (default: also cfg2/cfg3/cfg4 summaries under per_config)")
     args = ap.parse_args()
