@@ -4,19 +4,20 @@
 // stacked into dense 128-row tiles (row = candidate * g + head-in-group), so the group's prefix K/V is
 // streamed once for the whole group instead of once per candidate:
 //     S = Q_s K^T          128 x 128 tile, tcgen05.mma, operands in shared memory, accumulator in TMEM
-//     P = exp2(S*c - m)    two threads per row read the row of S from TMEM and write bf16 P over it
+//     P = exp2(S*c - m)    one thread per row reads the row of S from TMEM and writes bf16 P over it
 //     O += P V             tcgen05.mma, P from TMEM, V in its natural [token][d] layout (MN-major B operand)
 // K/V pages reach shared memory by TMA through tensor maps laid over the paged pools (the page id is a TMA
 // coordinate): V as one 4 KB box per page, K as two 2 KB boxes per page (one per 64-element d half).
 //
 // Work item = (group, kv head, prefix split, 128-row tile); every CTA has a list of items.  Inside an item the
 // 128-token K/V tiles are dealt alternately to two independent streams ("teams"): each team has its own S and O
-// accumulators in TMEM (S0 O0 S1 O1 = 512 columns), its own 256 softmax threads and its own running maximum and
+// accumulators in TMEM (S0 O0 S1 O1 = 512 columns), its own 128 softmax threads and its own running maximum and
 // row sum; the two are merged in the item's epilogue.  While one team
 // computes the exponentials of its tile, the tensor pipe runs the other team's products.
-// Warp roles: warp 0 and warps 18, 19 issue the TMA copies (warp 0 also stages the next item's query tile), warp 1
-// lane 0 issues the MMAs (warp 1 owns the TMEM allocation), warps 2-9 are team 0 and warps 10-17 team 1 (two
-// threads per TMEM lane, each owning 64 of the tile's 128 columns): softmax, rescale, epilogue.
+// Warp roles: warp 0 and warps 10, 11 issue the TMA copies (warp 0 also stages the next item's query tile), warp 1
+// lane 0 issues the MMAs (warp 1 owns the TMEM allocation), warps 2-5 are team 0 and warps 6-9 team 1 (one thread
+// per TMEM lane, holding its whole row of 128 scores in registers: twelve warps leave each thread 168 registers,
+// and a row needs no exchange between threads): softmax, rescale, epilogue.
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
 #include <algorithm>
@@ -36,7 +37,7 @@ constexpr int kTileN = 128;      // tokens per K/V tile (8 pages)
 constexpr int kKSlots = 3;        // K tiles in flight or in use (TMA, two 2 KB boxes per page: one per d half)
 constexpr int kVSlots = 2;        // V tiles (TMA, one 4 KB box per page)
 constexpr int kTeams = 2;              // independent tile streams: tile t of an item belongs to team t & 1
-constexpr int kSoftmaxThreads = 256;   // per team, two threads per row: columns [0,64) and [64,128)
+constexpr int kSoftmaxThreads = 128;   // per team: one thread per row of the tile
 constexpr int kProducers = 3;          // copy-issuing warps: K d-half 0 (+ query staging), K d-half 1, V
 constexpr int kThreads = 64 + kTeams * kSoftmaxThreads + (kProducers - 1) * 32;
 constexpr uint32_t kHalfBytes = kTileN * 64 * 2;        // one head-dim (or token) half of a 128x128 bf16 tile
@@ -52,9 +53,8 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint8_t v[kVSlots][kTileBytes];     // [page][d half][16 tokens][64], 128-byte swizzle
   uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
   uint64_t q_ready[2], q_free[2], s_full[kTeams], p_full[kTeams], pv_done[kTeams];
-  uint64_t pair[kTeams][4];           // the two warps of a team that share a TMEM lane quadrant meet here
   uint64_t both;                      // the two teams meet here around an item's epilogue
-  float xch[kTeams][2][kTileM];       // [team][column half][row]: row extremum / row sum exchange
+  float xch[kTeams][2][kTileM];       // [team][m, l][row]: the teams show each other their running maximum and row sum
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
   volatile int abort;
@@ -275,7 +275,7 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
   return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
 }
 
-__global__ void __maxnreg__(96)
+__global__ void __maxnreg__(168)
 prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
                  float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
@@ -312,7 +312,6 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       mbar_init(&sm.s_full[t], 1);
       mbar_init(&sm.p_full[t], kSoftmaxThreads);
       mbar_init(&sm.pv_done[t], 1);
-      for (int i = 0; i < 4; ++i) mbar_init(&sm.pair[t][i], 64);
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -514,19 +513,19 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       }
     }
   } else {
-    // ---------------------------------------------------------------- softmax / epilogue (two teams of 256 threads)
-    const int team = (warp - 2) >> 3;          // which of the item's two tile streams
+    // ---------------------------------------------------------------- softmax / epilogue (two teams of 128 threads)
+    // One thread owns one row of its team's tile: all 128 scores sit in its registers, so the row maximum and the
+    // row sum need no exchange between threads.
+    const int team = (warp - 2) >> 2;          // which of the item's two tile streams
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may access
-    const int half = ((warp - 2) >> 2) & 1;    // which 64 of the tile's 128 columns this thread owns
     const int r = quad * 32 + lane;            // row of the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
-    uint32_t pair_n = 0;                       // completed meetings of this warp pair
     uint32_t team_tiles = 0;                   // tiles this team has taken so far (all items)
     uint32_t other_tiles = 0;                  // ... and the other team
     uint32_t both_n = 0;                       // completed meetings of the two teams
     // The CTA's first item with work: its stacked query tile (128 rows x 16 chunks of 16 bytes) is staged here by
-    // all 512 softmax threads at once, four chunks each, instead of by the one producer warp in eight rounds -
+    // all 256 softmax threads at once, eight chunks each, instead of by the one producer warp in eight rounds -
     // nothing can start before it is in place.  Later items are staged by the producer under the item before.
     {
       int k0 = k_begin;
@@ -537,9 +536,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       }
       if (k0 < k_end) {
         const int tid = threadIdx.x - 64;
-        uint4 qv[4];
+        constexpr int kPer = kTileM * 16 / (kTeams * kSoftmaxThreads);
+        uint4 qv[kPer];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kPer; ++i) {
           const int idx = i * (kTeams * kSoftmaxThreads) + tid, row = idx >> 4, c = idx & 15;
           const int cand = qi.mt * cand_per_tile + row / g;
           qv[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -549,7 +549,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           }
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kPer; ++i) {
           const int idx = i * (kTeams * kSoftmaxThreads) + tid, row = idx >> 4, c = idx & 15;
           *reinterpret_cast<uint4 *>(sm.q[0] + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = qv[i];
         }
@@ -558,23 +558,6 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         if (warp == 2) mbar_arrive(&sm.q_ready[0]);                                       // its 32 arrivals
       }
     }
-    // The two threads of a row meet (bounded).
-    auto meet = [&]() -> bool {
-      mbar_arrive(&sm.pair[team][quad]);
-      bool w = mbar_wait(sm, p, &sm.pair[team][quad], pair_n & 1);
-      ++pair_n;
-      return __all_sync(0xffffffffu, w);
-    };
-    // Exchanges one float with the thread that owns the other half of the row.  The slot is reused: between the
-    // exchanges of two tiles lies a barrier round of the whole team (every thread announces its P after reading
-    // here, and the next tile's S follows the product that waited for all of them); around the epilogue's
-    // exchange, which has no such round on either side, the pair meets once more.
-    auto exchange = [&](float mine, float &theirs) -> bool {
-      sm.xch[team][half][r] = mine;
-      const bool w = meet();
-      if (w) theirs = sm.xch[team][half ^ 1][r];
-      return w;
-    };
     for (int k = k_begin; k < k_end && !sm.abort; ++k) {
       const Item it = decode_item(p, lvs, __ldg(item_list + k));
       if (it.mt * cand_per_tile >= it.n_cand) continue;
@@ -584,16 +567,16 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const size_t slot = qrow * p.n_parts + it.part;
       const int n_tiles = it.lo < it.hi ? (it.hi - it.lo + kTileN - 1) / kTileN : 0;
       if (n_tiles == 0) {   // no tokens in this split
-        if (row_ok && half == 0 && team == 0) lse_part[slot] = -INFINITY;
+        if (row_ok && team == 0) lse_part[slot] = -INFINITY;
         continue;
       }
       const int my_tiles = (n_tiles - team + 1) / kTeams, ot_tiles = n_tiles - my_tiles;   // tiles team, team + 2, ...
-      float m = -INFINITY, l = 0.f;   // m in log2 units (already multiplied by sl2); l: this thread's columns only
+      float m = -INFINITY, l = 0.f;   // running maximum in log2 units (already multiplied by sl2) and row sum
       // tokens of the item this row may see: the split's end, or less under a per-candidate limit (causal mask)
       const int hi_row = it.limits && row_ok ? min(it.hi, __ldg(it.limits + cand)) : it.hi;
       bool alive = true;
       for (int t = team; t < n_tiles && alive; t += kTeams, ++team_tiles) {
-        const int t0 = it.lo + t * kTileN, c0 = half * 64;
+        const int t0 = it.lo + t * kTileN;
         alive = mbar_wait(sm, p, &sm.s_full[team], team_tiles & 1);
         alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
         if (!alive) break;
@@ -601,47 +584,42 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
         const uint32_t page_ok = sm.page_ok[(kt + t) & 7];
         const bool full_tile = page_ok == 0xffu && t0 + kTileN <= hi_row;
-        // This thread's half row of S is read twice, 32 columns at a time - once for the row extremum, once for the
-        // exponentials - so that no more than 32 scores are held in registers at any time.
-        auto load_chunk = [&](int c, uint32_t (&sv)[32]) {
-          tmem_ld32(tmem_s + lane_addr + c0 + c * 32, sv);
+        // the whole row of S into registers: four loads in flight, one wait
+        uint32_t sv[kTileN];
+        auto load_row = [&]() {
+#pragma unroll
+          for (int c = 0; c < kTileN / 32; ++c)
+            tmem_ld32(tmem_s + lane_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
           tmem_wait_ld();
           if (!full_tile) {   // ragged tail or a bad page: masked scores become -inf (sl2 > 0) / +inf (sl2 < 0)
             const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int col = c0 + c * 32 + i;
+            for (int col = 0; col < kTileN; ++col) {
               const bool ok = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < hi_row);
-              if (!ok) sv[i] = masked;
+              if (!ok) sv[col] = masked;
             }
           }
         };
+        load_row();
         // row extremum of the raw scores; times sl2 it is the row maximum of the scaled scores
-        float ext = sl2 >= 0.f ? -INFINITY : INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sv[32];
-          load_chunk(c, sv);
-          float e4[4];
+        float ext;
+        {
+          float e8[8];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) e4[i] = __uint_as_float(sv[i]);
+          for (int i = 0; i < 8; ++i) e8[i] = __uint_as_float(sv[i]);
           if (sl2 >= 0.f) {
 #pragma unroll
-            for (int i = 4; i < 32; ++i) e4[i & 3] = fmaxf(e4[i & 3], __uint_as_float(sv[i]));
-            ext = fmaxf(ext, fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3])));
+            for (int i = 8; i < kTileN; ++i) e8[i & 7] = fmaxf(e8[i & 7], __uint_as_float(sv[i]));
+            ext = fmaxf(fmaxf(fmaxf(e8[0], e8[1]), fmaxf(e8[2], e8[3])), fmaxf(fmaxf(e8[4], e8[5]), fmaxf(e8[6], e8[7])));
           } else {
 #pragma unroll
-            for (int i = 4; i < 32; ++i) e4[i & 3] = fminf(e4[i & 3], __uint_as_float(sv[i]));
-            ext = fminf(ext, fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3])));
+            for (int i = 8; i < kTileN; ++i) e8[i & 7] = fminf(e8[i & 7], __uint_as_float(sv[i]));
+            ext = fminf(fminf(fminf(e8[0], e8[1]), fminf(e8[2], e8[3])), fminf(fminf(e8[4], e8[5]), fminf(e8[6], e8[7])));
           }
         }
-        float ext_other = ext;
-        alive = exchange(ext, ext_other);
-        if (!alive) break;
-        ext = sl2 >= 0.f ? fmaxf(ext, ext_other) : fminf(ext, ext_other);
         const float mx = (ext == INFINITY || ext == -INFINITY) ? -INFINITY : ext * sl2;   // all masked -> -inf
         // The running maximum moves only when the new one is clearly larger (2^8): P stays bounded by
-        // 2^8 and the accumulator in TMEM is rescaled rarely.  Both threads of a row decide alike.
+        // 2^8 and the accumulator in TMEM is rescaled rarely.
         float m_use = m;
         bool rescale = false;
         if (mx > m + 8.f) {
@@ -656,38 +634,36 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if (!alive) break;
           tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < 2; ++c) {   // this thread's 64 columns of O
+          for (int c = 0; c < D / 32; ++c) {   // this row of O
             uint32_t v[32];
-            tmem_ld32(tmem_o + lane_addr + c0 + c * 32, v);
+            tmem_ld32(tmem_o + lane_addr + c * 32, v);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-            tmem_st32(tmem_o + lane_addr + c0 + c * 32, v);
+            tmem_st32(tmem_o + lane_addr + c * 32, v);
           }
           tmem_wait_st();
+          load_row();   // the scores are read again rather than kept across this rare path
         }
         l *= alpha;
         m = m_use;
         const float neg_m = m == -INFINITY ? 0.f : -m;
         // P goes to TMEM as the A operand of the second product: lane = row, one column per token pair, written
-        // over the first half of the S columns this thread has read (the team's next first product, which
-        // overwrites S, is issued after the second product that reads this P).
+        // over S (all of it is in registers by now; the team's next first product, which overwrites S, is issued
+        // after the second product that reads this P).  Tokens [64 h + 32 c, +32) go to columns [64 h + 16 c, +16).
         float lsum[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sv[32], pw[16];                 // 32 tokens -> 16 packed columns
-          load_chunk(c, sv);
+#pragma unroll
+        for (int c = 0; c < kTileN / 32; ++c) {
+          uint32_t pw[16];                 // 32 tokens -> 16 packed columns
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * j]), sl2, neg_m));       // masked: exp2(-inf) = 0
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * j + 1]), sl2, neg_m));
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j]), sl2, neg_m));       // masked: exp2(-inf) = 0
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j + 1]), sl2, neg_m));
             lsum[j & 1] += p0;
             lsum[2 + (j & 1)] += p1;
             pw[j] = pack_bf16x2(p0, p1);
           }
-          // columns [c0 + 16 c, c0 + 16 c + 16): inside S columns [c0, c0 + 32), which this thread is done with
-          // (chunk 1 is re-read from [c0 + 32, c0 + 64) after chunk 0's P has been written)
-          tmem_st16(tmem_s + lane_addr + c0 + c * 16, pw);
+          tmem_st16(tmem_s + lane_addr + (c >> 1) * 64 + (c & 1) * 16, pw);
         }
         l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
         tmem_wait_st();
@@ -700,15 +676,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       other_tiles += ot_tiles;
       if (!alive) break;
       // ---- epilogue: the two streams of the item are merged here, so the item writes one part.
-      // Row sum of this team (the two halves'), then both teams publish (m, l) of every row and meet.
-      float l_other = 0.f;
-      alive = meet() && exchange(l, l_other) && meet();
-      if (!alive) break;
-      const float l_row = l + l_other;
-      if (half == 0) {   // the pair is past its last read of the exchange slots (second meeting above)
-        sm.xch[team][0][r] = m;
-        sm.xch[team][1][r] = l_row;
-      }
+      // Both teams publish (m, l) of every row and meet.
+      const float l_row = l;
+      sm.xch[team][0][r] = m;
+      sm.xch[team][1][r] = l_row;
       auto teams_meet = [&]() -> bool {
         mbar_arrive(&sm.both);
         bool w = mbar_wait(sm, p, &sm.both, both_n & 1);
@@ -730,16 +701,17 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       if (!__all_sync(0xffffffffu, alive)) break;
       tc_fence_after();
       const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-      // Each of the row's four threads takes 32 of the 128 output columns: [64 half + 32 team, +32).  A thread holds
-      // 32 columns of ONE row; a store instruction issued like that touches 32 rows, so the 32x32 block is
+      // Each of the row's two threads takes 64 of the 128 output columns, [64 team, +64), 32 at a time.  A thread
+      // holds 32 columns of ONE row; a store instruction issued like that touches 32 rows, so the 32x32 block is
       // transposed across the warp first (lane j then holds column j of all 32 rows) and every store instruction
       // writes 128 contiguous bytes of one row.
-      const int col0 = half * 64 + team * 32;
-      const unsigned long long my_off = (unsigned long long)slot * D + col0;
       const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_all > 0.f);
-      {
+      const float w_me = a_me * inv, w_ot = a_ot * inv;
+#pragma unroll 1
+      for (int cc = 0; cc < 2; ++cc) {
+        const int col0 = team * 64 + cc * 32;
+        const unsigned long long my_off = (unsigned long long)slot * D + col0;
         uint32_t v[32];
-        const float w_me = a_me * inv, w_ot = a_ot * inv;
         if (have_me) {
           tmem_ld32(tmem_o + lane_addr + col0, v);
           tmem_wait_ld();
@@ -774,7 +746,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if ((store_mask >> i) & 1u) o_part[off + lane] = __uint_as_float(v[i]);
         }
       }
-      if (row_ok && half == 0 && team == 0) lse_part[slot] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
+      if (row_ok && team == 0) lse_part[slot] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
       tc_fence_before();
       // nobody goes on (to overwrite an accumulator or an exchange slot) before everybody has read both
       alive = teams_meet();
