@@ -702,9 +702,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       tc_fence_after();
       const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
       // Each of the row's two threads takes 64 of the 128 output columns, [64 team, +64), 32 at a time.  A thread
-      // holds 32 columns of ONE row; a store instruction issued like that touches 32 rows, so the 32x32 block is
-      // transposed across the warp first (lane j then holds column j of all 32 rows) and every store instruction
-      // writes 128 contiguous bytes of one row.
+      // holds 32 columns (128 bytes) of ONE row; a store instruction issued like that touches 32 rows, 16 bytes of
+      // each, which costs the store path 32 cycles an instruction and leaves sectors half written.  So each group
+      // of 8 lanes first transposes its 8 rows x 8 pieces of 16 bytes (48 shuffles); a store instruction then
+      // writes 4 rows, 128 contiguous bytes of each.
       const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_all > 0.f);
       const float w_me = a_me * inv, w_ot = a_ot * inv;
 #pragma unroll 1
@@ -728,22 +729,30 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaf(__uint_as_float(w[i]), w_ot, __uint_as_float(v[i])));
         }
+        // transpose 8 x 8 blocks of 16-byte pieces inside each group of 8 lanes
 #pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) {
+        for (int s = 4; s >= 1; s >>= 1) {
           const bool up = (lane & s) != 0;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if (i & s) continue;
-            const uint32_t send = up ? v[i] : v[i | s];
-            const uint32_t got = __shfl_xor_sync(0xffffffffu, send, s);
-            if (up) v[i] = got; else v[i | s] = got;
+          for (int k = 0; k < 8; ++k) {
+            if (k & s) continue;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              const uint32_t send = up ? v[4 * k + w] : v[4 * (k | s) + w];
+              const uint32_t got = __shfl_xor_sync(0xffffffffu, send, s);
+              if (up) v[4 * k + w] = got; else v[4 * (k | s) + w] = got;
+            }
           }
         }
-        // v[i] now is element (row i of this warp's 32 rows, column col0 + lane)
+        // piece k of this lane now is (row 8 (lane / 8) + k of this warp's 32 rows, columns col0 + 4 (lane % 8) ...)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const unsigned long long off = __shfl_sync(0xffffffffu, my_off, i);
-          if ((store_mask >> i) & 1u) o_part[off + lane] = __uint_as_float(v[i]);
+        for (int k = 0; k < 8; ++k) {
+          const int src = (lane & 24) + k;
+          const unsigned long long off = __shfl_sync(0xffffffffu, my_off, src);
+          if ((store_mask >> src) & 1u)
+            *reinterpret_cast<float4 *>(o_part + off + 4 * (lane & 7)) =
+                make_float4(__uint_as_float(v[4 * k]), __uint_as_float(v[4 * k + 1]), __uint_as_float(v[4 * k + 2]),
+                            __uint_as_float(v[4 * k + 3]));
         }
       }
       if (row_ok && team == 0) lse_part[slot] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
