@@ -151,6 +151,19 @@ size_t mc_workspace_bytes(const mc_kv_layout_t *layout);
  * the device.  A candidate whose page row is full is left unchanged and MC_ERR_INVALID_ARG is latched. */
 mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *stream);
 
+/* mc_kv_append with rotary position embedding (the step of the language model's decode layer that precedes the
+ * attention; the paper takes the model as given and does not define it - the definition is the published one of
+ * Su et al., "RoFormer").  A head's d elements are d/2 complex numbers, element i the real and element i + d/2
+ * the imaginary part; the one at index i of a token at position pos is multiplied by exp(j pos theta_i),
+ * theta_i = theta_base^(-2 i / d).  pos of candidate b's new token = suffix_len[b] (before the increment) plus
+ * pos_offset[b] when pos_offset (device int32 [B]) is given, else plus the prefix lengths of b's groups on every
+ * cascade level, read on the device.  The rotated key row is stored in the cache, v_new unchanged; when q
+ * (device [B][Hq][d], 16-byte aligned) is not NULL its rows are rotated in place to the same position.  Angles
+ * are formed in double precision, the rotation in single precision, results rounded to `dtype`.  Errors as
+ * mc_kv_append; theta_base <= 0 is MC_ERR_INVALID_ARG. */
+mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *q,
+                              const int32_t *pos_offset, double theta_base, void *stream);
+
 /* Prefix pass: for every group and kv head, the stacked queries of all the group's candidates attend
  * to the group's prefix; writes parts [0, n_prefix_parts) of every row.  q: device [B][Hq][d]. */
 mc_status_t mc_prefix_attn(mc_kv_layout_t *layout, const void *q, float scale,

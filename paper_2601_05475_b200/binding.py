@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, byref, c_char_p, c_float, c_int32, c_size_t, c_uint64, c_void_p
+from ctypes import POINTER, byref, c_char_p, c_double, c_float, c_int32, c_size_t, c_uint64, c_void_p
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmaxcode_attn.so")
 _lib = None
@@ -43,6 +43,7 @@ EXPORTS = {
     "mc_kv_layout_geometry": (c_int32, [c_void_p, POINTER(PartGeometry)]),
     "mc_workspace_bytes": (c_size_t, [c_void_p]),
     "mc_kv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "mc_kv_append_rope": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_double, c_void_p]),
     "mc_prefix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
     "mc_suffix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
     "mc_merge_lse": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -144,6 +145,11 @@ def mc_kv_layout_validate(layout: int, scratch, scratch_bytes: int, stream: int 
 
 def mc_kv_append(layout: int, k_new, v_new, stream: int = 0) -> None:
     _check(lib().mc_kv_append(layout, _ptr(k_new), _ptr(v_new), stream), "mc_kv_append")
+
+
+def mc_kv_append_rope(layout: int, k_new, v_new, q, pos_offset, theta_base: float, stream: int = 0) -> None:
+    _check(lib().mc_kv_append_rope(layout, _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(pos_offset), theta_base, stream),
+           "mc_kv_append_rope")
 
 
 def mc_prefix_attn(layout: int, q, scale: float, o_part, lse_part, stream: int = 0) -> None:

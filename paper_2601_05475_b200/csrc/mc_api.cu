@@ -2,6 +2,7 @@
 // drivers that enqueue the passes.
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -71,6 +72,83 @@ __global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__re
     const size_t dst = (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + c;
     const size_t src = ((size_t)b * p.Hkv + h) * row_vec + c;
     if (which) vp[dst] = v_new[src]; else kp[dst] = k_new[src];
+  }
+  __syncthreads();  // every thread has read s and issued its stores before the length moves
+  if (threadIdx.x == 0) suffix_len[b] = s + 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// append with rotary position embedding: one block per candidate.  The head's d elements are d/2 complex
+// numbers (element i the real, i + d/2 the imaginary part); the one at index i is multiplied by
+// exp(j pos theta_i), theta_i = base^(-2 i / d), pos = the token's position in its whole sequence.  The angle is
+// formed and reduced in double precision (positions reach 10^5, where a single-precision angle is off by
+// 10^-2 radians); the rotation itself is single precision.  K is stored rotated, V as it is, q in place.
+// ------------------------------------------------------------------------------------------------
+struct RopeLevels {
+  int n;
+  int G[1 + kMaxOuterLevels];
+  const int32_t *group_offsets[1 + kMaxOuterLevels], *prefix_len[1 + kMaxOuterLevels];
+};
+
+template <typename T> __device__ __forceinline__ float rope_load(const T *p);
+template <> __device__ __forceinline__ float rope_load<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float rope_load<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void rope_store(float *p, float v) { *p = v; }
+__device__ __forceinline__ void rope_store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+template <typename T>
+__global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels lv, const T *__restrict__ k_new,
+                                                          const uint4 *__restrict__ v_new, T *q,
+                                                          const int32_t *__restrict__ pos_offset, double log2_base,
+                                                          int32_t *suffix_len) {
+  const int b = blockIdx.x;
+  const int s = suffix_len[b];
+  const int pg = s >> 4;
+  int page = -1;
+  if (s >= 0 && pg < p.max_sp) page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + pg);
+  if ((unsigned)page >= (unsigned)p.num_pages) {  // row full, or a bad table entry: leave the candidate alone
+    if (threadIdx.x == 0) latch(p, kDevBadPage);
+    return;
+  }
+  // position of the new token: the tokens before it, on every level of the cascade
+  long long pos = s;
+  if (pos_offset) {
+    pos += __ldg(pos_offset + b);
+  } else {
+    for (int k = 0; k < lv.n; ++k) {
+      int lo = 0, hi = lv.G[k];
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(lv.group_offsets[k] + mid) <= b) lo = mid; else hi = mid;
+      }
+      pos += max(__ldg(lv.prefix_len[k] + lo), 0);
+    }
+  }
+  const int half = p.d / 2, lanes = blockDim.x / half;   // d/2 divides the block size (d = 64 or 128)
+  const int i = threadIdx.x % half, h0 = threadIdx.x / half;
+  double sn, cs;
+  sincos((double)pos * exp2(-2.0 * i / p.d * log2_base), &sn, &cs);
+  const float c = (float)cs, sf = (float)sn;
+  T *kp = reinterpret_cast<T *>(const_cast<void *>(p.k_pool));
+  for (int h = h0; h < p.Hkv; h += lanes) {
+    const T *src = k_new + ((size_t)b * p.Hkv + h) * p.d;
+    T *dst = kp + (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * p.d;
+    const float re = rope_load(src + i), im = rope_load(src + i + half);
+    rope_store(dst + i, re * c - im * sf);
+    rope_store(dst + i + half, re * sf + im * c);
+  }
+  if (q)
+    for (int h = h0; h < p.Hq; h += lanes) {
+      T *row = q + ((size_t)b * p.Hq + h) * p.d;
+      const float re = rope_load(row + i), im = rope_load(row + i + half);
+      rope_store(row + i, re * c - im * sf);
+      rope_store(row + i + half, re * sf + im * c);
+    }
+  const int row_vec = p.d * (int)sizeof(T) / 16, n_vec = p.Hkv * row_vec;
+  uint4 *vp = reinterpret_cast<uint4 *>(const_cast<void *>(p.v_pool));
+  for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
+    const int h = j / row_vec, cc = j % row_vec;
+    vp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = v_new[((size_t)b * p.Hkv + h) * row_vec + cc];
   }
   __syncthreads();  // every thread has read s and issued its stores before the length moves
   if (threadIdx.x == 0) suffix_len[b] = s + 1;
@@ -487,6 +565,35 @@ mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *
   const int e = L->desc.dtype == MC_F32 ? 4 : 2;
   mc::append_kernel<<<L->p.B, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       L->p, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), L->desc.suffix_len, e);
+  mc::count_launch();
+  return mc::check_launch();
+}
+
+mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *q,
+                              const int32_t *pos_offset, double theta_base, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new) || (q && !mc::aligned16(q)))
+    return MC_ERR_INVALID_ARG;
+  if (!(theta_base > 0.0) || L->p.d % 2 != 0 || 256 % (L->p.d / 2) != 0) return MC_ERR_INVALID_ARG;
+  mc::RopeLevels lv;
+  lv.n = 1 + L->n_outer;
+  for (int k = 0; k < lv.n; ++k) {
+    const mc::Params &pk = k == 0 ? L->p : L->outer_p[k - 1];
+    lv.G[k] = pk.G;
+    lv.group_offsets[k] = pk.group_offsets;
+    lv.prefix_len[k] = pk.prefix_len;
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const double l2b = std::log2(theta_base);
+  if (L->desc.dtype == MC_F32)
+    mc::append_rope_kernel<float><<<L->p.B, 256, 0, st>>>(L->p, lv, reinterpret_cast<const float *>(k_new),
+                                                          reinterpret_cast<const uint4 *>(v_new),
+                                                          reinterpret_cast<float *>(q), pos_offset, l2b,
+                                                          L->desc.suffix_len);
+  else
+    mc::append_rope_kernel<__nv_bfloat16><<<L->p.B, 256, 0, st>>>(
+        L->p, lv, reinterpret_cast<const __nv_bfloat16 *>(k_new), reinterpret_cast<const uint4 *>(v_new),
+        reinterpret_cast<__nv_bfloat16 *>(q), pos_offset, l2b, L->desc.suffix_len);
   mc::count_launch();
   return mc::check_launch();
 }
