@@ -77,7 +77,9 @@ typedef struct {
   int32_t page_size;             /* must be 16 */
   int32_t num_pages;             /* pages in each pool */
   int32_t max_prefix_pages;      /* row stride of prefix_pages */
-  int32_t max_suffix_pages;      /* row stride of suffix_pages */
+  int32_t max_suffix_pages;      /* row stride of suffix_pages; 0: no private tokens at all (scoring whole
+                                    sequences): suffix_pages / suffix_len may be NULL, no suffix part slots,
+                                    no suffix launch, mc_kv_append returns MC_ERR_INVALID_ARG */
   int32_t dtype;                 /* mc_dtype_t */
   void *k_pool, *v_pool;         /* device */
   const int32_t *group_offsets;  /* device, [G+1] */

@@ -22,6 +22,7 @@ struct Layout {
   int32_t *host_status;  // pinned host int, target of the status read-back
   size_t o_part_bytes, lse_part_bytes, staging_off[5], ws_bytes;
   bool use_mma;
+  bool has_suffix;            // false: no private tokens (max_suffix_pages = 0), the suffix pass is not launched
   SuffixTmaPlan *sfx_plan;    // non-null: the suffix pass runs on the TMA-fed kernel
   PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
@@ -200,6 +201,7 @@ mc_status_t check_q(const Layout *L, const void *q) {
 
 mc_status_t run_level(Layout *L, const Params &p, int mode, const void *q, float scale, float *o_part,
                       float *lse_part, cudaStream_t st) {
+  if (mode == kSuffix && !L->has_suffix) return MC_OK;
   if (mode == kSuffix && L->sfx_plan) return launch_suffix_tma(p, L->sfx_plan, q, scale, o_part, lse_part, st, false);
   if (L->use_mma) return launch_mma(p, mode, q, scale, o_part, lse_part, st);
   return launch_fma(p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
@@ -293,11 +295,13 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   if (out) *out = nullptr;
   if (!d || !out) return MC_ERR_INVALID_ARG;
   if (d->num_groups < 1 || d->batch < 1 || d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_pages < 1 ||
-      d->max_prefix_pages < 1 || d->max_suffix_pages < 1 || d->batch < d->num_groups)
+      d->max_prefix_pages < 1 || d->max_suffix_pages < 0 || d->batch < d->num_groups)
     return MC_ERR_INVALID_ARG;
   if (d->num_q_heads % d->num_kv_heads != 0) return MC_ERR_INVALID_ARG;
-  if (!d->k_pool || !d->v_pool || !d->group_offsets || !d->prefix_pages || !d->prefix_len || !d->suffix_pages ||
-      !d->suffix_len)
+  // max_suffix_pages = 0: a layout without private tokens (scoring of whole sequences); no suffix tables, no suffix
+  // part slots, no suffix launch, appends refused
+  if (!d->k_pool || !d->v_pool || !d->group_offsets || !d->prefix_pages || !d->prefix_len ||
+      (d->max_suffix_pages > 0 && (!d->suffix_pages || !d->suffix_len)))
     return MC_ERR_INVALID_ARG;
   if (!mc::aligned16(d->k_pool) || !mc::aligned16(d->v_pool)) return MC_ERR_INVALID_ARG;
   if (n_outer < 0 || n_outer > mc::kMaxOuterLevels || (n_outer > 0 && !outer)) return MC_ERR_INVALID_ARG;
@@ -343,7 +347,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   int32_t *sl = nullptr;
   {
     sl = new (std::nothrow) int32_t[p.B];
-    if (sl && cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
+    if (sl && max_s > 0 && cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
       double suffix_tokens = 0.0;
       for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
       suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : 2) / 6.8e6;   // stream at ~6.8 TB/s
@@ -402,7 +406,8 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     pk.n_parts = n_parts;
   }
   L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
-  L->sfx_plan = L->use_mma && mc::env_int("MC_SUFFIX_TMA", 1) ? mc::suffix_tma_plan(p, d->dtype) : nullptr;
+  L->has_suffix = n_parts > part_base;
+  L->sfx_plan = L->has_suffix && L->use_mma && mc::env_int("MC_SUFFIX_TMA", 1) ? mc::suffix_tma_plan(p, d->dtype) : nullptr;
   // Suffix CTAs are launched longest first (by the lengths as they are now; appends change them slowly), so
   // that the launch ends on short items instead of a few long ones.  Without it the order is as numbered.
   L->suffix_order = nullptr;
@@ -562,6 +567,7 @@ mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t 
 mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *stream) {
   Layout *L = reinterpret_cast<Layout *>(layout);
   if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new)) return MC_ERR_INVALID_ARG;
+  if (!L->has_suffix) return MC_ERR_INVALID_ARG;   // a layout without private tokens has nowhere to append
   const int e = L->desc.dtype == MC_F32 ? 4 : 2;
   mc::append_kernel<<<L->p.B, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       L->p, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), L->desc.suffix_len, e);
@@ -574,7 +580,7 @@ mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const v
   Layout *L = reinterpret_cast<Layout *>(layout);
   if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new) || (q && !mc::aligned16(q)))
     return MC_ERR_INVALID_ARG;
-  if (!(theta_base > 0.0) || L->p.d % 2 != 0 || 256 % (L->p.d / 2) != 0) return MC_ERR_INVALID_ARG;
+  if (!L->has_suffix || !(theta_base > 0.0) || L->p.d % 2 != 0 || 256 % (L->p.d / 2) != 0) return MC_ERR_INVALID_ARG;
   mc::RopeLevels lv;
   lv.n = 1 + L->n_outer;
   for (int k = 0; k < lv.n; ++k) {
@@ -646,9 +652,11 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
     // the step is replayed from a captured graph.  The merge, launched the ordinary way, waits for both.
     if (k_new && (s = mc_kv_append(layout, k_new, v_new, st)) != MC_OK) return s;
     if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st)) != MC_OK) return s;
-    s = L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
-                    : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
-    if (s != MC_OK) return s;
+    if (L->has_suffix) {
+      s = L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
+                      : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
+      if (s != MC_OK) return s;
+    }
     return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
   }
   // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix

@@ -175,7 +175,8 @@ class ScoringDeviceProblem:
     level is the shared prompts and whose one outer level is each sequence's own tokens under a causal row limit.
     Memory and marshalling only."""
 
-    def __init__(self, hp: "wl.ScoringHostProblem", device="cuda"):
+    def __init__(self, hp: "wl.ScoringHostProblem", device="cuda", suffix_storage: bool = False):
+        """suffix_storage: give the layout (empty) suffix tables, as a decode layout has, instead of none."""
         cfg = hp.cfg
         self.cfg, self.hp = cfg, hp
         i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
@@ -188,11 +189,12 @@ class ScoringDeviceProblem:
         d = mc.LayoutDesc()
         d.num_groups, d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = cfg.G, Bv, cfg.Hq, cfg.Hkv, cfg.d
         d.page_size, d.num_pages = wl.PAGE, hp.k_pool.shape[0]
-        d.max_prefix_pages, d.max_suffix_pages = hp.prefix_pages.shape[1], 1
+        d.max_prefix_pages, d.max_suffix_pages = hp.prefix_pages.shape[1], 1 if suffix_storage else 0
         d.dtype = mc.MC_F32 if cfg.dtype == "f32" else mc.MC_BF16
         d.k_pool, d.v_pool = self.k_pool.data_ptr(), self.v_pool.data_ptr()
         d.group_offsets, d.prefix_pages, d.prefix_len = (self.t[k].data_ptr() for k in ("go", "pp", "pl"))
-        d.suffix_pages, d.suffix_len = self.t["sp"].data_ptr(), self.t["sl"].data_ptr()
+        if suffix_storage:
+            d.suffix_pages, d.suffix_len = self.t["sp"].data_ptr(), self.t["sl"].data_ptr()
         lv = mc.PrefixLevel()
         lv.num_groups, lv.max_pages = cfg.B, hp.seq_pages.shape[1]
         lv.group_offsets, lv.pages, lv.len = (self.t[k].data_ptr() for k in ("so", "qp", "ql"))

@@ -26,12 +26,16 @@ CASES = {
 }
 
 
+@pytest.mark.parametrize("suffix_storage", [False, True])
 @pytest.mark.parametrize("name", list(CASES))
-def test_scoring_matches_oracle(name):
+def test_scoring_matches_oracle(name, suffix_storage):
+    """suffix_storage False: a layout without private tokens (no suffix part slot, no suffix launch); True: a decode
+    layout whose suffixes happen to be empty (the suffix pass runs and reports empty parts)."""
     cfg, prefix_len, seq_len = CASES[name]
     hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
     q = wl.draw_scoring_q(cfg, seq_len)
-    dp = ScoringDeviceProblem(hp)
+    dp = ScoringDeviceProblem(hp, suffix_storage=suffix_storage)
+    assert dp.geom.n_parts == dp.geom.n_prefix_parts + (1 if suffix_storage else 0)
     assert (dp.geom.prefix_ctas > 0) == (cfg.dtype == "bf16")      # bf16 cases run on the tcgen05 kernel
     scratch = torch.empty(hp.k_pool.shape[0], dtype=torch.int32, device="cuda")
     assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_OK
@@ -45,6 +49,10 @@ def test_scoring_matches_oracle(name):
     tol = (1e-5, 1e-5) if cfg.dtype == "f32" else (2e-2, 2e-3)
     assert err.max() <= tol[0] and err.mean() <= tol[1], (err.max(), err.mean())
     assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    if not suffix_storage:       # nowhere to append
+        kv = to_device(cfg, np.zeros((dp.n_virtual, cfg.Hkv, cfg.d), dtype=np.float32))
+        with pytest.raises(mc.McError):
+            mc.mc_kv_append(dp.layout, kv, kv)
     dp.close()
 
 
