@@ -21,6 +21,7 @@
 // Every mbarrier wait is bounded: on expiry the CTA latches MC_ERR_TIMEOUT, stops issuing work, waits
 // (bounded) for its outstanding copies, frees its TMEM and returns.
 #include <algorithm>
+#include <cstdlib>
 #include <functional>
 #include <queue>
 #include <utility>
@@ -220,6 +221,8 @@ struct TcLevel {
   const int32_t *group_offsets, *prefix_pages, *prefix_len;
   const int32_t *row_limit;   // per candidate: tokens of this level it may see (non-decreasing within a group), or null
   int32_t max_pp, n_splits, part_base, part_tokens, n_mt, item_end;
+  int32_t n_groups;
+  int32_t chain;   // >= 0: an item of this level also covers, for its rows, the whole prefix of that (coarser) level
 };
 struct TcLevels {
   int32_t n;
@@ -233,6 +236,10 @@ struct Item {
   int lo, hi;            // token range of this split
   const int32_t *pages;
   const int32_t *limits; // per-candidate token limits of the group (indexed from its first candidate), or null
+  // second token range, of the coarser level this level is chained to (lo2 >= hi2: none): the rows of the tile lie
+  // in one group of that level, whose prefix the item attends in the same pass, into the same accumulator
+  int lo2, hi2, part2;
+  const int32_t *pages2, *limits2;
 };
 
 __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs, int item) {
@@ -267,12 +274,39 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
     const int last = min((it.mt + 1) * cand_per_tile, it.n_cand) - 1;
     if (last >= it.mt * cand_per_tile) it.hi = min(it.hi, max(__ldg(it.limits + last), 0));
   }
+  it.lo2 = it.hi2 = 0;
+  it.part2 = -1;
+  it.pages2 = it.limits2 = nullptr;
+  if (L.chain >= 0) {
+    const TcLevel &C = lvs.lv[L.chain];
+    int lo = 0, hi = C.n_groups;   // the coarser level's group that holds this group: offsets[lo] <= b0 < offsets[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(C.group_offsets + mid) <= it.b0) lo = mid; else hi = mid;
+    }
+    int len2 = __ldg(C.prefix_len + lo);
+    const int cap2 = C.max_pp * kPage;
+    if (len2 < 0 || len2 > cap2) {
+      latch(p, kDevBadPage);
+      len2 = len2 < 0 ? 0 : cap2;
+    }
+    it.part2 = C.part_base;
+    it.hi2 = len2;
+    it.pages2 = C.prefix_pages + (size_t)lo * C.max_pp;
+    if (C.row_limit) {
+      it.limits2 = C.row_limit + it.b0;
+      const int cand_per_tile = kTileM / p.g;
+      const int last = min((it.mt + 1) * cand_per_tile, it.n_cand) - 1;
+      if (last >= it.mt * cand_per_tile) it.hi2 = min(it.hi2, max(__ldg(it.limits2 + last), 0));
+    }
+  }
   return it;
 }
+__device__ __forceinline__ int tiles_of(int lo, int hi) { return lo < hi ? (hi - lo + kTileN - 1) / kTileN : 0; }
 
 // An item with no rows or no tokens is skipped by every role alike.
 __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile) {
-  return it.lo < it.hi && it.mt * cand_per_tile < it.n_cand;
+  return (it.lo < it.hi || it.lo2 < it.hi2) && it.mt * cand_per_tile < it.n_cand;
 }
 
 __global__ void __maxnreg__(168)
@@ -395,21 +429,25 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     while (ok && cur < k_end && !sm.abort) {
       const int nxt_idx = next_item(cur + 1, nxt);
       int round = nxt_idx < k_end && prole == 0 ? 0 : kQRounds + 1;   // staging state of the next item's query tile
-      const int last_pg = (it.hi - 1) >> 4;
+      for (int seg = 0; seg < 2 && ok; ++seg) {
+      const int seg_lo = seg ? it.lo2 : it.lo, seg_hi = seg ? it.hi2 : it.hi;
+      const int32_t *seg_pages = seg ? it.pages2 : it.pages;
+      if (seg_lo >= seg_hi) continue;
+      const int last_pg = (seg_hi - 1) >> 4;
       // Page ids are read 32 at a time (four tiles' worth, one per lane) a block ahead of their use, so that no
       // tile waits for a table look-up.  Pages past the end of the prefix repeat the last valid page: finite
       // data, masked later.
-      auto load_ids = [&](int blk) -> int { return __ldg(it.pages + min((it.lo >> 4) + blk * 32 + lane, last_pg)); };
+      auto load_ids = [&](int blk) -> int { return __ldg(seg_pages + min((seg_lo >> 4) + blk * 32 + lane, last_pg)); };
       int ids_cur = load_ids(0), ids_next = load_ids(1);
       int tile = 0;
-      for (int t0 = it.lo; t0 < it.hi; t0 += kTileN, ++kt, ++tile) {
+      for (int t0 = seg_lo; t0 < seg_hi; t0 += kTileN, ++kt, ++tile) {
         // lane pg (and every lane with the same low three bits) gets the id of the tile's page pg
         int pid = __shfl_sync(0xffffffffu, ids_cur, (tile & 3) * 8 + (lane & 7));
         if ((tile & 3) == 3) {
           ids_cur = ids_next;
           ids_next = load_ids((tile >> 2) + 2);
         }
-        const bool in_range = t0 + (lane & 7) * kPage < it.hi, good = (unsigned)pid < (unsigned)p.num_pages;
+        const bool in_range = t0 + (lane & 7) * kPage < seg_hi, good = (unsigned)pid < (unsigned)p.num_pages;
         if (lane < 8 && in_range && !good && prole == 0) latch(p, kDevBadPage);
         if (!good) pid = 0;   // a bad page id is replaced by page 0 and its 16 columns are masked
         const uint32_t okmask = __ballot_sync(0xffffffffu, in_range && good) & 0xffu;
@@ -444,6 +482,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if (!ok) break;
         }
       }
+      }   // token ranges of the item
       while (ok && round <= kQRounds) ok = q_step(nxt, it_n + 1, round);   // short item: finish the staging now
       it = nxt;
       cur = nxt_idx;
@@ -461,7 +500,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         ++it_n;
         tc_fence_after();
         const uint64_t q_desc = smem_desc(smem_u32(sm.q[qb]), 16, 1024);
-        const int n_tiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+        const int n_tiles = tiles_of(it.lo, it.hi) + tiles_of(it.lo2, it.hi2);
         // Tile t belongs to team t & 1.  Per team the order on the tensor pipe is S(t), O += P(t) V(t), S(t+2), ...:
         // P(t) lies over S(t), so S(t+2) may only follow the second product of tile t; the other team's products
         // fill the gaps.  Products complete in issue order.  The first product of the next item follows this item's
@@ -565,7 +604,9 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const bool row_ok = cand < it.n_cand;
       const size_t qrow = (size_t)(it.b0 + cand) * p.Hq + (size_t)it.h * g + (r % g);
       const size_t slot = qrow * p.n_parts + it.part;
-      const int n_tiles = it.lo < it.hi ? (it.hi - it.lo + kTileN - 1) / kTileN : 0;
+      const int n_tiles1 = tiles_of(it.lo, it.hi), n_tiles = n_tiles1 + tiles_of(it.lo2, it.hi2);
+      // a chained item answers for the coarser level's part slot of its rows too: it stays empty
+      if (row_ok && team == 0 && it.part2 >= 0) lse_part[qrow * p.n_parts + it.part2] = -INFINITY;
       if (n_tiles == 0) {   // no tokens in this split
         if (row_ok && team == 0) lse_part[slot] = -INFINITY;
         continue;
@@ -573,10 +614,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const int my_tiles = (n_tiles - team + 1) / kTeams, ot_tiles = n_tiles - my_tiles;   // tiles team, team + 2, ...
       float m = -INFINITY, l = 0.f;   // running maximum in log2 units (already multiplied by sl2) and row sum
       // tokens of the item this row may see: the split's end, or less under a per-candidate limit (causal mask)
-      const int hi_row = it.limits && row_ok ? min(it.hi, __ldg(it.limits + cand)) : it.hi;
+      const int hi_row1 = it.limits && row_ok ? min(it.hi, __ldg(it.limits + cand)) : it.hi;
+      const int hi_row2 = it.limits2 && row_ok ? min(it.hi2, __ldg(it.limits2 + cand)) : it.hi2;
       bool alive = true;
       for (int t = team; t < n_tiles && alive; t += kTeams, ++team_tiles) {
-        const int t0 = it.lo + t * kTileN;
+        const int t0 = t < n_tiles1 ? it.lo + t * kTileN : it.lo2 + (t - n_tiles1) * kTileN;
+        const int hi_row = t < n_tiles1 ? hi_row1 : hi_row2;
         alive = mbar_wait(sm, p, &sm.s_full[team], team_tiles & 1);
         alive = __all_sync(0xffffffffu, alive);   // also reconverges the warp before the collective TMEM loads
         if (!alive) break;
@@ -850,6 +893,11 @@ bool prefix_tc_supported(const Params &p, int dtype) {
 
 namespace {
 
+bool env_chain_levels() {
+  const char *e = std::getenv("MC_PREFIX_CHAIN");
+  return !(e && *e == '0');
+}
+
 // Longest-processing-time-first assignment of items (sorted by cost, descending) to `grid` CTAs; returns the
 // largest CTA load and, if asked, which CTA each item went to.
 double lpt_assign(const std::vector<int> &by_cost, const std::vector<double> &cost, int grid, std::vector<int> *owner) {
@@ -891,6 +939,45 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   long long items = 0;
   plan->levels.n = n_levels;
   std::vector<double> cost;
+  // Two single-split levels of which one's groups nest in the other's, with as many 128-row tiles: the finer level's
+  // items take the coarser level's tokens along (one item, one accumulator, one part per row tile instead of two
+  // items and two parts), and the coarser level gets no items of its own.
+  int fine = -1, coarse = -1;
+  std::vector<int32_t> coarse_len, coarse_go;
+  if (n_levels == 2 && levels[0].n_prefix_parts == 1 && levels[1].n_prefix_parts == 1 && env_chain_levels()) {
+    std::vector<int32_t> go[2];
+    bool known = true;
+    for (int k = 0; k < 2; ++k) {
+      go[k].resize((size_t)levels[k].G + 1);
+      known = known && cudaMemcpy(go[k].data(), levels[k].group_offsets, sizeof(int32_t) * go[k].size(),
+                                  cudaMemcpyDeviceToHost) == cudaSuccess;
+    }
+    (void)cudaGetLastError();
+    for (int f = 0; f < 2 && known && fine < 0; ++f) {
+      const int c = 1 - f;
+      if (levels[f].G < levels[c].G) continue;
+      // every boundary of the coarser level is a boundary of the finer one, and the row tiles add up to as many
+      bool nested = true;
+      size_t i = 0;
+      long long tiles_f = 0, tiles_c = 0;
+      for (int j = 0; j <= levels[c].G && nested; ++j) {
+        while (i < go[f].size() && go[f][i] < go[c][(size_t)j]) ++i;
+        nested = i < go[f].size() && go[f][i] == go[c][(size_t)j];
+      }
+      for (int j = 0; j < levels[f].G; ++j) tiles_f += ((long long)(go[f][(size_t)j + 1] - go[f][(size_t)j]) * p.g + kTileM - 1) / kTileM;
+      for (int j = 0; j < levels[c].G; ++j) tiles_c += ((long long)(go[c][(size_t)j + 1] - go[c][(size_t)j]) * p.g + kTileM - 1) / kTileM;
+      if (nested && tiles_f <= tiles_c) {
+        coarse_len.resize((size_t)levels[c].G);
+        if (cudaMemcpy(coarse_len.data(), levels[c].prefix_len, sizeof(int32_t) * coarse_len.size(),
+                       cudaMemcpyDeviceToHost) == cudaSuccess) {
+          fine = f;
+          coarse = c;
+          coarse_go = go[c];
+        }
+        (void)cudaGetLastError();
+      }
+    }
+  }
   for (int k = 0; k < n_levels; ++k) {
     const Params &pk = levels[k];
     TcLevel &lv = plan->levels.lv[k];
@@ -902,6 +989,8 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.n_splits = pk.n_prefix_parts;
     lv.part_base = pk.prefix_part_base;
     lv.part_tokens = pk.prefix_part_tokens;
+    lv.n_groups = pk.G;
+    lv.chain = k == fine ? coarse : -1;
     lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
     const long long level_items = (long long)pk.G * pk.Hkv * lv.n_splits * lv.n_mt;
     items += level_items;
@@ -929,14 +1018,27 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
       l = l < 0 ? 0 : l > cap ? cap : l;
       const long long lo = (long long)sp * lv.part_tokens;
       const long long tokens = (l < lo + lv.part_tokens ? l : lo + lv.part_tokens) - lo;
+      long long tiles = tokens > 0 ? (tokens + kTileN - 1) / kTileN : 0;
+      if (k == fine && known) {   // plus the tokens of the coarser group around this one
+        size_t j2 = 0;
+        while (j2 + 1 < coarse_go.size() - 1 && coarse_go[j2 + 1] <= go[(size_t)j]) ++j2;
+        const long long cap2 = (long long)levels[coarse].max_pp * kPage;
+        long long l2 = coarse_len[j2];
+        l2 = l2 < 0 ? 0 : l2 > cap2 ? cap2 : l2;
+        tiles += (l2 + kTileN - 1) / kTileN;
+      }
       double c = 0.0;
-      if (tokens > 0 && mt * cand_per_tile < n_cand) c = (double)((tokens + kTileN - 1) / kTileN) * tile_us + item_us;
+      if (k != coarse && tiles > 0 && mt * cand_per_tile < n_cand) c = (double)tiles * tile_us + item_us;
       cost.push_back(c);
     }
   }
   plan->n_items = (int)items;
-  std::vector<int> by_cost((size_t)plan->n_items);
-  for (int i = 0; i < plan->n_items; ++i) by_cost[(size_t)i] = i;
+  const int coarse_begin = coarse < 0 ? 0 : coarse == 0 ? 0 : plan->levels.lv[coarse - 1].item_end;
+  const int coarse_end = coarse < 0 ? 0 : plan->levels.lv[coarse].item_end;
+  std::vector<int> by_cost;
+  by_cost.reserve((size_t)plan->n_items);
+  for (int i = 0; i < plan->n_items; ++i)
+    if (i < coarse_begin || i >= coarse_end) by_cost.push_back(i);   // the coarser level of a chain has no items
   std::stable_sort(by_cost.begin(), by_cost.end(), [&](int a, int b) { return cost[(size_t)a] > cost[(size_t)b]; });
   int live = 0;
   for (int i = 0; i < plan->n_items; ++i) live += cost[(size_t)i] > 0.0;
@@ -957,12 +1059,12 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   plan->grid = grid;
   std::vector<int> owner((size_t)plan->n_items, 0);
   lpt_assign(by_cost, cost, grid, &owner);
-  std::vector<int32_t> lists((size_t)grid + 1 + (size_t)plan->n_items, 0);
-  for (int i = 0; i < plan->n_items; ++i) lists[(size_t)owner[(size_t)i] + 1] += 1;
+  std::vector<int32_t> lists((size_t)grid + 1 + by_cost.size(), 0);
+  for (size_t i = 0; i < by_cost.size(); ++i) lists[(size_t)owner[(size_t)by_cost[i]] + 1] += 1;
   for (int c = 0; c < grid; ++c) lists[(size_t)c + 1] += lists[(size_t)c];
   std::vector<int32_t> fill(lists.begin(), lists.begin() + grid);
-  for (int i = 0; i < plan->n_items; ++i) {   // costliest first within each CTA
-    const int it = by_cost[(size_t)i];
+  for (size_t i = 0; i < by_cost.size(); ++i) {   // costliest first within each CTA
+    const int it = by_cost[i];
     lists[(size_t)grid + 1 + (size_t)fill[(size_t)owner[(size_t)it]]++] = it;
   }
   if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

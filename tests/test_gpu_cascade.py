@@ -42,8 +42,11 @@ CASES = {
 }
 
 
+@pytest.mark.parametrize("chain", ["1", "0"])
 @pytest.mark.parametrize("name", list(CASES))
-def test_cascade_matches_oracle(name):
+def test_cascade_matches_oracle(name, chain, monkeypatch):
+    """chain: two nested single-split levels run as one item per row tile (the default) or as separate items."""
+    monkeypatch.setenv("MC_PREFIX_CHAIN", chain)
     cfg, outer = CASES[name]
     hp = wl.make_host_problem(cfg)
     for i, (go, lens) in enumerate(outer):

@@ -28,12 +28,15 @@ CASES = {
 
 @pytest.mark.parametrize("suffix_storage", [False, True])
 @pytest.mark.parametrize("name", list(CASES))
-def test_scoring_matches_oracle(name, suffix_storage):
-    """suffix_storage False: a layout without private tokens (no suffix part slot, no suffix launch); True: a decode
+def test_scoring_matches_oracle(name, suffix_storage, monkeypatch):
+    """suffix_storage True also runs the two levels as separate items (MC_PREFIX_CHAIN=0) instead of chained ones.
+    suffix_storage False: a layout without private tokens (no suffix part slot, no suffix launch); True: a decode
     layout whose suffixes happen to be empty (the suffix pass runs and reports empty parts)."""
     cfg, prefix_len, seq_len = CASES[name]
     hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
     q = wl.draw_scoring_q(cfg, seq_len)
+    if suffix_storage:
+        monkeypatch.setenv("MC_PREFIX_CHAIN", "0")
     dp = ScoringDeviceProblem(hp, suffix_storage=suffix_storage)
     assert dp.geom.n_parts == dp.geom.n_prefix_parts + (1 if suffix_storage else 0)
     assert (dp.geom.prefix_ctas > 0) == (cfg.dtype == "bf16")      # bf16 cases run on the tcgen05 kernel
