@@ -646,6 +646,12 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
   // The two passes write disjoint part slots and run side by side.  The prefix pass (tensor-bound, a few
   // persistent CTAs, each needing an SM's whole shared memory) must get its CTAs placed before the suffix pass
   // (HBM-bound, thousands of short CTAs) fills every SM.
+  if (L->tc_plan && scale != 0.f && !L->has_suffix && mc::prefix_tc_one_part_per_row(L->tc_plan) &&
+      mc::env_int("MC_PREFIX_DIRECT", 1)) {
+    // No private tokens and one part per row from the prefix pass: it writes the final output itself, no merge.
+    if (k_new) return MC_ERR_INVALID_ARG;   // nowhere to append
+    return mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st, o, lse);
+  }
   if (L->tc_plan && L->use_mma && scale != 0.f && L->pdl) {
     // One stream: the suffix pass is launched behind the tensor-core prefix pass as its programmatic
     // dependent, so it starts once every prefix CTA is running, not when they end.  The order holds when

@@ -313,7 +313,11 @@ __global__ void __maxnreg__(168)
 prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
                  float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
-                 const int32_t *__restrict__ cta_begin) {
+                 const int32_t *__restrict__ cta_begin, __nv_bfloat16 *__restrict__ o_final,
+                 float *__restrict__ lse_final) {
+  // o_final != null: every row gets exactly one part from this launch and none from anywhere else, so the item
+  // writes the row's final output (bf16) and log-sum-exp itself and no merge follows.
+  const bool direct = o_final != nullptr;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base
@@ -606,9 +610,16 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       const size_t slot = qrow * p.n_parts + it.part;
       const int n_tiles1 = tiles_of(it.lo, it.hi), n_tiles = n_tiles1 + tiles_of(it.lo2, it.hi2);
       // a chained item answers for the coarser level's part slot of its rows too: it stays empty
-      if (row_ok && team == 0 && it.part2 >= 0) lse_part[qrow * p.n_parts + it.part2] = -INFINITY;
+      if (!direct && row_ok && team == 0 && it.part2 >= 0) lse_part[qrow * p.n_parts + it.part2] = -INFINITY;
       if (n_tiles == 0) {   // no tokens in this split
-        if (row_ok && team == 0) lse_part[slot] = -INFINITY;
+        if (direct && row_ok) {   // the row's output is zero, its log-sum-exp -infinity; each team writes 64 columns
+          uint4 *dst = reinterpret_cast<uint4 *>(o_final + qrow * D + team * 64);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (team == 0) lse_final[qrow] = -INFINITY;
+        } else if (row_ok && team == 0) {
+          lse_part[slot] = -INFINITY;
+        }
         continue;
       }
       const int my_tiles = (n_tiles - team + 1) / kTeams, ot_tiles = n_tiles - my_tiles;   // tiles team, team + 2, ...
@@ -749,12 +760,12 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       // each, which costs the store path 32 cycles an instruction and leaves sectors half written.  So each group
       // of 8 lanes first transposes its 8 rows x 8 pieces of 16 bytes (48 shuffles); a store instruction then
       // writes 4 rows, 128 contiguous bytes of each.
-      const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && l_all > 0.f);
+      const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && (direct || l_all > 0.f));
       const float w_me = a_me * inv, w_ot = a_ot * inv;
 #pragma unroll 1
       for (int cc = 0; cc < 2; ++cc) {
         const int col0 = team * 64 + cc * 32;
-        const unsigned long long my_off = (unsigned long long)slot * D + col0;
+        const unsigned long long my_off = (unsigned long long)(direct ? qrow : slot) * D + col0;
         uint32_t v[32];
         if (have_me) {
           tmem_ld32(tmem_o + lane_addr + col0, v);
@@ -792,13 +803,18 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         for (int k = 0; k < 8; ++k) {
           const int src = (lane & 24) + k;
           const unsigned long long off = __shfl_sync(0xffffffffu, my_off, src);
-          if ((store_mask >> src) & 1u)
+          if (!((store_mask >> src) & 1u)) continue;
+          if (direct)
+            *reinterpret_cast<uint2 *>(o_final + off + 4 * (lane & 7)) =
+                make_uint2(pack_bf16x2(__uint_as_float(v[4 * k]), __uint_as_float(v[4 * k + 1])),
+                           pack_bf16x2(__uint_as_float(v[4 * k + 2]), __uint_as_float(v[4 * k + 3])));
+          else
             *reinterpret_cast<float4 *>(o_part + off + 4 * (lane & 7)) =
                 make_float4(__uint_as_float(v[4 * k]), __uint_as_float(v[4 * k + 1]), __uint_as_float(v[4 * k + 2]),
                             __uint_as_float(v[4 * k + 3]));
         }
       }
-      if (row_ok && team == 0) lse_part[slot] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
+      if (row_ok && team == 0) (direct ? lse_final[qrow] : lse_part[slot]) = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
       tc_fence_before();
       // nobody goes on (to overwrite an accumulator or an exchange slot) before everybody has read both
       alive = teams_meet();
@@ -880,6 +896,7 @@ struct PrefixTcPlan {
   CUtensorMap k_map, v_map;
   TcLevels levels;
   int n_items, grid;
+  bool one_part_per_row;   // every row gets exactly one part from this pass: one single-split level, or two chained
   int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
@@ -1057,6 +1074,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     grid = lo;
   }
   plan->grid = grid;
+  plan->one_part_per_row = (n_levels == 1 && levels[0].n_prefix_parts == 1) || fine >= 0;
   std::vector<int> owner((size_t)plan->n_items, 0);
   lpt_assign(by_cost, cost, grid, &owner);
   std::vector<int32_t> lists((size_t)grid + 1 + by_cost.size(), 0);
@@ -1086,11 +1104,15 @@ void prefix_tc_plan_free(PrefixTcPlan *plan) {
 int prefix_tc_grid(const PrefixTcPlan *plan) { return plan ? plan->grid : 0; }
 
 
+bool prefix_tc_one_part_per_row(const PrefixTcPlan *plan) { return plan && plan->one_part_per_row; }
+
+// o_final / lse_final non-null (only for a plan with one part per row, and only when no other pass adds parts): the
+// pass writes the final bf16 output and log-sum-exp of every row itself instead of partial results.
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
-                             float *lse_part, cudaStream_t stream) {
+                             float *lse_part, cudaStream_t stream, void *o_final, float *lse_final) {
   prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
       p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part,
-      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists);
+      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final);
   count_launch();
   return check_launch();
 }

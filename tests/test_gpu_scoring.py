@@ -89,3 +89,35 @@ def test_decreasing_row_limits_are_reported_by_validate():
     scratch = torch.empty(hp.k_pool.shape[0], dtype=torch.int32, device="cuda")
     assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_ERR_INVALID_ARG
     dp.close()
+
+
+@pytest.mark.parametrize("direct", ["1", "0"])
+def test_prefix_only_layout_single_level(direct, monkeypatch):
+    """A plain two-level layout without suffix storage: the prefix pass is the whole step and (direct = 1) writes the
+    final output itself, or (direct = 0) one part per row that the merge turns into the output."""
+    from paper_2601_05475_b200.harness import DeviceProblem
+    monkeypatch.setenv("MC_PREFIX_DIRECT", direct)
+    monkeypatch.setenv("MC_PREFIX_PART_TOKENS", "4096")      # one split: one part per row
+    cfg = wl.Config("ponly", "bf16", 3, 5, 16, 4, 128, ("loguniform", 1, 700), ("fixed", (0,)), permute_pages=True, seed=31)
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    d = dp.desc
+    d.max_suffix_pages, d.suffix_pages, d.suffix_len = 0, 0, 0
+    layout = mc.mc_kv_layout_create(d)
+    geom = mc.mc_kv_layout_geometry(layout)
+    assert geom.n_parts == geom.n_prefix_parts == 1 and geom.prefix_ctas > 0
+    q = wl.draw_q(cfg, 0)
+    o = torch.full((cfg.B, cfg.Hq, cfg.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((cfg.B, cfg.Hq), float("nan"), dtype=torch.float32, device="cuda")
+    launches = mc.mc_launch_count()
+    mc.mc_decode_attn(layout, to_device(cfg, q), cfg.scale, o, lse, dp.ws_ptr, dp.ws_bytes)
+    torch.cuda.synchronize()
+    assert mc.mc_launch_count() - launches == (1 if direct == "1" else 2)
+    assert mc.mc_get_last_status(layout) == mc.MC_OK
+    o_ref, lse_ref = orc.decode_attention(q, hp.k_prefix, hp.v_prefix, hp.k_suffix, hp.v_suffix,
+                                          hp.tables.group_offsets.tolist(), cfg.scale)
+    err = np.abs(o.float().cpu().numpy().astype(np.float64) - o_ref)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+    assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    mc.mc_kv_layout_destroy(layout)
+    dp.close()
