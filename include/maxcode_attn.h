@@ -183,7 +183,9 @@ mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const floa
                          void *o, float *lse, void *stream);
 
 /* The whole step: prefix pass, suffix pass, merge.  `ws` is device memory of at least
- * mc_workspace_bytes(layout) bytes, 256-byte aligned (else MC_ERR_WORKSPACE_TOO_SMALL / INVALID_ARG). */
+ * mc_workspace_bytes(layout) bytes, 256-byte aligned (else MC_ERR_WORKSPACE_TOO_SMALL / INVALID_ARG).
+ * On a layout without suffix storage (max_suffix_pages = 0) whose prefix pass yields one part per row (one
+ * unsplit level, or two nested unsplit levels), the prefix pass writes o and lse itself: one launch, `ws` unused. */
 mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale,
                            void *o, float *lse, void *ws, size_t ws_bytes, void *stream);
 
