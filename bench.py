@@ -381,11 +381,13 @@ def run_gpu(args):
         torch.cuda.synchronize()
         reps = 10
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = mc.mc_launch_count()
         e0.record()
         for _ in range(reps):
             dp.score(q, stream)
         e1.record()
         torch.cuda.synchronize()
+        launches = (mc.mc_launch_count() - launches) // reps
         ms = e0.elapsed_time(e1) / reps
         ok = mc.mc_get_last_status(dp.layout) == mc.MC_OK
         seen = sum(n * 4096 + n * (n + 1) // 2 for n in seq_len)               # (query, key) pairs that are not masked
@@ -394,7 +396,7 @@ def run_gpu(args):
         dp.close()
         return {"sequences": scfg.B, "tokens_per_sequence": 512, "prompt_tokens": 4096, "queries": nv, "ms": round(ms, 4),
                 "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "flops": flops, "prefix_ctas": ctas, "n_parts": n_parts,
-                "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
+                "launches_per_pass": int(launches), "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
 
     if args.scoring_only:      # profiling aid: only the scoring pass, one small JSON line
         if rank == 0:
