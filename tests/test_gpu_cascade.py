@@ -83,3 +83,45 @@ def test_cascade_rejects_bad_level_descriptions():
     assert mc.lib().mc_kv_layout_create_cascade(mc.byref(dp.desc), arr, 4, mc.byref(h)) == mc.MC_ERR_INVALID_ARG
     assert mc.lib().mc_kv_layout_create_cascade(mc.byref(dp.desc), None, 1, mc.byref(h)) == mc.MC_ERR_INVALID_ARG
     dp.close()
+
+
+@pytest.mark.parametrize("chain", ["1", "0"])
+def test_row_limits_on_the_coarser_level(chain, monkeypatch):
+    """An outer level whose candidates see only a per-candidate number of its tokens, in front of unsplit base
+    prefixes with the same group boundaries: the two levels run chained (one item per row tile, the limit applied to
+    the coarser level's token range) or apart; every row is the plain attention over what it may see."""
+    monkeypatch.setenv("MC_PREFIX_CHAIN", chain)
+    monkeypatch.setenv("MC_PREFIX_PART_TOKENS", "4096")      # one split per level
+    cfg = wl.Config("casl", "bf16", 2, 4, 16, 4, 128, ("fixed", 129), ("uniform", 0, 40), seed=19)
+    hp = wl.make_host_problem(cfg)
+    wl.add_outer_level(hp, [0, 4, 8], [200, 260], 0)
+    dp = DeviceProblem.from_host(hp)
+    limit = np.array([10, 10, 150, 200, 0, 33, 260, 300], dtype=np.int32)     # non-decreasing inside a group
+    limit_dev = torch.from_numpy(limit).cuda()
+    go, ln, pg = dp.outer_tensors[0]
+    lv = mc.PrefixLevel()
+    lv.num_groups, lv.max_pages = 2, pg.shape[1]
+    lv.group_offsets, lv.len, lv.pages, lv.row_limit = go.data_ptr(), ln.data_ptr(), pg.data_ptr(), limit_dev.data_ptr()
+    layout = mc.mc_kv_layout_create_cascade(dp.desc, [lv])
+    geom = mc.mc_kv_layout_geometry(layout)
+    assert geom.n_prefix_parts == 2 and geom.prefix_ctas > 0
+    ws = torch.empty(mc.mc_workspace_bytes(layout) + 256, dtype=torch.uint8, device="cuda")
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    q = wl.draw_q(cfg, 0)
+    mc.mc_decode_attn(layout, to_device(cfg, q), cfg.scale, dp.o, dp.lse, ws_ptr, mc.mc_workspace_bytes(layout))
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(layout) == mc.MC_OK
+    g = cfg.Hq // cfg.Hkv
+    o_ref = np.zeros((cfg.B, cfg.Hq, cfg.d))
+    lse_ref = np.zeros((cfg.B, cfg.Hq))
+    for b in range(cfg.B):
+        j = b // cfg.C
+        n = min(int(limit[b]), hp.outer[0].k[j].shape[0])
+        for hq in range(cfg.Hq):
+            h = hq // g
+            K = np.concatenate([hp.outer[0].k[j][:n, h], hp.k_prefix[j][:, h], hp.k_suffix[b][:, h]], axis=0)
+            V = np.concatenate([hp.outer[0].v[j][:n, h], hp.v_prefix[j][:, h], hp.v_suffix[b][:, h]], axis=0)
+            o_ref[b, hq], lse_ref[b, hq] = orc.attend(q[b, hq], K, V, cfg.scale)
+    check(cfg, dp.o, dp.lse, o_ref, lse_ref)
+    mc.mc_kv_layout_destroy(layout)
+    dp.close()
