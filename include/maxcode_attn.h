@@ -172,7 +172,8 @@ mc_status_t mc_prefix_attn(mc_kv_layout_t *layout, const void *q, float scale,
                            float *o_part, float *lse_part, void *stream);
 
 /* Suffix pass: every candidate attends to its private suffix, chunk by chunk; writes parts
- * [n_prefix_parts, n_parts) of every row. */
+ * [n_prefix_parts, n_parts) of every row.  On a layout without suffix storage (max_suffix_pages = 0) there are
+ * no such parts and the call launches nothing. */
 mc_status_t mc_suffix_attn(mc_kv_layout_t *layout, const void *q, float scale,
                            float *o_part, float *lse_part, void *stream);
 
