@@ -10,6 +10,7 @@ K/V + Q + O (+LSE) bytes of a step divided by its device time, in GB/s.  Prints 
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -29,17 +30,19 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of the dominant kernel relative to its algorithmic bytes, from the ncu capture summarised in
-# profiles/kernels_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch on cfg2; the traffic
-# grows in proportion to the tokens streamed, so it is scaled by the units of the timed workload).  The ratio
-# is only reported while the kernel source still has the hash it had when the counters were taken.
-SUFFIX_TRAFFIC_RATIO = 1.0145
-SUFFIX_KERNEL_SHA1 = "2ab0fcfbe70b0b84062a61c9673256b55cce990d"
+# DRAM traffic of the dominant kernel relative to its algorithmic bytes (dram__bytes_read.sum +
+# dram__bytes_write.sum per launch, one ncu capture per regime: chunks of a few hundred tokens as on cfg2, and
+# 4096-token chunks on a small problem of cfg4's shape; the traffic grows in proportion to the tokens streamed,
+# so the ratio is scaled by the units of the timed workload).  A ratio is only reported while the kernel source
+# still has the hash it had when the counters were taken.
+SUFFIX_TRAFFIC_RATIO = {"short_chunks": None, "long_chunks": None}
+SUFFIX_KERNEL_SHA1 = ""
 
 
-def suffix_traffic(algorithmic_bytes):
+def suffix_traffic(algorithmic_bytes, suffix_part_tokens):
     import hashlib
-    if SUFFIX_TRAFFIC_RATIO is None:
+    ratio = SUFFIX_TRAFFIC_RATIO["long_chunks" if suffix_part_tokens >= 2048 else "short_chunks"]
+    if ratio is None:
         return None
     src = os.path.join(ROOT, "paper_2601_05475_b200", "csrc", "mc_suffix_tma.cu")
     try:
@@ -47,7 +50,7 @@ def suffix_traffic(algorithmic_bytes):
             return None
     except OSError:
         return None
-    return algorithmic_bytes * SUFFIX_TRAFFIC_RATIO
+    return algorithmic_bytes * ratio
 
 
 def measured_peaks():
@@ -160,6 +163,44 @@ def aggregate_value(bytes_per_replica_step, ms_per_step, world):
     return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def spawn_replicas(n: int, argv, extra_env=None, script=None) -> int:
+    """`bench.py --gpus N` started as ONE process: starts N workers of this same script (or of `script`), one per
+    GPU, with the environment a torchrun launch would give them (rank 0 prints the line); returns the first
+    non-zero exit code."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen([sys.executable, script or os.path.abspath(__file__)] + list(argv), env=env))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
+
+
+def timed_blocks(run_block, sync, steps, min_seconds, max_blocks):
+    """Runs `run_block(block_index)` (which enqueues `steps` steps between two events and returns them) until
+    `min_seconds` of device time have been timed or `max_blocks` blocks have run; returns the per-block
+    milliseconds.  `sync` is the barrier + device synchronisation on both sides of every block."""
+    ms = []
+    while len(ms) < max_blocks and (not ms or sum(ms) * 1e-3 < min_seconds):
+        sync()
+        e0, e1 = run_block(len(ms))
+        sync()
+        ms.append(e0.elapsed_time(e1))
+    return ms
+
+
 # ---------------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------------
@@ -229,10 +270,21 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def measure(name, steps, warmup, want_kernel_split, outer=()):
+    def agree_seconds(x):
+        # every rank must run the same number of blocks (each block has a barrier): the ranks time different
+        # things, so the target is turned into "never stop on time" for N > 1 and the block cap decides
+        return x if world == 1 else (1e9 if x > 0 else 0.0)
+
+    def measure(name, steps, warmup, want_kernel_split, outer=(), min_seconds=0.0, max_timed_steps=None):
+        """Blocks of `steps` steps, each between a barrier + synchronize and timed with two events on the launching
+        stream, repeated until `min_seconds` have been timed (at most `max_timed_steps` steps in all, so that the
+        appends do not move the workload away from the configuration); the step time is the median block's."""
         cfg = wl.CONFIGS[name]
         appends = cfg.append_steps > 0
-        total_steps = 2 * (steps + warmup) + 8
+        if max_timed_steps is None:
+            max_timed_steps = 640 if appends else 4000
+        max_blocks = max(1, max_timed_steps // steps)
+        total_steps = warmup + max_blocks * steps + 16
         dp = make_device_problem(cfg, headroom_tokens=total_steps + 1 if appends else 1, outer=outer)
         stream = torch.cuda.current_stream().cuda_stream
         qs = [device_q(cfg, i) for i in range(4)]
@@ -251,26 +303,46 @@ def run_gpu(args):
             step(i)
         barrier()
         sampler = ClockSampler(torch.cuda.current_device())
-        if rank == 0:
+        if rank == 0 and min_seconds > 0:
             sampler.start()
         n0 = mc.mc_launch_count()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        for i in range(steps):
-            step(warmup + i)
-        ev1.record()
-        barrier()
-        launches = mc.mc_launch_count() - n0
-        clocks = sampler.stop() if rank == 0 else None
-        ms = ev0.elapsed_time(ev1) / steps
+
+        def run_block(blk):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                step(warmup + blk * steps + i)
+            e1.record()
+            return e0, e1
+
+        block_ms = timed_blocks(run_block, barrier, steps, agree_seconds(min_seconds), max_blocks)
+        launches = (mc.mc_launch_count() - n0) // len(block_ms)
+        clocks = sampler.stop() if (rank == 0 and min_seconds > 0) else None
         if mc.mc_get_last_status(dp.layout) != mc.MC_OK:
             raise RuntimeError("device status word reports an error")
-        # bytes of the average timed step (suffixes grow by one token per step when appending)
-        grow = (warmup + (steps + 1) / 2.0) * cfg.B * per_tok if appends else 0.0
+        # the median block (lower median: a block that was really run) and the bytes of ITS average step (suffixes
+        # grow by one token per step when appending)
+        order = sorted(range(len(block_ms)), key=lambda i: block_ms[i])
+        mid = order[(len(order) - 1) // 2]
+        ms = block_ms[mid] / steps
+        grow = (warmup + mid * steps + (steps + 1) / 2.0) * cfg.B * per_tok if appends else 0.0
         step_bytes = ub0["total"] + grow + (2 * cfg.B * cfg.Hkv * cfg.d * cfg.elem_bytes if appends else 0)
         res = {"ms": ms, "bytes": step_bytes, "launches": launches, "clocks": clocks, "cfg": cfg,
+               "blocks": len(block_ms), "block_ms_min": min(block_ms) / steps, "block_ms_max": max(block_ms) / steps,
                "prefix_ctas": int(dp.geom.prefix_ctas), "n_parts": int(dp.geom.n_parts),
-               "n_prefix_parts": int(dp.geom.n_prefix_parts)}
+               "n_prefix_parts": int(dp.geom.n_prefix_parts), "suffix_part_tokens": int(dp.geom.suffix_part_tokens)}
+
+        # what making the layout object costs on the host (it reads lengths back, plans both passes, encodes the
+        # tensor maps and allocates its small device state): median of five create / destroy pairs
+        if not outer:
+            t_create = []
+            for _ in range(5):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                h = mc.mc_kv_layout_create(dp.desc)
+                t_create.append((time.perf_counter() - t0) * 1e3)
+                mc.mc_kv_layout_destroy(h)
+            res["layout_create_ms"] = statistics.median(t_create)
 
         # end to end through the host-buffer entry point: pinned host q / k_new / v_new in, o / lse out
         pin = lambda t: t.cpu().pin_memory()
@@ -325,6 +397,60 @@ def run_gpu(args):
         del dp
         torch.cuda.empty_cache()
         return res
+
+    def measure_prefix_cold(name, steps, warmup, copies=6):
+        """The same step with the shared prefix NOT left in L2 by the step before: `copies` independent instances of
+        the configuration (own pools, own tables) take turns, so that between two steps on one instance the others
+        have streamed several times the L2 capacity, their own evict-last prefix lines included - what a decode
+        loop over the layers of a model does to one layer's prefix.  No appends (the lengths stay at step 0)."""
+        cfg = wl.CONFIGS[name]
+        dps = [make_device_problem(dataclasses.replace(cfg, seed=cfg.seed + 31 * c), headroom_tokens=1)
+               for c in range(copies)]
+        stream = torch.cuda.current_stream().cuda_stream
+        qs = [device_q(cfg, i) for i in range(4)]
+        per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+        total = sum(wl.unique_bytes(cfg, dp.prefix_len.cpu().numpy(), dp.suffix_len.cpu().numpy())["total"] for dp in dps)
+
+        def step(i):
+            dp = dps[i % copies]
+            mc.mc_decode_step(dp.layout, None, None, qs[i % 4], cfg.scale, dp.o, dp.lse, dp.ws_ptr, dp.ws_bytes, stream)
+
+        for i in range(max(warmup, copies)):
+            step(i)
+        barrier()
+        n = (steps + copies - 1) // copies * copies          # every instance equally often
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            step(i)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / n
+        for dp in dps:
+            dp.close()
+        del dps
+        torch.cuda.empty_cache()
+        return {"ms_per_step": ms, "gbs": total / copies / (ms * 1e-3) / 1e9, "instances": copies}
+
+    def measure_read_peak():
+        """Read-only streaming rate of this GPU: the library's probe kernel over 4 GiB (33 x L2), best of 5."""
+        n = 4 << 30
+        buf = torch.empty(n, dtype=torch.uint8, device="cuda")
+        buf.zero_()
+        sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+        stream = torch.cuda.current_stream().cuda_stream
+        best = 0.0
+        for i in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            mc.mc_hbm_read_probe(buf, n, sink, stream)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+        del buf
+        torch.cuda.empty_cache()
+        return best
 
     def measure_search():
         """The search bookkeeping on 2^17 problems x 8 trajectories x 8 steps (Section 3.1: K = 8, depth 8): one pass
@@ -398,22 +524,53 @@ def run_gpu(args):
                 "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "flops": flops, "prefix_ctas": ctas, "n_parts": n_parts,
                 "launches_per_pass": int(launches), "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
 
+    if args.pass_only:         # profiling aid: one pass alone on the launching stream, one small JSON line
+        cfg = wl.CONFIGS[args.workload]
+        dp = make_device_problem(cfg, headroom_tokens=1)
+        g = dp.geom
+        lse_off = (g.rows * g.n_parts * g.head_dim * 4 + 255) // 256 * 256
+        fn = {"suffix": mc.mc_suffix_attn, "prefix": mc.mc_prefix_attn}[args.pass_only]
+        q, stream = device_q(cfg, 0), torch.cuda.current_stream().cuda_stream
+        for _ in range(args.warmup):
+            fn(dp.layout, q, cfg.scale, dp.ws_ptr, dp.ws_ptr + lse_off, stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn(dp.layout, q, cfg.scale, dp.ws_ptr, dp.ws_ptr + lse_off, stream)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        tokens = float((dp.suffix_len if args.pass_only == "suffix" else dp.prefix_len).sum().item())
+        nbytes = tokens * 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+        ok = mc.mc_get_last_status(dp.layout) == mc.MC_OK
+        if rank == 0:
+            print(json.dumps({"pass": args.pass_only, "workload": cfg.name, "ms": ms, "algorithmic_bytes": nbytes,
+                              "gbs": nbytes / (ms * 1e-3) / 1e9, "suffix_part_tokens": int(g.suffix_part_tokens),
+                              "n_parts": int(g.n_parts), "prefix_ctas": int(g.prefix_ctas), "status_ok": ok,
+                              "forced_alu": os.environ.get("MC_FORCE_FMA", "0") not in ("", "0")}))
+        dp.close()
+        return 0
+
     if args.scoring_only:      # profiling aid: only the scoring pass, one small JSON line
         if rank == 0:
             print(json.dumps({"scoring_attention": measure_scoring()}))
         return 0
 
-    main = measure(args.workload, args.steps, args.warmup, True)
+    main = measure(args.workload, args.steps, args.warmup, True, min_seconds=1.0)
     others = {}
+    cold = None
     if args.all_configs:
         for name in ("cfg2", "cfg3", "cfg4"):
             if name != args.workload:
                 others[name] = measure(name, args.steps, args.warmup, True)
+        cold = measure_prefix_cold("cfg2", max(args.steps, 60), args.warmup)
         # a cascade deeper than two levels: configuration 3 behind a 4096-token prompt shared by all 256 candidates
         c3 = wl.CONFIGS["cfg3"]
         others["cfg3+root4096"] = measure("cfg3", args.steps, args.warmup, True, outer=[([0, c3.B], [4096])])
 
     search = measure_search() if args.all_configs else None
+    read_peak = measure_read_peak() if args.all_configs else None
 
     scoring = measure_scoring() if args.all_configs else None
 
@@ -441,6 +598,8 @@ def run_gpu(args):
             gbs = r["bytes"] / (r["ms"] * 1e-3) / 1e9
             out = {"gbs": round(gbs, 1), "frac_of_8tbs": round(gbs / NOMINAL_HBM_GBS, 4), "ms_per_step": round(r["ms"], 5),
                    "candidate_tokens_per_s": round(r["cfg"].B / (r["ms"] * 1e-3), 1)}
+            if "layout_create_ms" in r:
+                out["layout_create_ms"] = round(r["layout_create_ms"], 3)
             if "suffix_ms" in r:
                 out["suffix_ms"] = round(r["suffix_ms"], 5)
                 out["suffix_gbs"] = round(r["suffix_bytes"] / (r["suffix_ms"] * 1e-3) / 1e9, 1)
@@ -455,6 +614,14 @@ def run_gpu(args):
             cpu_value = sample_bytes / times[0] / 1e9
         else:
             n_rows, cores, cpu_value = 0, 0, None
+        per_config = {**{cfg.name: summary(main)}, **{k: summary(v) for k, v in others.items()}}
+        if cold and "cfg2" in per_config:
+            # two readings of configuration 2: `frac_of_8tbs` with the 33.6 MB prefix still in L2 from the step before
+            # (consecutive steps on ONE layout, as the configuration is worded), and this one with the prefix coming
+            # from HBM at every step (instances taking turns)
+            per_config["cfg2"]["frac_of_8tbs_prefix_cold"] = round(cold["gbs"] / NOMINAL_HBM_GBS, 4)
+            per_config["cfg2"]["ms_per_step_prefix_cold"] = round(cold["ms_per_step"], 5)
+            per_config["cfg2"]["prefix_cold_instances"] = cold["instances"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -468,8 +635,13 @@ def run_gpu(args):
             "candidate_tokens_per_s": world * cfg.B / (ms * 1e-3),
             "roofline": {"bound": "hbm", "kernel": "suffix_tma_kernel", "achieved": suffix_gbs, "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": suffix_gbs / peak,
-                         "frac_of_8tbs": suffix_gbs / NOMINAL_HBM_GBS, "traffic": suffix_traffic(main["suffix_bytes"]),
-                         "kernel_ms": main["suffix_ms"], "algorithmic_bytes": main["suffix_bytes"]},
+                         "frac_of_8tbs": suffix_gbs / NOMINAL_HBM_GBS,
+                         "traffic": suffix_traffic(main["suffix_bytes"], main["suffix_part_tokens"]),
+                         "kernel_ms": main["suffix_ms"], "algorithmic_bytes": main["suffix_bytes"],
+                         # the measured peak is a copy (reads + writes); this kernel only reads: the read-only
+                         # streaming rate of the library's probe kernel on this GPU, in this run, and the fraction of it
+                         "read_only_peak": read_peak,
+                         "frac_of_read_only_peak": (suffix_gbs / read_peak) if read_peak else None},
             "prefix_pass": prefix_summary(main, peaks),
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": "%d of %d (candidate, head) rows of %s, fp64 numpy, one thread per row"
@@ -478,7 +650,9 @@ def run_gpu(args):
                     "h2d_bytes_per_step": main["h2d"], "d2h_bytes_per_step": main["d2h"], "ms_per_step": e2e_ms},
             "gpu_launches": int(main["launches"]),
             "clocks": main["clocks"],
-            "per_config": {**{cfg.name: summary(main)}, **{k: summary(v) for k, v in others.items()}},
+            "timed": {"blocks": main["blocks"], "steps_per_block": args.steps, "ms_per_step_is": "median block",
+                      "ms_per_step_min_block": main["block_ms_min"], "ms_per_step_max_block": main["block_ms_max"]},
+            "per_config": per_config,
             "search_bookkeeping": (dict(search, frac_of_measured_hbm=round(search["gbs"] / peak, 4)) if search else None),
             "scoring_attention": (dict(scoring, bound="tensor", frac_of_measured_bf16=(
                 round(scoring["tflops"] / peaks["bf16_tflops"], 4) if peaks.get("bf16_tflops") else None)) if scoring else None),
@@ -499,10 +673,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false",
                     help="skip the CPU-oracle leg (profiling runs only; the default run reports it)")
     ap.add_argument("--scoring-only", action="store_true", help="run only the scoring pass (profiling aid)")
+    ap.add_argument("--pass-only", choices=["suffix", "prefix"], default=None,
+                    help="run only that pass of --workload, alone (profiling aid)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
                     help="time only --workload (default: also cfg2/cfg3/cfg4 summaries under per_config)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as one process: become the launcher of N replicas (one per GPU), as a torchrun launch would
+        return spawn_replicas(args.gpus, sys.argv[1:])
     if args.impl == "reference":
         return run_reference(args)
     return run_gpu(args)

@@ -224,7 +224,10 @@ mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, 
  *     (about 8 prefix splits and 16 suffix chunks, 256..4096 tokens); otherwise MC_ERR_WORKSPACE_TOO_SMALL and nothing
  *     is launched.  (Configuration 1 needs about 1.7 MiB; the large benchmark configurations do not fit.)
  *   - The first call on each device looks up the scratch array's device address (the device must be
- *     current); make that first call outside any stream capture.
+ *     current).  With CUDA's lazy module loading that look-up is also the moment the driver loads the module
+ *     holding the array and sets its 16 MiB aside on that device.  So make one call per device at start-up,
+ *     while memory is still to be had and outside any stream capture; if the device cannot spare the
+ *     16 MiB any more, that first call returns MC_ERR_CUDA.  Later calls reserve nothing.
  *   - All calls share the one array and it keeps the previous call's contents (the call clears the status
  *     word it uses; every part slot is rewritten).  Two calls whose kernels overlap on the GPU - different
  *     streams, or different threads - race on it: serialise them.
@@ -237,6 +240,13 @@ size_t mc_static_scratch_bytes(void);
 
 /* Reads and clears the device status word (synchronises `stream`): MC_OK, or the first latched error. */
 mc_status_t mc_get_last_status(mc_kv_layout_t *layout, void *stream);
+
+/* (No counterpart in the paper: a measurement aid.)  Streams `bytes` bytes of DEVICE memory at `buf` (16-byte
+ * aligned) through the SMs once with 16-byte read-only loads and stores nothing but, possibly, one word at `sink`
+ * (device uint32).  Timed on a buffer several times the L2 size it gives the read-only HBM rate a streaming kernel
+ * can reach on this GPU, the ceiling of the suffix pass; a copy-based figure counts reads and writes.
+ * Asynchronous on `stream`. */
+mc_status_t mc_hbm_read_probe(const void *buf, size_t bytes, uint32_t *sink, void *stream);
 
 /* Kernel launches issued by this library since it was loaded (all handles, all threads). */
 uint64_t mc_launch_count(void);

@@ -55,6 +55,7 @@ EXPORTS = {
     "mc_decode_attn_static": (c_int32, [POINTER(LayoutDesc), c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
     "mc_static_scratch_bytes": (c_size_t, []),
     "mc_get_last_status": (c_int32, [c_void_p, c_void_p]),
+    "mc_hbm_read_probe": (c_int32, [c_void_p, c_size_t, c_void_p, c_void_p]),
     "mc_launch_count": (c_uint64, []),
     "mc_status_string": (c_char_p, [c_int32]),
     "mc_search_returns": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_float, c_float, c_float, c_float,
@@ -189,6 +190,10 @@ def mc_decode_attn_static(desc: LayoutDesc, q, scale: float, o, lse, dev_status=
 
 def mc_static_scratch_bytes() -> int:
     return int(lib().mc_static_scratch_bytes())
+
+
+def mc_hbm_read_probe(buf, nbytes: int, sink, stream: int = 0) -> None:
+    _check(lib().mc_hbm_read_probe(_ptr(buf), nbytes, _ptr(sink), stream), "mc_hbm_read_probe")
 
 
 def mc_get_last_status(layout: int, stream: int = 0) -> int:

@@ -85,6 +85,9 @@ struct Layout;  // the opaque handle
 
 void count_launch();
 mc_status_t check_launch();
+// Limit, in SM clock cycles, of every bounded device-side wait of kernels planned from now on: about one second,
+// or MC_WAIT_CYCLES from the environment (tests shorten it to see a wait run out).
+long long wait_limit_cycles();
 
 // launchers (each enqueues on `stream` and returns the launch status)
 mc_status_t launch_fma(const Params &p, int dtype, int mode, const void *q, float scale, float *o_part,

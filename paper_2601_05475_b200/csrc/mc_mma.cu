@@ -143,9 +143,9 @@ __device__ __forceinline__ void compute_page(State &st, const PageRegs &r, const
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kWarps * 32, 2)
-attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
-                float *__restrict__ lse_part, int prefetch_pages) {
+__device__ __forceinline__ void
+attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
+              float *__restrict__ lse_part, int prefetch_pages) {
   constexpr bool STREAM = MODE == kSuffix;  // private suffix data is read exactly once
   const int lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
   const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
@@ -282,6 +282,18 @@ attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float 
       }
     }
   }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kWarps * 32, 2)
+attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
+                float *__restrict__ lse_part, int prefetch_pages) {
+  attn_mma_body<MODE>(p, q, sl2, o_part, lse_part, prefetch_pages);
+  // As the programmatic dependent of the prefix pass the suffix grid starts before that one ends; one thread of the
+  // grid waits for the prerequisite grid before it exits, so that this grid - and the merge behind it - cannot
+  // complete earlier.  Without a prerequisite the instruction returns at once.
+  if (MODE == kSuffix && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 }  // namespace

@@ -46,7 +46,7 @@ constexpr uint32_t kTileBytes = 2 * kHalfBytes;         // 32 KB
 constexpr uint32_t kPageBytes = kPage * D * 2;          // one (page, kv head) slab; one TMA box for V
 constexpr uint32_t kTmemCols = 512;                     // team T: S at 256 T, O at 256 T + 128; P (bf16 pairs) over S:
                                                         // the thread that owns S columns [64 h, 64 h + 64) writes [64 h, 64 h + 32)
-constexpr long long kWaitCycles = 2000000000ll;         // ~1 s
+constexpr long long kDrainCycles = 2000000ll;           // ~1 ms: what an aborting CTA grants its copies and products in flight
 
 struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint8_t q[2][kTileBytes];           // stacked query tile of the current and of the next item
@@ -59,6 +59,7 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
   uint32_t tmem_base;
   volatile int abort;
+  long long wait_cycles;              // limit of every wait of this CTA
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -90,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(Smem &sm, const Params &p, uint64_t *b
     if (mbar_try_wait(bar, parity)) return true;
     __nanosleep(32);   // a polling warp must not take issue slots from the softmax warps of its scheduler
     if (sm.abort) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > sm.wait_cycles) {
       sm.abort = 1;
       latch(p, kDevTimeout);
       return false;
@@ -314,7 +315,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
                  float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
                  const int32_t *__restrict__ cta_begin, __nv_bfloat16 *__restrict__ o_final,
-                 float *__restrict__ lse_final) {
+                 float *__restrict__ lse_final, long long wait_cycles) {
   // o_final != null: every row gets exactly one part from this launch and none from anywhere else, so the item
   // writes the row's final output (bf16) and log-sum-exp itself and no merge follows.
   const bool direct = o_final != nullptr;
@@ -352,6 +353,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       mbar_init(&sm.pv_done[t], 1);
     }
     sm.abort = 0;
+    sm.wait_cycles = wait_cycles;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 1) {
@@ -826,7 +828,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   if (sm.abort && warp == 0 && lane == 0) {
     // give copies that are still in flight a bounded time to land before the CTA's shared memory goes away
     const long long t0 = clock64();
-    while (clock64() - t0 < 2000000ll) { }
+    while (clock64() - t0 < kDrainCycles) { }
   }
   tc_fence_before();
   __syncthreads();
@@ -897,6 +899,7 @@ struct PrefixTcPlan {
   TcLevels levels;
   int n_items, grid;
   bool one_part_per_row;   // every row gets exactly one part from this pass: one single-split level, or two chained
+  long long wait_cycles;   // limit of every device-side wait
   int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
@@ -947,6 +950,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   if (n_levels < 1 || n_levels > kMaxTcLevels) return nullptr;
   PrefixTcPlan *plan = new PrefixTcPlan();
   plan->dev_lists = nullptr;
+  plan->wait_cycles = wait_limit_cycles();
   const Params &p = levels[0];
   if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
       !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true)) {
@@ -1112,7 +1116,8 @@ mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const vo
                              float *lse_part, cudaStream_t stream, void *o_final, float *lse_final) {
   prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
       p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part,
-      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final);
+      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final,
+      plan->wait_cycles);
   count_launch();
   return check_launch();
 }

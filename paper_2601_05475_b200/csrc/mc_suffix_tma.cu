@@ -28,7 +28,7 @@ constexpr int kW = 2;                      // warps (items) per CTA
 constexpr int kStages = 4;                 // page stages per warp: two being computed, two in flight
 constexpr uint32_t kSlabBytes = kPage * D * 2;       // one (page, kv head) slab of K or of V
 constexpr uint32_t kStageBytes = 2 * kSlabBytes;
-constexpr long long kWaitCycles = 2000000000ll;      // ~1 s
+constexpr long long kDrainCycles = 2000000ll;        // ~1 ms: what a warp that gives up grants its copies in flight
 
 struct __align__(1024) Smem {
   uint8_t ring[kW][kStages][kStageBytes];   // [warp][stage][K slab | V slab], each slab [d half][16 tokens][64], swizzled
@@ -52,13 +52,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false once the limit has expired (MC_ERR_TIMEOUT is latched).
-__device__ __forceinline__ bool mbar_wait(const Params &p, uint64_t *bar, uint32_t parity) {
+// Bounded wait: false once `limit` cycles have passed (MC_ERR_TIMEOUT is latched).
+__device__ __forceinline__ bool mbar_wait(const Params &p, uint64_t *bar, uint32_t parity, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       latch(p, kDevTimeout);
       return false;
     }
@@ -112,10 +112,10 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(kW * 32)
-suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t k_off, uint32_t v_off,
-                  const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
-                  float *__restrict__ lse_part) {
+__device__ __forceinline__ void
+suffix_tma_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32_t v_off,
+                const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
+                float *__restrict__ lse_part, long long wait_cycles) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tig = lane & 3;
@@ -214,7 +214,8 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t
 #pragma unroll 1
   for (int o = 0; o < n_ord; o += 2) {
     const int s0 = o % kStages, s1 = (o + 1) % kStages;
-    alive = mbar_wait(p, &full[s0], (o / kStages) & 1) && mbar_wait(p, &full[s1], ((o + 1) / kStages) & 1);
+    alive = mbar_wait(p, &full[s0], (o / kStages) & 1, wait_cycles) &&
+            mbar_wait(p, &full[s1], ((o + 1) / kStages) & 1, wait_cycles);
     alive = __all_sync(0xffffffffu, alive);
     if (!alive) break;
     const uint32_t base0 = smem_u32(ring[s0]), base1 = smem_u32(ring[s1]);
@@ -313,7 +314,13 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t
       if (nb & 1) good1 = good_mask(nb, ids1); else good0 = good_mask(nb, ids0);
     }
   }
-  if (!alive) return;
+  if (!alive) {
+    // A wait ran out: the warp writes no result.  Copies into its ring may still be in flight; they get a bounded
+    // time to land before the warp leaves and the CTA's shared memory can go to another CTA.
+    const long long t0 = clock64();
+    while (clock64() - t0 < kDrainCycles) { }
+    return;
+  }
 
 #pragma unroll
   for (int sh = 4; sh <= 16; sh <<= 1) {
@@ -339,11 +346,25 @@ suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t
   }
 }
 
+__global__ void __launch_bounds__(kW * 32)
+suffix_tma_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t k_off, uint32_t v_off,
+                  const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
+                  float *__restrict__ lse_part, long long wait_cycles) {
+  suffix_tma_body(p, kv_map, k_off, v_off, q, sl2, o_part, lse_part, wait_cycles);
+  // Launched as the programmatic dependent of the prefix pass, this grid starts before that one ends.  The merge
+  // behind it needs both: one thread of the grid (in the CTA that is scheduled last) waits for the prerequisite
+  // grid to complete and its writes to be visible before it exits, so this grid cannot complete earlier.  Only
+  // that thread waits - a CTA that waited would keep its SM slot from the next CTA of the stream.  Launched the
+  // ordinary way there is no prerequisite and the instruction returns at once.
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
 }  // namespace
 
 struct SuffixTmaPlan {
   CUtensorMap kv_map;
   uint32_t k_off, v_off;   // where a stage holds the K slab and the V slab
+  long long wait_cycles;   // limit of every device-side wait
 };
 
 int suffix_tma_items_per_cta() { return kW; }
@@ -356,6 +377,7 @@ SuffixTmaPlan *suffix_tma_plan(const Params &p, int dtype) {
   const uintptr_t ka = reinterpret_cast<uintptr_t>(p.k_pool), va = reinterpret_cast<uintptr_t>(p.v_pool);
   plan->k_off = ka < va ? 0u : kSlabBytes;
   plan->v_off = ka < va ? kSlabBytes : 0u;
+  plan->wait_cycles = wait_limit_cycles();
   if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||
       !encode_kv_pair_map(&plan->kv_map, ka < va ? p.k_pool : p.v_pool, (unsigned long long)(ka < va ? va - ka : ka - va),
                           p.num_pages, p.Hkv) ||
@@ -385,7 +407,8 @@ mc_status_t launch_suffix_tma(const Params &p, const SuffixTmaPlan *plan, const 
   cfg.attrs = &attr;
   cfg.numAttrs = beside_previous ? 1 : 0;
   const cudaError_t e = cudaLaunchKernelEx(&cfg, suffix_tma_kernel, p, plan->kv_map, plan->k_off, plan->v_off,
-                                           reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part);
+                                           reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
+                                           plan->wait_cycles);
   count_launch();
   return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }

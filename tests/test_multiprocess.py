@@ -40,6 +40,37 @@ def test_two_gloo_ranks_agree_on_the_slowest_time():
         assert value == pytest.approx(2 * 3.0e9 / 2.5e-3 / 1e9)
 
 
+def test_launcher_starts_replicas(tmp_path):
+    """`bench.py --gpus 2` started as one process becomes the launcher: two workers with the ranks, the local ranks
+    and the rendezvous address of a torchrun launch; the line reports n_gpus = 2 and the aggregate of both."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    out = tmp_path / "line.json"
+    rc = bench.spawn_replicas(2, [str(out)], script=os.path.join(ROOT, "tests", "replica_worker.py"))
+    assert rc == 0
+    line = json.loads(out.read_text())
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 3.0
+    assert line["value"] == pytest.approx(2 * 4.0e9 / 3.0e-3 / 1e9)
+
+
+def test_timed_blocks_stop_on_time_or_on_the_cap():
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class Ev:
+        def __init__(self, t):
+            self.t = t
+
+        def elapsed_time(self, other):
+            return other.t - self.t
+    calls = []
+    run = lambda blk: (calls.append(blk), (Ev(0.0), Ev(300.0)))[1]          # every block takes 300 ms
+    assert bench.timed_blocks(run, lambda: None, 20, 1.0, 64) == [300.0] * 4  # 1.2 s >= 1 s after four blocks
+    assert bench.timed_blocks(run, lambda: None, 20, 1.0, 2) == [300.0] * 2   # the cap
+    assert bench.timed_blocks(run, lambda: None, 20, 0.0, 64) == [300.0]      # no target: one block
+
+
 def test_single_process_is_identity():
     sys.path.insert(0, ROOT)
     import bench
