@@ -10,7 +10,6 @@ K/V + Q + O (+LSE) bytes of a step divided by its device time, in GB/s.  Prints 
 from __future__ import annotations
 
 import argparse
-import dataclasses
 import json
 import os
 import statistics
@@ -404,8 +403,7 @@ def run_gpu(args):
         have streamed several times the L2 capacity, their own evict-last prefix lines included - what a decode
         loop over the layers of a model does to one layer's prefix.  No appends (the lengths stay at step 0)."""
         cfg = wl.CONFIGS[name]
-        dps = [make_device_problem(dataclasses.replace(cfg, seed=cfg.seed + 31 * c), headroom_tokens=1)
-               for c in range(copies)]
+        dps = [make_device_problem(cfg, headroom_tokens=1) for _ in range(copies)]      # same lengths, own memory
         stream = torch.cuda.current_stream().cuda_stream
         qs = [device_q(cfg, i) for i in range(4)]
         per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes

@@ -709,7 +709,10 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
                       : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
       if (s != MC_OK) return s;
     }
-    return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
+    // The merge is the suffix pass's programmatic dependent in turn (MC_PDL_MERGE=0: an ordinary launch): its CTAs
+    // are resident and waiting when the last suffix CTA ends, instead of being launched then.
+    return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st,
+                            L->has_suffix && L->sfx_plan && mc::env_int("MC_PDL_MERGE", 1));
   }
   // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix
   // pages and lengths) and the suffix pass on the handle's side stream; the merge joins them.

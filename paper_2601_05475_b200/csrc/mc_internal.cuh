@@ -97,7 +97,7 @@ mc_status_t launch_fma(const Params &p, int dtype, int mode, const void *q, floa
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
                        cudaStream_t stream, bool beside_previous = false);
 mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
-                         float *lse, cudaStream_t stream);
+                         float *lse, cudaStream_t stream, bool beside_previous = false);
 bool mma_supported(const Params &p, int dtype);
 int mma_items_per_cta();
 

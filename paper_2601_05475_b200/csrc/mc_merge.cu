@@ -38,6 +38,11 @@ merge_lse_kernel(int rows, int n_parts, const float *__restrict__ o_part, const 
   constexpr int VEC = D / 32;
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  // Launched as the programmatic dependent of the suffix pass, this grid's CTAs may become resident while that
+  // pass's last CTAs still run; nothing is read before the prerequisite grid has completed and its writes are
+  // visible (and through the suffix grid's own wait, the prefix pass's).  Launched the ordinary way, this
+  // returns at once.
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
   if (row >= rows) return;
   const float *lp = lse_part + (size_t)row * n_parts;
   float m = -INFINITY;
@@ -74,24 +79,33 @@ merge_lse_kernel(int rows, int n_parts, const float *__restrict__ o_part, const 
 
 template <typename T, int D>
 mc_status_t launch_t(const Params &p, const float *o_part, const float *lse_part, void *o, float *lse,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, bool beside_previous) {
   const int rows = p.B * p.Hq;
-  const unsigned grid = (unsigned)((rows + kWarpsPerBlock - 1) / kWarpsPerBlock);
-  merge_lse_kernel<T, D><<<grid, kWarpsPerBlock * 32, 0, stream>>>(rows, p.n_parts, o_part, lse_part, (T *)o, lse);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((rows + kWarpsPerBlock - 1) / kWarpsPerBlock));
+  cfg.blockDim = dim3(kWarpsPerBlock * 32);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = beside_previous ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, merge_lse_kernel<T, D>, rows, (int)p.n_parts, o_part, lse_part,
+                                           (T *)o, lse);
   count_launch();
-  return check_launch();
+  return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }
 
 }  // namespace
 
 mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const float *lse_part, void *o,
-                         float *lse, cudaStream_t stream) {
+                         float *lse, cudaStream_t stream, bool beside_previous) {
   if (dtype == MC_F32) {
-    if (p.d == 64) return launch_t<float, 64>(p, o_part, lse_part, o, lse, stream);
-    if (p.d == 128) return launch_t<float, 128>(p, o_part, lse_part, o, lse, stream);
+    if (p.d == 64) return launch_t<float, 64>(p, o_part, lse_part, o, lse, stream, beside_previous);
+    if (p.d == 128) return launch_t<float, 128>(p, o_part, lse_part, o, lse, stream, beside_previous);
   } else if (dtype == MC_BF16) {
-    if (p.d == 64) return launch_t<__nv_bfloat16, 64>(p, o_part, lse_part, o, lse, stream);
-    if (p.d == 128) return launch_t<__nv_bfloat16, 128>(p, o_part, lse_part, o, lse, stream);
+    if (p.d == 64) return launch_t<__nv_bfloat16, 64>(p, o_part, lse_part, o, lse, stream, beside_previous);
+    if (p.d == 128) return launch_t<__nv_bfloat16, 128>(p, o_part, lse_part, o, lse, stream, beside_previous);
   }
   return MC_ERR_UNSUPPORTED;
 }

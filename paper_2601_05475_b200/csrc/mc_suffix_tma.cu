@@ -128,6 +128,9 @@ suffix_tma_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   __syncthreads();
+  // A kernel launched behind this one as its programmatic dependent (the merge, which waits for this grid's
+  // completion before it reads anything) may take its place on the SMs once every CTA of this grid has started.
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
   const int n_chunks = p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * n_chunks;
