@@ -62,6 +62,9 @@ int env_int(const char *name, int dflt) {
 __global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__restrict__ k_new,
                                                      const uint4 *__restrict__ v_new, int32_t *suffix_len,
                                                      int elem_bytes) {
+  // The prefix pass, when it is launched behind this kernel as its programmatic dependent, reads nothing this
+  // kernel writes and may start at once; it holds back the suffix pass until this grid has completed.
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int b = blockIdx.x;
   const int s = suffix_len[b];
   const int pg = s >> 4;
@@ -703,7 +706,12 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
     // dependent, so it starts once every prefix CTA is running, not when they end.  The order holds when
     // the step is replayed from a captured graph.  The merge, launched the ordinary way, waits for both.
     if (k_new && (s = mc_kv_append(layout, k_new, v_new, st)) != MC_OK) return s;
-    if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st)) != MC_OK) return s;
+    // Behind an append of its own the prefix pass is launched as that kernel's programmatic dependent: it needs
+    // nothing of the append, so its start-up runs beside it; the suffix pass, which does, is released by the
+    // prefix CTAs only after they have seen the append grid complete (MC_PDL_APPEND=0: an ordinary launch).
+    const bool early = k_new != nullptr && mc::env_int("MC_PDL_APPEND", 1);
+    if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st, nullptr, nullptr, early)) != MC_OK)
+      return s;
     if (L->has_suffix) {
       s = L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
                       : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);

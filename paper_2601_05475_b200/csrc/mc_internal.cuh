@@ -112,7 +112,8 @@ int prefix_tc_grid(const PrefixTcPlan *plan);
 bool prefix_tc_shape_supported(const Params &p, int dtype);   // everything but the part geometry
 bool prefix_tc_one_part_per_row(const PrefixTcPlan *plan);
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
-                             float *lse_part, cudaStream_t stream, void *o_final = nullptr, float *lse_final = nullptr);
+                             float *lse_part, cudaStream_t stream, void *o_final = nullptr, float *lse_final = nullptr,
+                             bool beside_previous = false);
 
 
 // Tensor map over a paged pool [page][kv head][16 tokens][128] (bf16) for TMA copies with the 128-byte swizzle:

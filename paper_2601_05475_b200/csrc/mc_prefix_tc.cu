@@ -331,9 +331,6 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   const int k_begin = __ldg(cta_begin + blockIdx.x), k_end = __ldg(cta_begin + blockIdx.x + 1);
 
   if (threadIdx.x == 0) {
-    // This CTA holds its SM now: a kernel launched behind this one as its programmatic dependent (the suffix
-    // pass, which needs nothing this kernel writes) may start as soon as every CTA of this grid has said so.
-    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     for (int s = 0; s < kKSlots; ++s) {
       mbar_init(&sm.full_k[s], 2);   // one arrival per K d half
       mbar_init(&sm.empty_k[s], 1);
@@ -365,6 +362,16 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
+  if (threadIdx.x == kThreads - 1) {
+    // This CTA holds its SM now: a kernel launched behind this one as its programmatic dependent (the suffix
+    // pass, which needs nothing this kernel writes) may start as soon as every CTA of this grid has said so.
+    // When this grid was itself launched as the programmatic dependent of the append, the suffix pass needs what
+    // that kernel wrote: the word is given only once the append grid has completed (a short wait, taken by a
+    // thread of a copy-issuing warp whose lanes 8-31 have nothing else to do, while the CTA sets itself up).
+    // Launched the ordinary way the wait returns at once.
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  }
   // team T: S at columns [256 T, 256 T + 128), O at [256 T + 128, 256 T + 256)
 
   // Counters advance identically in every role: `kt` counts K/V tiles, `it_n` counts items with work.
@@ -1113,13 +1120,24 @@ bool prefix_tc_one_part_per_row(const PrefixTcPlan *plan) { return plan && plan-
 // o_final / lse_final non-null (only for a plan with one part per row, and only when no other pass adds parts): the
 // pass writes the final bf16 output and log-sum-exp of every row itself instead of partial results.
 mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const void *q, float scale, float *o_part,
-                             float *lse_part, cudaStream_t stream, void *o_final, float *lse_final) {
-  prefix_tc_kernel<<<plan->grid, kThreads, sizeof(Smem), stream>>>(
-      p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part,
-      lse_part, plan->dev_lists + plan->grid + 1, plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final,
-      plan->wait_cycles);
+                             float *lse_part, cudaStream_t stream, void *o_final, float *lse_final,
+                             bool beside_previous) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)plan->grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = sizeof(Smem);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = beside_previous ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(
+      &cfg, prefix_tc_kernel, p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q),
+      scale * kLog2e, o_part, lse_part, (const int32_t *)(plan->dev_lists + plan->grid + 1),
+      (const int32_t *)plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles);
   count_launch();
-  return check_launch();
+  return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }
 
 }  // namespace mc
