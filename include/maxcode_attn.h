@@ -64,7 +64,13 @@ typedef enum {
   MC_ERR_TIMEOUT = 6             /* a bounded device-side wait gave up */
 } mc_status_t;
 
-typedef enum { MC_F32 = 0, MC_BF16 = 1 } mc_dtype_t;
+/* MC_F32 / MC_BF16: the cache, q and o all have that type.  MC_FP8_E4M3: the cache holds 8-bit floating-point codes
+ * (E4M3 of Micikevicius et al., "FP8 Formats for Deep Learning": 1 sign, 4 exponent bits with bias 7, 3 mantissa
+ * bits, no infinities, largest magnitude 448) with one float scale per (page, kv head) for K and one for V - a code
+ * stands for decode(code) * scale - while q, o, k_new and v_new are bf16.  The paper takes the model and its cache as
+ * given; this halves the bytes per cached token (2 * Hkv * d instead of 4 * Hkv * d).  head_dim must be 128 and
+ * Hq / Hkv at most 8. */
+typedef enum { MC_F32 = 0, MC_BF16 = 1, MC_FP8_E4M3 = 2 } mc_dtype_t;
 
 typedef struct mc_kv_layout mc_kv_layout_t;   /* opaque, owned by the library */
 
@@ -87,6 +93,9 @@ typedef struct {
   const int32_t *prefix_len;     /* device, [G] */
   const int32_t *suffix_pages;   /* device, [B][max_suffix_pages] */
   int32_t *suffix_len;           /* device, [B]; mc_kv_append increments it */
+  float *k_scale, *v_scale;      /* device, [num_pages][Hkv] each; MC_FP8_E4M3 only (else ignored, may be NULL).  Read by
+                                    the attention passes; mc_kv_append writes the entry of a page when it writes the
+                                    page's first token */
 } mc_kv_layout_desc_t;
 
 typedef struct {
@@ -150,7 +159,12 @@ size_t mc_workspace_bytes(const mc_kv_layout_t *layout);
 
 /* Appends one token per candidate: writes k_new/v_new [B][Hkv][d] (device, `dtype`) into slot
  * suffix_len[b] % 16 of page suffix_pages[b][suffix_len[b] / 16], then increments suffix_len[b], all on
- * the device.  A candidate whose page row is full is left unchanged and MC_ERR_INVALID_ARG is latched. */
+ * the device.  A candidate whose page row is full is left unchanged and MC_ERR_INVALID_ARG is latched.
+ * MC_FP8_E4M3: k_new / v_new are bf16 and are quantised on the way in.  The token that opens a page (slot 0) fixes
+ * that page's scales, per kv head and for K and V separately: scale = (2 * max|row|) / 448 (1 for a row of zeros), so
+ * later rows up to twice as large still fit and larger values saturate at +-448 * scale; the other 15 tokens of the
+ * page use the stored scale.  code = e4m3(x / scale), the quotient rounded once in single precision, the conversion
+ * to the nearest code, ties to even.  The cache therefore does not depend on how tokens were grouped into calls. */
 mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *stream);
 
 /* mc_kv_append with rotary position embedding (the step of the language model's decode layer that precedes the

@@ -15,14 +15,14 @@ _lib = None
 
 MC_OK, MC_ERR_INVALID_ARG, MC_ERR_UNSUPPORTED, MC_ERR_OUT_OF_MEMORY, MC_ERR_WORKSPACE_TOO_SMALL, MC_ERR_CUDA, \
     MC_ERR_TIMEOUT = range(7)
-MC_F32, MC_BF16 = 0, 1
+MC_F32, MC_BF16, MC_FP8_E4M3 = 0, 1, 2
 
 
 class LayoutDesc(ctypes.Structure):
     _fields_ = [(n, c_int32) for n in ("num_groups", "batch", "num_q_heads", "num_kv_heads", "head_dim", "page_size",
                                        "num_pages", "max_prefix_pages", "max_suffix_pages", "dtype")] + \
                [(n, c_void_p) for n in ("k_pool", "v_pool", "group_offsets", "prefix_pages", "prefix_len",
-                                        "suffix_pages", "suffix_len")]
+                                        "suffix_pages", "suffix_len", "k_scale", "v_scale")]
 
 
 class PrefixLevel(ctypes.Structure):

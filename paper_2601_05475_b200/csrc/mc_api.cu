@@ -24,6 +24,8 @@ struct Layout {
   bool use_mma;
   bool has_suffix;            // false: no private tokens (max_suffix_pages = 0), the suffix pass is not launched
   SuffixTmaPlan *sfx_plan;    // non-null: the suffix pass runs on the TMA-fed kernel
+  Fp8Plan *fp8;               // non-null: e4m3 cache, both passes run on its kernel
+  int io_dtype;               // type of q and o: the cache's, or bf16 over an e4m3 cache
   PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
   Params outer_p[kMaxOuterLevels];
@@ -238,9 +240,10 @@ mc_status_t check_q(const Layout *L, const void *q) {
 mc_status_t run_level(Layout *L, const Params &p, int mode, const void *q, float scale, float *o_part,
                       float *lse_part, cudaStream_t st) {
   if (mode == kSuffix && !L->has_suffix) return MC_OK;
+  if (L->fp8) return launch_fp8(p, L->fp8, mode, q, scale, o_part, lse_part, st);
   if (mode == kSuffix && L->sfx_plan) return launch_suffix_tma(p, L->sfx_plan, q, scale, o_part, lse_part, st, false);
   if (L->use_mma) return launch_mma(p, mode, q, scale, o_part, lse_part, st);
-  return launch_fma(p, L->desc.dtype, mode, q, scale, o_part, lse_part, st);
+  return launch_fma(p, L->io_dtype, mode, q, scale, o_part, lse_part, st);
 }
 
 // The prefix pass covers every level of the cascade (outermost first), the suffix pass the private tokens.
@@ -359,14 +362,21 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
         !outer[k].group_offsets || !outer[k].pages || !outer[k].len)
       return MC_ERR_INVALID_ARG;
   if (d->page_size != mc::kPage) return MC_ERR_UNSUPPORTED;
-  if (d->dtype != MC_F32 && d->dtype != MC_BF16) return MC_ERR_UNSUPPORTED;
+  if (d->dtype != MC_F32 && d->dtype != MC_BF16 && d->dtype != MC_FP8_E4M3) return MC_ERR_UNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return MC_ERR_UNSUPPORTED;
   if ((long long)d->batch * d->num_q_heads > (1ll << 30)) return MC_ERR_UNSUPPORTED;
+  const bool fp8 = d->dtype == MC_FP8_E4M3;
+  if (fp8 && (!d->k_scale || !d->v_scale || (reinterpret_cast<uintptr_t>(d->k_scale) & 3u) ||
+              (reinterpret_cast<uintptr_t>(d->v_scale) & 3u)))
+    return MC_ERR_INVALID_ARG;
+  if (fp8 && (d->head_dim != 128 || d->num_q_heads / d->num_kv_heads > 8)) return MC_ERR_UNSUPPORTED;
 
   Layout *L = new (std::nothrow) Layout();
   if (!L) return MC_ERR_OUT_OF_MEMORY;
   L->desc = *d;
   L->n_outer = n_outer;
+  L->io_dtype = fp8 ? MC_BF16 : d->dtype;
+  L->fp8 = nullptr;
   mc::Params &p = L->p;
   p.k_pool = d->k_pool; p.v_pool = d->v_pool;
   p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
@@ -375,6 +385,8 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   p.g = d->num_q_heads / d->num_kv_heads;
   p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
   p.row_limit = nullptr;
+  p.k_scale = fp8 ? d->k_scale : nullptr;
+  p.v_scale = fp8 ? d->v_scale : nullptr;
   for (int k = 0; k < n_outer; ++k) {   // an outer level is the same cache seen through another group map
     mc::Params &po = L->outer_p[k];
     po = p;
@@ -399,7 +411,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     if (sl && max_s > 0 && cudaMemcpy(sl, d->suffix_len, sizeof(int32_t) * p.B, cudaMemcpyDeviceToHost) == cudaSuccess) {
       double suffix_tokens = 0.0;
       for (int b = 0; b < p.B; ++b) suffix_tokens += sl[b] > 0 ? sl[b] : 0;
-      suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : 2) / 6.8e6;   // stream at ~6.8 TB/s
+      suffix_us = suffix_tokens * 2.0 * p.Hkv * p.d * (d->dtype == MC_F32 ? 4 : fp8 ? 1 : 2) / 6.8e6;   // stream at ~6.8 TB/s
       suffix_tokens_now = suffix_tokens;
     } else {
       delete[] sl;
@@ -428,7 +440,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
   // The levels of the cascade share one persistent grid, so every item has the whole budget.
-  const bool want_tc = mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0);
+  const bool want_tc = !fp8 && mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0);
   mc::LevelWork work[1 + mc::kMaxOuterLevels];
   int nsp[1 + mc::kMaxOuterLevels];
   const double budget_us = suffix_us * 0.9;
@@ -457,11 +469,17 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   L->use_mma = mc::mma_supported(p, d->dtype) && !mc::env_int("MC_FORCE_FMA", 0);
   L->has_suffix = n_parts > part_base;
   L->sfx_plan = L->has_suffix && L->use_mma && mc::env_int("MC_SUFFIX_TMA", 1) ? mc::suffix_tma_plan(p, d->dtype) : nullptr;
+  if (fp8 && !(L->fp8 = mc::fp8_plan(p))) {
+    delete[] sl;
+    delete L;
+    return MC_ERR_UNSUPPORTED;
+  }
   // Suffix CTAs are launched longest first (by the lengths as they are now; appends change them slowly), so
   // that the launch ends on short items instead of a few long ones.  Without it the order is as numbered.
   L->suffix_order = nullptr;
-  if (L->use_mma && sl && mc::env_int("MC_SUFFIX_ORDER", 1)) {
-    const int per = L->sfx_plan ? mc::suffix_tma_items_per_cta() : mc::mma_items_per_cta(), n_chunks = n_parts - part_base;
+  if ((L->use_mma || L->fp8) && sl && mc::env_int("MC_SUFFIX_ORDER", 1)) {
+    const int per = L->fp8 ? mc::fp8_items_per_cta() : L->sfx_plan ? mc::suffix_tma_items_per_cta() : mc::mma_items_per_cta();
+    const int n_chunks = n_parts - part_base;
     const long long n_items = (long long)p.B * p.Hkv * n_chunks, n_ctas = (n_items + per - 1) / per;
     if (n_ctas > 1 && n_ctas < (1ll << 24)) {
       std::vector<int32_t> order((size_t)n_ctas), key((size_t)n_ctas);
@@ -490,7 +508,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   p.suffix_order = L->suffix_order;
   for (int k = 0; k < n_outer; ++k) L->outer_p[k].suffix_order = L->suffix_order;
 
-  const size_t rows = (size_t)p.B * p.Hq, e = d->dtype == MC_F32 ? 4 : 2;
+  const size_t rows = (size_t)p.B * p.Hq, e = L->io_dtype == MC_F32 ? 4 : 2;
   L->o_part_bytes = mc::align_up(rows * p.n_parts * p.d * sizeof(float), 256);
   L->lse_part_bytes = mc::align_up(rows * p.n_parts * sizeof(float), 256);
   size_t off = L->o_part_bytes + L->lse_part_bytes;
@@ -502,6 +520,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) {
     cudaFree(L->suffix_order);
     mc::suffix_tma_plan_free(L->sfx_plan);
+    mc::fp8_plan_free(L->fp8);
     delete L;
     return MC_ERR_OUT_OF_MEMORY;
   }
@@ -510,6 +529,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     cudaFree(L->dev_status);
     cudaFree(L->suffix_order);
     mc::suffix_tma_plan_free(L->sfx_plan);
+    mc::fp8_plan_free(L->fp8);
     delete L;
     return MC_ERR_CUDA;
   }
@@ -560,6 +580,7 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   if (L->join_ev) cudaEventDestroy(L->join_ev);
   mc::prefix_tc_plan_free(L->tc_plan);
   mc::suffix_tma_plan_free(L->sfx_plan);
+  mc::fp8_plan_free(L->fp8);
   cudaFree(L->dev_status);
   cudaFree(L->suffix_order);
   cudaFreeHost(L->host_status);
@@ -617,6 +638,7 @@ mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *
   Layout *L = reinterpret_cast<Layout *>(layout);
   if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new)) return MC_ERR_INVALID_ARG;
   if (!L->has_suffix) return MC_ERR_INVALID_ARG;   // a layout without private tokens has nowhere to append
+  if (L->fp8) return mc::launch_append_fp8(L->p, k_new, v_new, L->desc.suffix_len, reinterpret_cast<cudaStream_t>(stream));
   const int e = L->desc.dtype == MC_F32 ? 4 : 2;
   mc::append_kernel<<<L->p.B, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       L->p, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), L->desc.suffix_len, e);
@@ -630,6 +652,7 @@ mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const v
   if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new) || (q && !mc::aligned16(q)))
     return MC_ERR_INVALID_ARG;
   if (!L->has_suffix || !(theta_base > 0.0) || L->p.d % 2 != 0 || 256 % (L->p.d / 2) != 0) return MC_ERR_INVALID_ARG;
+  if (L->fp8) return MC_ERR_UNSUPPORTED;   // the rotary append does not quantise
   mc::RopeLevels lv;
   lv.n = 1 + L->n_outer;
   for (int k = 0; k < lv.n; ++k) {
@@ -676,7 +699,7 @@ mc_status_t mc_merge_lse(mc_kv_layout_t *layout, const float *o_part, const floa
   Layout *L = reinterpret_cast<Layout *>(layout);
   if (!L || !o_part || !lse_part || !o || !lse || !mc::aligned16(o_part) || !mc::aligned16(o))
     return MC_ERR_INVALID_ARG;
-  return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, reinterpret_cast<cudaStream_t>(stream));
+  return mc::launch_merge(L->p, L->io_dtype, o_part, lse_part, o, lse, reinterpret_cast<cudaStream_t>(stream));
 }
 
 static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const void *v_new, const void *q,
@@ -719,7 +742,7 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
     }
     // The merge is the suffix pass's programmatic dependent in turn (MC_PDL_MERGE=0: an ordinary launch): its CTAs
     // are resident and waiting when the last suffix CTA ends, instead of being launched then.
-    return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st,
+    return mc::launch_merge(L->p, L->io_dtype, o_part, lse_part, o, lse, st,
                             L->has_suffix && L->sfx_plan && mc::env_int("MC_PDL_MERGE", 1));
   }
   // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix
@@ -733,7 +756,7 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
   if (cudaEventRecord(L->join_ev, L->side_stream) != cudaSuccess ||
       cudaStreamWaitEvent(st, L->join_ev, 0) != cudaSuccess)
     return MC_ERR_CUDA;
-  return mc::launch_merge(L->p, L->desc.dtype, o_part, lse_part, o, lse, st);
+  return mc::launch_merge(L->p, L->io_dtype, o_part, lse_part, o, lse, st);
 }
 
 mc_status_t mc_decode_attn(mc_kv_layout_t *layout, const void *q, float scale, void *o, float *lse, void *ws,
@@ -756,7 +779,7 @@ mc_status_t mc_decode_step_host(mc_kv_layout_t *layout, const void *k_new_host, 
   if (ws_bytes < L->ws_bytes) return MC_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char *base = static_cast<char *>(ws);
-  const size_t e = L->desc.dtype == MC_F32 ? 4 : 2, rows = (size_t)L->p.B * L->p.Hq;
+  const size_t e = L->io_dtype == MC_F32 ? 4 : 2, rows = (size_t)L->p.B * L->p.Hq;
   const size_t q_bytes = rows * L->p.d * e, kv_bytes = (size_t)L->p.B * L->p.Hkv * L->p.d * e;
   void *q_dev = base + L->staging_off[0], *k_dev = base + L->staging_off[1], *v_dev = base + L->staging_off[2];
   void *o_dev = base + L->staging_off[3];

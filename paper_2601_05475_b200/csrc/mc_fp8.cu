@@ -176,26 +176,34 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
   const int32_t *row_pages = sp.pages + (sp.lo >> 4);
   const float *k_scale = p.k_scale, *v_scale = p.v_scale;
   // Page ids, their validity and their two scales are read 32 pages at a time (lane = page ordinal in the block), a
-  // block ahead of their use.  A page with an id outside the pool is loaded from page 0 and masked.
-  int ids[2];
-  float sk[2], sv[2];
-  uint32_t good[2];
-  auto load_block = [&](int blk) {
+  // block ahead of their use: block k's registers take block k + 2 once block k is consumed - first the ids, four
+  // iterations later (the load has returned by then) their validity and the two scales they lead to.  A page with an
+  // id outside the pool is loaded from page 0 and masked.
+  int ids0 = 0, ids1 = 0;          // blocks with an even / odd index (registers, selected by the block's parity)
+  float sk0 = 0.f, sk1 = 0.f, sv0 = 0.f, sv1 = 0.f;
+  uint32_t good0 = 0u, good1 = 0u;
+  auto load_ids = [&](int blk) {
     const int o = blk * 32 + lane;
-    int id = o < n_pages ? __ldg(row_pages + o) : 0;
+    const int id = o < n_pages ? __ldg(row_pages + o) : 0;
+    if (blk & 1) ids1 = id; else ids0 = id;
+  };
+  auto finish_block = [&](int blk) {
+    const int o = blk * 32 + lane;
+    int id = blk & 1 ? ids1 : ids0;
     const bool ok = o >= n_pages || (unsigned)id < (unsigned)p.num_pages;
     if (!ok) {
       latch(p, kDevBadPage);
       id = 0;
     }
-    ids[blk & 1] = id;
-    good[blk & 1] = __ballot_sync(0xffffffffu, ok);
+    const uint32_t gm = __ballot_sync(0xffffffffu, ok);
     const size_t slab = (size_t)id * p.Hkv + h;
-    sk[blk & 1] = o < n_pages ? __ldg(k_scale + slab) : 0.f;
-    sv[blk & 1] = o < n_pages ? __ldg(v_scale + slab) : 0.f;
+    const float a = o < n_pages ? __ldg(k_scale + slab) : 0.f, c = o < n_pages ? __ldg(v_scale + slab) : 0.f;
+    if (blk & 1) { ids1 = id; good1 = gm; sk1 = a; sv1 = c; } else { ids0 = id; good0 = gm; sk0 = a; sv0 = c; }
   };
-  load_block(0);
-  load_block(1);
+  load_ids(0);
+  load_ids(1);
+  finish_block(0);
+  finish_block(1);
   // B operand of the first product: Q^T as f16, column n = head gid; k-step c covers d in [16 c, 16 c + 16) in the
   // order the K fragments deliver it: slots 2t, 2t+1 <- d = 16c + 4t, +1; slots 2t+8, 2t+9 <- d = 16c + 4t + 2, +3
   uint32_t qf[8][2];
@@ -216,9 +224,10 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
   // Pages o and o + 1 (o even), each issued by the lane that holds its id.  The pad page repeats the last page.
   auto issue_pair = [&](int o) {
     if ((lane & 30) != (o & 30)) return;
+    int id = (o >> 5) & 1 ? ids1 : ids0;                                      // o is even: o and o + 1 share a block
+    const int id_even = __shfl_sync(0x3u << (lane & 30), id, lane & 30);
     o += lane & 1;
-    int id = ids[(o >> 5) & 1];
-    if (o >= n_pages) id = __shfl_sync(0x3u << (lane & 30), id, lane & 30);   // the pair's even lane holds the last page
+    if (o >= n_pages) id = id_even;                                           // (n_pages is odd then: o - 1 is the last page)
     const int s = o % kStages;
     mbar_expect_tx(&full[s], kStageBytes);
     tma_load_stage(smem_u32(ring[s]), &kv_map, id * p.Hkv + h, &full[s], pol);
@@ -247,9 +256,10 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
     alive = __all_sync(0xffffffffu, alive);
     if (!alive) break;
     const uint32_t base[2] = {smem_u32(ring[s0]), smem_u32(ring[s1])};
-    const int blk = (o >> 5) & 1;
-    const float ks0 = __shfl_sync(0xffffffffu, sk[blk], o & 31), ks1 = __shfl_sync(0xffffffffu, sk[blk], (o + 1) & 31);
-    const float vs0 = __shfl_sync(0xffffffffu, sv[blk], o & 31), vs1 = __shfl_sync(0xffffffffu, sv[blk], (o + 1) & 31);
+    const bool odd_blk = (o >> 5) & 1;
+    const float skb = odd_blk ? sk1 : sk0, svb = odd_blk ? sv1 : sv0;
+    const float ks0 = __shfl_sync(0xffffffffu, skb, o & 31), ks1 = __shfl_sync(0xffffffffu, skb, (o + 1) & 31);
+    const float vs0 = __shfl_sync(0xffffffffu, svb, o & 31), vs1 = __shfl_sync(0xffffffffu, svb, (o + 1) & 31);
     // ---- scores of both pages: two independent chains per page (even / odd 16-wide step)
     float sc[2][2][4];
 #pragma unroll
@@ -273,7 +283,7 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
     }
     // ---- masks: tokens at or beyond the part's end, the pad page, pages with a bad id
     const int tok0 = sp.lo + o * kPage;
-    const uint32_t gm = good[blk];   // o is even: o and o + 1 lie in the same block of 32
+    const uint32_t gm = odd_blk ? good1 : good0;   // o is even: o and o + 1 lie in the same block of 32
     const int hi0 = (gm >> (o & 31)) & 1u ? sp.hi : 0;
     const int hi1 = (o + 1 < n_pages) && ((gm >> ((o + 1) & 31)) & 1u) ? sp.hi : 0;
     const float c0 = sl2 * ks0, c1 = sl2 * ks1;
@@ -338,13 +348,9 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
     }
     __syncwarp();   // every lane has read both stages before they are refilled
     if (o + kStages < n_ord) issue_pair(o + kStages);
-    // block k's registers are reloaded with block k + 2 once block k is consumed and its last pages have been issued
-    // (issue runs kStages pages ahead of compute, so block k is fully issued when compute reaches page 32 k + 32 - kStages)
     const int done = o + 2;
-    if ((done & 31) == 0 && done + 32 < n_ord + 32) {
-      // pages [done + 32 - kStages, done + 32) of the block after next are issued from the OTHER register set: safe
-      load_block((done >> 5) + 1);
-    }
+    if ((done & 31) == 0) load_ids((done >> 5) + 1);
+    if ((done & 31) == 8 && done >= 40) finish_block((done >> 5) + 1);
   }
   if (!alive) {
     const long long t0 = clock64();

@@ -31,6 +31,7 @@ struct Params {
   const int32_t *row_limit;                          // per candidate: tokens of this prefix level it may see (null: all)
   const int32_t *suffix_order;                       // launch order of the suffix pass's CTAs (null: as numbered)
   int32_t *status;
+  const float *k_scale, *v_scale;                    // e4m3 cache only: one scale per (page, kv head), [num_pages][Hkv]
 };
 
 enum Mode : int { kPrefix = 0, kSuffix = 1 };
@@ -129,5 +130,17 @@ void suffix_tma_plan_free(SuffixTmaPlan *plan);
 int suffix_tma_items_per_cta();
 mc_status_t launch_suffix_tma(const Params &p, const SuffixTmaPlan *plan, const void *q, float scale, float *o_part,
                               float *lse_part, cudaStream_t stream, bool beside_previous);
+
+// KV cache in e4m3 with per-(page, kv head) scales (bf16 queries and outputs, d = 128, g <= 8): both passes on one
+// TMA-fed warp-level kernel, and the quantising append
+struct Fp8Plan;
+Fp8Plan *fp8_plan(const Params &p);
+void fp8_plan_free(Fp8Plan *plan);
+int fp8_items_per_cta();
+bool fp8_supported(const Params &p);
+mc_status_t launch_fp8(const Params &p, const Fp8Plan *plan, int mode, const void *q, float scale, float *o_part,
+                       float *lse_part, cudaStream_t stream);
+mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_new, int32_t *suffix_len,
+                              cudaStream_t stream);
 
 }  // namespace mc

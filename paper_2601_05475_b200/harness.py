@@ -15,14 +15,14 @@ from . import workload as wl
 def to_device(cfg: wl.Config, x: np.ndarray, device="cuda") -> torch.Tensor:
     """float32 values (storage-representable) -> device tensor of the storage dtype."""
     t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
-    if cfg.dtype == "bf16":
+    if cfg.dtype != "f32":
         t = t.to(torch.bfloat16)
     return t.to(device)
 
 
 def storage_to_device(cfg: wl.Config, a: np.ndarray, device="cuda") -> torch.Tensor:
-    """Storage array (float32, or uint16 bf16 bits) -> device tensor."""
-    if cfg.dtype == "f32":
+    """Storage array (float32, uint16 bf16 bits, or uint8 e4m3 codes) -> device tensor."""
+    if cfg.dtype == "f32" or a.dtype == np.uint8:
         return torch.from_numpy(a).to(device)
     return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
 
@@ -31,9 +31,11 @@ class DeviceProblem:
     """Pools, tables and lengths on the device plus the library's layout handle and workspace."""
 
     def __init__(self, cfg: wl.Config, tables: wl.PageTables, prefix_len: np.ndarray, suffix_len: np.ndarray,
-                 k_pool: torch.Tensor, v_pool: torch.Tensor, device="cuda", outer=()):
+                 k_pool: torch.Tensor, v_pool: torch.Tensor, device="cuda", outer=(), k_scale=None, v_scale=None):
+        """k_scale, v_scale: float32 [num_pages][Hkv] device tensors, for an e4m3 cache (cfg.dtype == "fp8")."""
         self.cfg, self.tables, self.device = cfg, tables, device
         self.k_pool, self.v_pool = k_pool, v_pool
+        self.k_scale, self.v_scale = k_scale, v_scale
         i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
         self.prefix_pages, self.suffix_pages = i32(tables.prefix_pages), i32(tables.suffix_pages)
         self.prefix_len, self.suffix_len = i32(prefix_len), i32(suffix_len)
@@ -42,8 +44,10 @@ class DeviceProblem:
         d.num_groups, d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = cfg.G, cfg.B, cfg.Hq, cfg.Hkv, cfg.d
         d.page_size, d.num_pages = wl.PAGE, tables.num_pages
         d.max_prefix_pages, d.max_suffix_pages = tables.max_prefix_pages, tables.max_suffix_pages
-        d.dtype = mc.MC_F32 if cfg.dtype == "f32" else mc.MC_BF16
+        d.dtype = {"f32": mc.MC_F32, "bf16": mc.MC_BF16, "fp8": mc.MC_FP8_E4M3}[cfg.dtype]
         d.k_pool, d.v_pool = k_pool.data_ptr(), v_pool.data_ptr()
+        if cfg.dtype == "fp8":
+            d.k_scale, d.v_scale = k_scale.data_ptr(), v_scale.data_ptr()
         d.group_offsets, d.prefix_pages = self.group_offsets.data_ptr(), self.prefix_pages.data_ptr()
         d.prefix_len, d.suffix_pages = self.prefix_len.data_ptr(), self.suffix_pages.data_ptr()
         d.suffix_len = self.suffix_len.data_ptr()
@@ -116,17 +120,32 @@ def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, d
     gen = torch.Generator(device=device)
     gen.manual_seed(cfg.seed * 1000003 + 17)
     shape = (tables.num_pages, cfg.Hkv, wl.PAGE, cfg.d)
-    k_pool = torch.empty(shape, dtype=tdtype, device=device)
-    v_pool = torch.empty(shape, dtype=tdtype, device=device)
+    fp8 = cfg.dtype == "fp8"
+    k_pool = torch.empty(shape, dtype=torch.uint8 if fp8 else tdtype, device=device)
+    v_pool = torch.empty(shape, dtype=torch.uint8 if fp8 else tdtype, device=device)
+    k_scale = torch.empty((tables.num_pages, cfg.Hkv), dtype=torch.float32, device=device) if fp8 else None
+    v_scale = torch.empty((tables.num_pages, cfg.Hkv), dtype=torch.float32, device=device) if fp8 else None
     step = max(1, (1 << 28) // (cfg.Hkv * wl.PAGE * cfg.d))          # pages per chunk, bounds temporaries
     for lo in range(0, tables.num_pages, step):
         hi = min(tables.num_pages, lo + step)
-        k_pool[lo:hi].normal_(generator=gen)
-        v_pool[lo:hi].normal_(generator=gen)
+        k = torch.empty((hi - lo,) + shape[1:], dtype=tdtype, device=device).normal_(generator=gen)
+        v = torch.empty((hi - lo,) + shape[1:], dtype=tdtype, device=device).normal_(generator=gen)
         if cfg.k_outlier_prob > 0.0:
             mask = torch.rand((hi - lo, cfg.Hkv, wl.PAGE, 1), device=device, generator=gen) < cfg.k_outlier_prob
-            k_pool[lo:hi] = torch.where(mask, k_pool[lo:hi] * cfg.k_outlier_scale, k_pool[lo:hi])
-    dp = DeviceProblem(cfg, tables, prefix_len, suffix_len, k_pool, v_pool, device, outer=outer_np)
+            k = torch.where(mask, k * cfg.k_outlier_scale, k)
+        if fp8:
+            # an input generator, not the library's quantiser: every page gets the scale its first token would have
+            # given it (twice that row's largest magnitude over 448) and torch's cast makes the codes; whatever
+            # lands in the pools IS the input, and the tests read it back from there
+            for src, pool, sc in ((k, k_pool, k_scale), (v, v_pool, v_scale)):
+                s = (src[:, :, 0].float().abs().amax(dim=-1) * 2.0 / 448.0).clamp_min(1e-30)
+                sc[lo:hi] = s
+                pool[lo:hi] = (src.float() / s[:, :, None, None]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+        else:
+            k_pool[lo:hi], v_pool[lo:hi] = k, v
+        del k, v
+    dp = DeviceProblem(cfg, tables, prefix_len, suffix_len, k_pool, v_pool, device, outer=outer_np,
+                       k_scale=k_scale, v_scale=v_scale)
     dp.outer_np = outer_np
     return dp
 
@@ -149,7 +168,8 @@ def device_append(cfg: wl.Config, step: int, device="cuda"):
 
 def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int] = None):
     """Copies candidate b's whole history for kv head h to the host, in token order, by plain indexing
-    through the page tables: returns (K [n][d], V [n][d]) as float32 numpy arrays."""
+    through the page tables: returns (K [n][d], V [n][d]) as float32 numpy arrays - for an e4m3 cache each of the
+    two is a pair (codes uint8 [n][d], the scale of every token's page float32 [n]) instead."""
     j = int(np.searchsorted(dp.tables.group_offsets, b, side="right") - 1)
     P = int(dp.prefix_len[j].item())
     s = int(dp.suffix_len[b].item()) if suffix_len_now is None else suffix_len_now
@@ -159,14 +179,21 @@ def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int
         segments.append((pages[jo], int(lens[jo])))
     segments += [(dp.tables.prefix_pages[j], P), (dp.tables.suffix_pages[b], s)]
     out = []
-    for pool in (dp.k_pool, dp.v_pool):
-        parts = []
+    for pool, scale in ((dp.k_pool, dp.k_scale), (dp.v_pool, dp.v_scale)):
+        parts, scales = [], []
         for pages_row, n in segments:
             n_pages = (n + wl.PAGE - 1) // wl.PAGE
             if n_pages:
                 ids = torch.from_numpy(np.ascontiguousarray(pages_row[:n_pages], dtype=np.int64)).to(pool.device)
-                parts.append(pool[ids, h].reshape(n_pages * wl.PAGE, -1)[:n].float().cpu().numpy())
-        out.append(np.concatenate(parts, axis=0) if parts else np.zeros((0, dp.cfg.d), dtype=np.float32))
+                rows = pool[ids, h].reshape(n_pages * wl.PAGE, -1)[:n]
+                parts.append(rows.cpu().numpy() if pool.dtype == torch.uint8 else rows.float().cpu().numpy())
+                if scale is not None:
+                    scales.append(scale[ids, h].cpu().numpy().repeat(wl.PAGE)[:n])
+        empty = np.zeros((0, dp.cfg.d), dtype=np.uint8 if pool.dtype == torch.uint8 else np.float32)
+        rows = np.concatenate(parts, axis=0) if parts else empty
+        if scale is not None:      # an e4m3 cache: the codes and each token's scale, for the caller to decode
+            rows = (rows, np.concatenate(scales) if scales else np.zeros(0, dtype=np.float32))
+        out.append(rows)
     return out[0], out[1]
 
 

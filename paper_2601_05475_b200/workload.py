@@ -71,7 +71,7 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 @dataclasses.dataclass(frozen=True)
 class Config:
     name: str
-    dtype: str                      # "f32" | "bf16"
+    dtype: str                      # "f32" | "bf16" | "fp8" (e4m3 cache with per-page scales; q, o, new tokens bf16)
     G: int                          # prompt groups
     C: int                          # candidates per group
     Hq: int
@@ -99,7 +99,13 @@ class Config:
 
     @property
     def elem_bytes(self) -> int:
+        """Bytes per element of q, o and the appended rows."""
         return 4 if self.dtype == "f32" else 2
+
+    @property
+    def kv_elem_bytes(self) -> int:
+        """Bytes per cached K or V element."""
+        return 1 if self.dtype == "fp8" else self.elem_bytes
 
 
 CONFIGS: Dict[str, Config] = {
@@ -378,9 +384,13 @@ def make_host_problem(cfg: Config, *, headroom_tokens: Optional[int] = None, per
 def unique_bytes(cfg: Config, prefix_len: np.ndarray, suffix_len: np.ndarray) -> Dict[str, int]:
     """Minimum unique traffic of one decode step: every valid prefix token once per group, every valid
     suffix token once, all KV heads, K and V; plus Q read, O write, LSE write."""
-    per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+    per_tok = 2 * cfg.Hkv * cfg.d * cfg.kv_elem_bytes
     kv_prefix = int(prefix_len.astype(np.int64).sum()) * per_tok
     kv_suffix = int(suffix_len.astype(np.int64).sum()) * per_tok
+    if cfg.dtype == "fp8":           # plus the K and the V scale of every page that holds a token, per kv head
+        pages = lambda n: int(((n.astype(np.int64) + PAGE - 1) // PAGE).sum())
+        kv_prefix += pages(prefix_len) * 2 * cfg.Hkv * 4
+        kv_suffix += pages(suffix_len) * 2 * cfg.Hkv * 4
     qo = 2 * cfg.B * cfg.Hq * cfg.d * cfg.elem_bytes
     lse = cfg.B * cfg.Hq * 4
     return {"kv_prefix": kv_prefix, "kv_suffix": kv_suffix, "q_o": qo, "lse": lse,
