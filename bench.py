@@ -290,7 +290,7 @@ def run_gpu(args):
         kv = [device_append(cfg, i) for i in range(4)] if appends else None
         len0 = dp.suffix_len.clone()
         ub0 = wl.unique_bytes(cfg, dp.prefix_len.cpu().numpy(), len0.cpu().numpy())
-        per_tok = 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+        per_tok = 2 * cfg.Hkv * cfg.d * cfg.kv_elem_bytes + (2 * cfg.Hkv * 4 / wl.PAGE if cfg.dtype == "fp8" else 0)
         outer_tokens = sum(int(np.sum(lens)) for (_, lens) in outer)          # each outer token is unique once
         ub0["total"] += outer_tokens * per_tok
 
@@ -540,7 +540,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / args.steps
         tokens = float((dp.suffix_len if args.pass_only == "suffix" else dp.prefix_len).sum().item())
-        nbytes = tokens * 2 * cfg.Hkv * cfg.d * cfg.elem_bytes
+        nbytes = tokens * 2 * cfg.Hkv * cfg.d * cfg.kv_elem_bytes
         ok = mc.mc_get_last_status(dp.layout) == mc.MC_OK
         if rank == 0:
             print(json.dumps({"pass": args.pass_only, "workload": cfg.name, "ms": ms, "algorithmic_bytes": nbytes,
@@ -559,7 +559,7 @@ def run_gpu(args):
     others = {}
     cold = None
     if args.all_configs:
-        for name in ("cfg2", "cfg3", "cfg4"):
+        for name in ("cfg2", "cfg3", "cfg4", "cfg4_fp8"):
             if name != args.workload:
                 others[name] = measure(name, args.steps, args.warmup, True)
         cold = measure_prefix_cold("cfg2", max(args.steps, 60), args.warmup)

@@ -151,6 +151,13 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout);
  * twice.  Synchronises `stream`.  `scratch` is device memory of at least num_pages*4 bytes. */
 mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t scratch_bytes, void *stream);
 
+/* MC_FP8_E4M3 layouts whose prefix pass runs on the tensor cores keep the prefix levels widened to 16-bit pools of
+ * their own (made by mc_kv_layout_create*, which waits for them; 4 * Hkv * d bytes per prefix page slot of the
+ * tables): that pass needs 16-bit operands and the prefix does not change while the candidates decode.  After
+ * changing prefix pages, their scales, the prefix tables or prefix_len of such a layout, call this to widen them
+ * again (asynchronous on `stream`).  On every other layout it does nothing and returns MC_OK. */
+mc_status_t mc_kv_layout_refresh_prefix(mc_kv_layout_t *layout, void *stream);
+
 /* Part geometry chosen at create time (needed to size and index o_part / lse_part). */
 mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry_t *out);
 

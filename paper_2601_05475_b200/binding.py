@@ -40,6 +40,7 @@ EXPORTS = {
     "mc_kv_layout_create_cascade": (c_int32, [POINTER(LayoutDesc), POINTER(PrefixLevel), c_int32, POINTER(c_void_p)]),
     "mc_kv_layout_destroy": (c_int32, [c_void_p]),
     "mc_kv_layout_validate": (c_int32, [c_void_p, c_void_p, c_size_t, c_void_p]),
+    "mc_kv_layout_refresh_prefix": (c_int32, [c_void_p, c_void_p]),
     "mc_kv_layout_geometry": (c_int32, [c_void_p, POINTER(PartGeometry)]),
     "mc_workspace_bytes": (c_size_t, [c_void_p]),
     "mc_kv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -128,6 +129,10 @@ def mc_kv_layout_create_cascade(desc: LayoutDesc, outer) -> int:
 
 def mc_kv_layout_destroy(layout: int) -> None:
     _check(lib().mc_kv_layout_destroy(layout), "mc_kv_layout_destroy")
+
+
+def mc_kv_layout_refresh_prefix(layout: int, stream: int = 0) -> None:
+    _check(lib().mc_kv_layout_refresh_prefix(layout, stream), "mc_kv_layout_refresh_prefix")
 
 
 def mc_kv_layout_geometry(layout: int) -> PartGeometry:

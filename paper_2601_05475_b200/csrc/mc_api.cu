@@ -24,7 +24,10 @@ struct Layout {
   bool use_mma;
   bool has_suffix;            // false: no private tokens (max_suffix_pages = 0), the suffix pass is not launched
   SuffixTmaPlan *sfx_plan;    // non-null: the suffix pass runs on the TMA-fed kernel
-  Fp8Plan *fp8;               // non-null: e4m3 cache, both passes run on its kernel
+  Fp8Plan *fp8;               // non-null: e4m3 cache; its kernel runs the suffix pass and, without tc_plan, the prefix pass
+  Params xp;                  // e4m3 cache with tc_plan: the base level seen through the expanded (bf16) prefix pools
+  Params x_src[1 + kMaxOuterLevels];   // ... and the levels the expansion reads, outermost first
+  int x_n;
   int io_dtype;               // type of q and o: the cache's, or bf16 over an e4m3 cache
   PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
@@ -250,7 +253,8 @@ mc_status_t run_level(Layout *L, const Params &p, int mode, const void *q, float
 mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_part, float *lse_part,
                      cudaStream_t st) {
   if (mode == kPrefix) {
-    if (L->tc_plan && scale != 0.f) return launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st);
+    if (L->tc_plan && scale != 0.f)
+      return launch_prefix_tc(L->fp8 ? L->xp : L->p, L->tc_plan, q, scale, o_part, lse_part, st);
     for (int k = L->n_outer - 1; k >= 0; --k) {
       mc_status_t s = run_level(L, L->outer_p[k], kPrefix, q, scale, o_part, lse_part, st);
       if (s != MC_OK) return s;
@@ -377,6 +381,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   L->n_outer = n_outer;
   L->io_dtype = fp8 ? MC_BF16 : d->dtype;
   L->fp8 = nullptr;
+  L->x_n = 0;
   mc::Params &p = L->p;
   p.k_pool = d->k_pool; p.v_pool = d->v_pool;
   p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
@@ -440,7 +445,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   if (mc::env_int("MC_SUFFIX_PART_TOKENS", 0) > 0) ts = mc::env_int("MC_SUFFIX_PART_TOKENS", ts) / mc::kPage * mc::kPage;
   if (ts < mc::kPage) ts = mc::kPage;
   // The levels of the cascade share one persistent grid, so every item has the whole budget.
-  const bool want_tc = !fp8 && mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0);
+  const bool want_tc = mc::env_int("MC_PREFIX_TC", 1) && !mc::env_int("MC_FORCE_FMA", 0);
   mc::LevelWork work[1 + mc::kMaxOuterLevels];
   int nsp[1 + mc::kMaxOuterLevels];
   const double budget_us = suffix_us * 0.9;
@@ -550,14 +555,32 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
       for (int k = n_outer, i = 0; k >= 0; --k, ++i) {
         levels[i] = k == 0 ? p : L->outer_p[k - 1];
         max_group[i] = work[k].max_group;
-        all = all && mc::prefix_tc_supported(levels[i], d->dtype) && max_group[i] <= p.B;
+        all = all && mc::prefix_tc_supported(levels[i], MC_BF16) && (fp8 || d->dtype == MC_BF16) && max_group[i] <= p.B;
       }
       // The suffix pass reaches the memory roofline from little more than half of the SMs and cannot share an SM
       // with a prefix CTA, so the prefix pass gets enough CTAs to end early (a tenth of the suffix pass's time,
       // measured alone; beside the suffix stream it runs about a third longer) and frees its SMs for the rest.
+      const float *k_scale = nullptr;
+      if (all && fp8) {
+        // An e4m3 cache: the pass runs on the prefix levels widened once to 16-bit pools of their own (the prefix
+        // does not change while candidates decode; mc_kv_layout_refresh_prefix repeats the widening).
+        mc::Params widened[1 + mc::kMaxOuterLevels];
+        all = mc::fp8_expand_alloc(L->fp8, levels, n_outer + 1, widened) &&
+              mc::fp8_expand_launch(L->fp8, levels, n_outer + 1, nullptr) == MC_OK &&
+              cudaStreamSynchronize(nullptr) == cudaSuccess;
+        if (all) {
+          L->x_n = n_outer + 1;
+          for (int i = 0; i <= n_outer; ++i) {
+            L->x_src[i] = levels[i];
+            levels[i] = widened[i];
+          }
+          L->xp = widened[n_outer];
+          k_scale = mc::fp8_expanded_k_scale(L->fp8);
+        }
+      }
       if (all)
         L->tc_plan = mc::prefix_tc_plan(levels, max_group, n_outer + 1, sms, mc::env_int("MC_PREFIX_CTAS", 0),
-                                        0.1 * budget_us, mc::kTileUs, mc::kItemUs);
+                                        0.1 * budget_us, mc::kTileUs, mc::kItemUs, k_scale);
     }
     (void)cudaGetLastError();
   }
@@ -586,6 +609,13 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   cudaFreeHost(L->host_status);
   delete L;
   return MC_OK;
+}
+
+mc_status_t mc_kv_layout_refresh_prefix(mc_kv_layout_t *layout, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L) return MC_ERR_INVALID_ARG;
+  if (!L->fp8 || L->x_n == 0) return MC_OK;   // nothing is kept: every pass reads the pools themselves
+  return mc::fp8_expand_launch(L->fp8, L->x_src, L->x_n, reinterpret_cast<cudaStream_t>(stream));
 }
 
 mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry_t *g) {
@@ -722,9 +752,9 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
       mc::env_int("MC_PREFIX_DIRECT", 1)) {
     // No private tokens and one part per row from the prefix pass: it writes the final output itself, no merge.
     if (k_new) return MC_ERR_INVALID_ARG;   // nowhere to append
-    return mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st, o, lse);
+    return mc::launch_prefix_tc(L->fp8 ? L->xp : L->p, L->tc_plan, q, scale, o_part, lse_part, st, o, lse);
   }
-  if (L->tc_plan && L->use_mma && scale != 0.f && L->pdl) {
+  if (L->tc_plan && (L->use_mma || L->fp8) && scale != 0.f && L->pdl) {
     // One stream: the suffix pass is launched behind the tensor-core prefix pass as its programmatic
     // dependent, so it starts once every prefix CTA is running, not when they end.  The order holds when
     // the step is replayed from a captured graph.  The merge, launched the ordinary way, waits for both.
@@ -733,17 +763,19 @@ static mc_status_t decode_impl(mc_kv_layout_t *layout, const void *k_new, const 
     // nothing of the append, so its start-up runs beside it; the suffix pass, which does, is released by the
     // prefix CTAs only after they have seen the append grid complete (MC_PDL_APPEND=0: an ordinary launch).
     const bool early = k_new != nullptr && mc::env_int("MC_PDL_APPEND", 1);
-    if ((s = mc::launch_prefix_tc(L->p, L->tc_plan, q, scale, o_part, lse_part, st, nullptr, nullptr, early)) != MC_OK)
+    if ((s = mc::launch_prefix_tc(L->fp8 ? L->xp : L->p, L->tc_plan, q, scale, o_part, lse_part, st, nullptr, nullptr,
+                                  early)) != MC_OK)
       return s;
     if (L->has_suffix) {
-      s = L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
-                      : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
+      s = L->fp8        ? mc::launch_fp8(L->p, L->fp8, mc::kSuffix, q, scale, o_part, lse_part, st, true)
+          : L->sfx_plan ? mc::launch_suffix_tma(L->p, L->sfx_plan, q, scale, o_part, lse_part, st, true)
+                        : mc::launch_mma(L->p, mc::kSuffix, q, scale, o_part, lse_part, st, true);
       if (s != MC_OK) return s;
     }
     // The merge is the suffix pass's programmatic dependent in turn (MC_PDL_MERGE=0: an ordinary launch): its CTAs
     // are resident and waiting when the last suffix CTA ends, instead of being launched then.
     return mc::launch_merge(L->p, L->io_dtype, o_part, lse_part, o, lse, st,
-                            L->has_suffix && L->sfx_plan && mc::env_int("MC_PDL_MERGE", 1));
+                            L->has_suffix && (L->sfx_plan || L->fp8) && mc::env_int("MC_PDL_MERGE", 1));
   }
   // Otherwise two streams: the prefix pass first, on the caller's stream; the append (it touches only suffix
   // pages and lengths) and the suffix pass on the handle's side stream; the merge joins them.

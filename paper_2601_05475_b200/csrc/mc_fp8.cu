@@ -148,6 +148,9 @@ attn_fp8_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint32
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   __syncthreads();
+  // (a kernel launched behind this one as its programmatic dependent - the merge, which waits for this grid's
+  // completion before it reads anything - may take its place on the SMs once every CTA of this grid has started)
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
   const int nparts_mode = MODE == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
@@ -385,6 +388,66 @@ attn_fp8_kernel(Params p, const __grid_constant__ CUtensorMap kv_map, uint32_t k
                 const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
                 float *__restrict__ lse_part, long long wait_cycles) {
   attn_fp8_body<MODE>(p, kv_map, k_off, v_off, q, sl2, o_part, lse_part, wait_cycles);
+  // Launched as the programmatic dependent of the tensor-core prefix pass, the suffix grid starts before that one
+  // ends; one thread of the grid waits for the prerequisite grid before it exits, so that this grid - and the merge
+  // behind it - cannot complete earlier.  Without a prerequisite the instruction returns at once.
+  if (MODE == kSuffix && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Expansion of the prefix levels for the tensor-core prefix pass.  That pass wants 16-bit operands in shared
+// memory, and the prefix does not change while candidates decode: its pages are widened once into pools of their
+// own - K as the exact codes in bf16 (e4m3 fits bf16 exactly; the page's K scale travels beside it and multiplies
+// the scores in the softmax, so no rounding touches the scores), V as bf16(code * scale) (one rounding of relative
+// size 2^-9 on the values that are averaged).  One CTA per (group, page index) of a level; page (j, i) lands at the
+// fixed id base + j * max_pages + i, and the level's table of expanded ids gets that id, or -1 for a page whose
+// source id lies outside the pool.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+expand_prefix_kernel(Params p, int base, __nv_bfloat16 *__restrict__ kx, __nv_bfloat16 *__restrict__ vx,
+                     float *__restrict__ kx_scale, int32_t *__restrict__ xpages) {
+  const int j = blockIdx.x / p.max_pp, i = blockIdx.x % p.max_pp;
+  int len = __ldg(p.prefix_len + j);
+  len = len < 0 ? 0 : len > p.max_pp * kPage ? p.max_pp * kPage : len;
+  if (i * kPage >= len) return;
+  const int pid = __ldg(p.prefix_pages + (size_t)j * p.max_pp + i);
+  const int cid = base + blockIdx.x;
+  if ((unsigned)pid >= (unsigned)p.num_pages) {
+    if (threadIdx.x == 0) {
+      latch(p, kDevBadPage);
+      xpages[blockIdx.x] = -1;
+    }
+    return;
+  }
+  if (threadIdx.x == 0) xpages[blockIdx.x] = cid;
+  if (threadIdx.x < p.Hkv) kx_scale[(size_t)cid * p.Hkv + threadIdx.x] = __ldg(p.k_scale + (size_t)pid * p.Hkv + threadIdx.x);
+  const int n_vec = p.Hkv * kPage * D / 16;   // 16-byte pieces of one page of one pool
+  const uint4 *ksrc = reinterpret_cast<const uint4 *>(p.k_pool) + (size_t)pid * n_vec;
+  const uint4 *vsrc = reinterpret_cast<const uint4 *>(p.v_pool) + (size_t)pid * n_vec;
+  uint4 *kdst = reinterpret_cast<uint4 *>(kx) + (size_t)cid * n_vec * 2;
+  uint4 *vdst = reinterpret_cast<uint4 *>(vx) + (size_t)cid * n_vec * 2;
+  for (int t = threadIdx.x; t < 2 * n_vec; t += blockDim.x) {
+    const bool is_v = t >= n_vec;
+    const int c = is_v ? t - n_vec : t;
+    const uint4 w = __ldg((is_v ? vsrc : ksrc) + c);
+    const float sc = is_v ? __ldg(p.v_scale + (size_t)pid * p.Hkv + c / (kPage * D / 16)) : 1.f;
+    const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+    uint32_t out[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint32_t lo, hi;
+      widen4(in[k], lo, hi);
+      const __half2 a = *reinterpret_cast<__half2 *>(&lo), b = *reinterpret_cast<__half2 *>(&hi);
+      const float2 fa = __half22float2(a), fb = __half22float2(b);
+      const __nv_bfloat162 ra = __floats2bfloat162_rn(fa.x * sc, fa.y * sc), rb = __floats2bfloat162_rn(fb.x * sc, fb.y * sc);
+      out[2 * k] = *reinterpret_cast<const uint32_t *>(&ra);
+      out[2 * k + 1] = *reinterpret_cast<const uint32_t *>(&rb);
+    }
+    uint4 *dst = (is_v ? vdst : kdst) + 2 * c;
+    dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+    dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -474,6 +537,11 @@ struct Fp8Plan {
   CUtensorMap kv_map;
   uint32_t k_off, v_off;   // where a stage holds the K slab and the V slab
   long long wait_cycles;   // limit of every device-side wait
+  // the prefix levels widened to bf16 for the tensor-core prefix pass (null: not made)
+  __nv_bfloat16 *kx, *vx;
+  float *kx_scale;
+  int32_t *xpages;         // expanded page ids, level after level, [G_k][max_pages_k] each
+  int x_pages;             // pages in kx / vx
 };
 
 int fp8_items_per_cta() { return kW; }
@@ -487,6 +555,10 @@ Fp8Plan *fp8_plan(const Params &p) {
   plan->k_off = ka < va ? 0u : kSlabBytes;
   plan->v_off = ka < va ? kSlabBytes : 0u;
   plan->wait_cycles = wait_limit_cycles();
+  plan->kx = plan->vx = nullptr;
+  plan->kx_scale = nullptr;
+  plan->xpages = nullptr;
+  plan->x_pages = 0;
   if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||
       !encode_kv8_pair_map(&plan->kv_map, ka < va ? p.k_pool : p.v_pool, (unsigned long long)(ka < va ? va - ka : ka - va),
                            p.num_pages, p.Hkv) ||
@@ -501,23 +573,84 @@ Fp8Plan *fp8_plan(const Params &p) {
   return plan;
 }
 
-void fp8_plan_free(Fp8Plan *plan) { delete plan; }
+void fp8_plan_free(Fp8Plan *plan) {
+  if (!plan) return;
+  cudaFree(plan->kx);
+  cudaFree(plan->vx);
+  cudaFree(plan->kx_scale);
+  cudaFree(plan->xpages);
+  delete plan;
+}
+
+// Allocates the expanded pools for `n_levels` prefix levels and fills `expanded[k]` with level k seen through them
+// (pools, page table, page count, scale array; everything else as in levels[k]).  false: out of memory or too large.
+bool fp8_expand_alloc(Fp8Plan *plan, const Params *levels, int n_levels, Params *expanded) {
+  long long total = 0;
+  for (int k = 0; k < n_levels; ++k) total += (long long)levels[k].G * levels[k].max_pp;
+  if (total < 1 || total > 0x7fffffffLL / levels[0].Hkv) return false;
+  const size_t pool_bytes = (size_t)total * levels[0].Hkv * kPage * D * sizeof(__nv_bfloat16);
+  if (cudaMalloc(&plan->kx, pool_bytes) != cudaSuccess || cudaMalloc(&plan->vx, pool_bytes) != cudaSuccess ||
+      cudaMalloc(&plan->kx_scale, (size_t)total * levels[0].Hkv * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&plan->xpages, (size_t)total * sizeof(int32_t)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    cudaFree(plan->kx); cudaFree(plan->vx); cudaFree(plan->kx_scale); cudaFree(plan->xpages);
+    plan->kx = plan->vx = nullptr;
+    plan->kx_scale = nullptr;
+    plan->xpages = nullptr;
+    return false;
+  }
+  plan->x_pages = (int)total;
+  long long base = 0;
+  for (int k = 0; k < n_levels; ++k) {
+    expanded[k] = levels[k];
+    expanded[k].k_pool = plan->kx;
+    expanded[k].v_pool = plan->vx;
+    expanded[k].num_pages = plan->x_pages;
+    expanded[k].prefix_pages = plan->xpages + base;
+    expanded[k].k_scale = plan->kx_scale;
+    expanded[k].v_scale = nullptr;
+    base += (long long)levels[k].G * levels[k].max_pp;
+  }
+  return true;
+}
+
+const float *fp8_expanded_k_scale(const Fp8Plan *plan) { return plan ? plan->kx_scale : nullptr; }
+
+// (Re)writes the expanded pools from the levels' pages as they are now; asynchronous on `stream`.
+mc_status_t fp8_expand_launch(const Fp8Plan *plan, const Params *levels, int n_levels, cudaStream_t stream) {
+  if (!plan->kx) return MC_OK;
+  long long base = 0;
+  for (int k = 0; k < n_levels; ++k) {
+    const long long n = (long long)levels[k].G * levels[k].max_pp;
+    expand_prefix_kernel<<<(unsigned)n, 256, 0, stream>>>(levels[k], (int)base, plan->kx, plan->vx, plan->kx_scale,
+                                                          plan->xpages + base);
+    count_launch();
+    base += n;
+  }
+  return check_launch();
+}
 
 mc_status_t launch_fp8(const Params &p, const Fp8Plan *plan, int mode, const void *q, float scale, float *o_part,
-                       float *lse_part, cudaStream_t stream) {
+                       float *lse_part, cudaStream_t stream, bool beside_previous) {
   const int nparts_mode = mode == kPrefix ? p.n_prefix_parts : p.n_parts - p.suffix_part_base;
   const long long n_items = (long long)p.B * p.Hkv * nparts_mode;
   if (n_items == 0) return MC_OK;
-  const unsigned grid = (unsigned)((n_items + kW - 1) / kW);
   const __nv_bfloat16 *qb = reinterpret_cast<const __nv_bfloat16 *>(q);
-  if (mode == kPrefix)
-    attn_fp8_kernel<kPrefix><<<grid, kW * 32, sizeof(Smem), stream>>>(p, plan->kv_map, plan->k_off, plan->v_off, qb,
-                                                                     scale * kLog2e, o_part, lse_part, plan->wait_cycles);
-  else
-    attn_fp8_kernel<kSuffix><<<grid, kW * 32, sizeof(Smem), stream>>>(p, plan->kv_map, plan->k_off, plan->v_off, qb,
-                                                                     scale * kLog2e, o_part, lse_part, plan->wait_cycles);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((n_items + kW - 1) / kW));
+  cfg.blockDim = dim3(kW * 32);
+  cfg.dynamicSmemBytes = sizeof(Smem);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = beside_previous && mode == kSuffix ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, mode == kPrefix ? attn_fp8_kernel<kPrefix> : attn_fp8_kernel<kSuffix>, p,
+                                           plan->kv_map, plan->k_off, plan->v_off, qb, scale * kLog2e, o_part, lse_part,
+                                           plan->wait_cycles);
   count_launch();
-  return check_launch();
+  return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }
 
 mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_new, int32_t *suffix_len,

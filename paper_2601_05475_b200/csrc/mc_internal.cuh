@@ -106,8 +106,10 @@ int mma_items_per_cta();
 constexpr int kMaxTcLevels = 4;
 struct PrefixTcPlan;
 bool prefix_tc_supported(const Params &p, int dtype);
+// `k_scale` non-null: the levels' pools are an e4m3 cache expanded to bf16 (K: the exact codes, V: dequantised) and
+// k_scale [page][kv head] holds each page's K scale, applied to the scores in the softmax.
 PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int fixed_ctas,
-                             double target_us, double tile_us, double item_us);
+                             double target_us, double tile_us, double item_us, const float *k_scale = nullptr);
 void prefix_tc_plan_free(PrefixTcPlan *plan);
 int prefix_tc_grid(const PrefixTcPlan *plan);
 bool prefix_tc_shape_supported(const Params &p, int dtype);   // everything but the part geometry
@@ -139,7 +141,11 @@ void fp8_plan_free(Fp8Plan *plan);
 int fp8_items_per_cta();
 bool fp8_supported(const Params &p);
 mc_status_t launch_fp8(const Params &p, const Fp8Plan *plan, int mode, const void *q, float scale, float *o_part,
-                       float *lse_part, cudaStream_t stream);
+                       float *lse_part, cudaStream_t stream, bool beside_previous = false);
+// the prefix levels widened to bf16 pools of their own, for the tensor-core prefix pass
+bool fp8_expand_alloc(Fp8Plan *plan, const Params *levels, int n_levels, Params *expanded);
+const float *fp8_expanded_k_scale(const Fp8Plan *plan);
+mc_status_t fp8_expand_launch(const Fp8Plan *plan, const Params *levels, int n_levels, cudaStream_t stream);
 mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_new, int32_t *suffix_len,
                               cudaStream_t stream);
 

@@ -57,6 +57,7 @@ struct __align__(1024) Smem {   // exactly the 227 KB a CTA may have
   uint64_t both;                      // the two teams meet here around an item's epilogue
   float xch[kTeams][2][kTileM];       // [team][m, l][row]: the teams show each other their running maximum and row sum
   uint32_t page_ok[8];                // per tile (index kt & 7): which of its 8 pages hold valid data
+  float kscale[8][8];                 // per tile (index kt & 7) and page: the K scale of an expanded e4m3 cache
   uint32_t tmem_base;
   volatile int abort;
   long long wait_cycles;              // limit of every wait of this CTA
@@ -310,12 +311,15 @@ __device__ __forceinline__ bool item_has_work(const Item &it, int cand_per_tile)
   return (it.lo < it.hi || it.lo2 < it.hi2) && it.mt * cand_per_tile < it.n_cand;
 }
 
+// KSCALE: the pools hold the exact codes of an e4m3 cache widened to bf16 (K) and its dequantised values (V); the
+// scores of every page are multiplied by that page's K scale (`k_scale` [page][kv head]) in the softmax.
+template <bool KSCALE>
 __global__ void __maxnreg__(168)
 prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
                  const __grid_constant__ CUtensorMap v_map, const __nv_bfloat16 *__restrict__ q, float sl2,
                  float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
                  const int32_t *__restrict__ cta_begin, __nv_bfloat16 *__restrict__ o_final,
-                 float *__restrict__ lse_final, long long wait_cycles) {
+                 float *__restrict__ lse_final, long long wait_cycles, const float *__restrict__ k_scale) {
   // o_final != null: every row gets exactly one part from this launch and none from anywhere else, so the item
   // writes the row's final output (bf16) and log-sum-exp itself and no merge follows.
   const bool direct = o_final != nullptr;
@@ -472,6 +476,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if (!ok) break;
           // page_ok is published before this warp's arrive on full_k; the softmax role reads it after s_full of
           // THIS tile, which follows full_k of this tile
+          if (KSCALE && prole == 0) {
+            if (lane < 8) sm.kscale[kt & 7][lane] = in_range && good ? __ldg(k_scale + (size_t)pid * p.Hkv + it.h) : 1.f;
+            __syncwarp();
+          }
           if (lane == 0) {
             if (prole == 0) sm.page_ok[kt & 7] = okmask;
             mbar_expect_tx(&sm.full_k[sk], kHalfBytes);
@@ -647,6 +655,10 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         // which of the tile's 8 pages hold valid data (inside the prefix, page id inside the pool)
         const uint32_t page_ok = sm.page_ok[(kt + t) & 7];
         const bool full_tile = page_ok == 0xffu && t0 + kTileN <= hi_row;
+        // per-page factor of the scores in log2 units: softmax scale x the page's K scale (sign of sl2 throughout)
+        float ck[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ck[i] = KSCALE ? sl2 * sm.kscale[(kt + t) & 7][i] : sl2;
         // the whole row of S into registers: four loads in flight, one wait
         uint32_t sv[kTileN];
         auto load_row = [&]() {
@@ -665,8 +677,9 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
         };
         load_row();
         // row extremum of the raw scores; times sl2 it is the row maximum of the scaled scores
-        float ext;
-        {
+        float mx;
+        if (!KSCALE) {
+          float ext;
           float e8[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) e8[i] = __uint_as_float(sv[i]);
@@ -679,8 +692,27 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
             for (int i = 8; i < kTileN; ++i) e8[i & 7] = fminf(e8[i & 7], __uint_as_float(sv[i]));
             ext = fminf(fminf(fminf(e8[0], e8[1]), fminf(e8[2], e8[3])), fminf(fminf(e8[4], e8[5]), fminf(e8[6], e8[7])));
           }
+          mx = (ext == INFINITY || ext == -INFINITY) ? -INFINITY : ext * sl2;   // all masked -> -inf
+        } else {
+          // every page has a factor of its own: the extremum of each page's 16 raw scores, scaled, then the maximum
+          mx = -INFINITY;
+#pragma unroll
+          for (int pg = 0; pg < 8; ++pg) {
+            float e4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) e4[i] = __uint_as_float(sv[16 * pg + i]);
+            if (sl2 >= 0.f) {
+#pragma unroll
+              for (int i = 4; i < 16; ++i) e4[i & 3] = fmaxf(e4[i & 3], __uint_as_float(sv[16 * pg + i]));
+              e4[0] = fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]));
+            } else {
+#pragma unroll
+              for (int i = 4; i < 16; ++i) e4[i & 3] = fminf(e4[i & 3], __uint_as_float(sv[16 * pg + i]));
+              e4[0] = fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
+            }
+            if (e4[0] != INFINITY && e4[0] != -INFINITY) mx = fmaxf(mx, e4[0] * ck[pg]);   // (all 16 masked: skipped)
+          }
         }
-        const float mx = (ext == INFINITY || ext == -INFINITY) ? -INFINITY : ext * sl2;   // all masked -> -inf
         // The running maximum moves only when the new one is clearly larger (2^8): P stays bounded by
         // 2^8 and the accumulator in TMEM is rescaled rarely.
         float m_use = m;
@@ -720,8 +752,9 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           uint32_t pw[16];                 // 32 tokens -> 16 packed columns
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j]), sl2, neg_m));       // masked: exp2(-inf) = 0
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j + 1]), sl2, neg_m));
+            const float cf = ck[(c * 32 + 2 * j) >> 4];
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j]), cf, neg_m));       // masked: exp2(-inf) = 0
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c * 32 + 2 * j + 1]), cf, neg_m));
             lsum[j & 1] += p0;
             lsum[2 + (j & 1)] += p1;
             pw[j] = pack_bf16x2(p0, p1);
@@ -907,6 +940,7 @@ struct PrefixTcPlan {
   int n_items, grid;
   bool one_part_per_row;   // every row gets exactly one part from this pass: one single-split level, or two chained
   long long wait_cycles;   // limit of every device-side wait
+  const float *k_scale;    // non-null: the pools are an expanded e4m3 cache, one K scale per (page, kv head)
   int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
@@ -953,10 +987,11 @@ double lpt_assign(const std::vector<int> &by_cost, const std::vector<double> &co
 // roofline from the rest) whose most loaded CTA stays within `target_us` - or `fixed_ctas` CTAs if that is positive.  The lists stay
 // valid when the lengths change later; only their balance is the create-time one.  nullptr when unavailable.
 PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_levels, int sm_count, int fixed_ctas,
-                             double target_us, double tile_us, double item_us) {
+                             double target_us, double tile_us, double item_us, const float *k_scale) {
   if (n_levels < 1 || n_levels > kMaxTcLevels) return nullptr;
   PrefixTcPlan *plan = new PrefixTcPlan();
   plan->dev_lists = nullptr;
+  plan->k_scale = k_scale;
   plan->wait_cycles = wait_limit_cycles();
   const Params &p = levels[0];
   if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
@@ -1096,7 +1131,9 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     const int it = by_cost[i];
     lists[(size_t)grid + 1 + (size_t)fill[(size_t)owner[(size_t)it]]++] = it;
   }
-  if (cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(prefix_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sizeof(Smem)) != cudaSuccess ||
+      cudaFuncSetAttribute(prefix_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sizeof(Smem)) != cudaSuccess ||
       cudaMalloc(&plan->dev_lists, sizeof(int32_t) * lists.size()) != cudaSuccess ||
       cudaMemcpy(plan->dev_lists, lists.data(), sizeof(int32_t) * lists.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -1133,9 +1170,10 @@ mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const vo
   cfg.attrs = &attr;
   cfg.numAttrs = beside_previous ? 1 : 0;
   const cudaError_t e = cudaLaunchKernelEx(
-      &cfg, prefix_tc_kernel, p, plan->levels, plan->k_map, plan->v_map, reinterpret_cast<const __nv_bfloat16 *>(q),
-      scale * kLog2e, o_part, lse_part, (const int32_t *)(plan->dev_lists + plan->grid + 1),
-      (const int32_t *)plan->dev_lists, reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles);
+      &cfg, plan->k_scale ? prefix_tc_kernel<true> : prefix_tc_kernel<false>, p, plan->levels, plan->k_map, plan->v_map,
+      reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
+      (const int32_t *)(plan->dev_lists + plan->grid + 1), (const int32_t *)plan->dev_lists,
+      reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles, plan->k_scale);
   count_launch();
   return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }

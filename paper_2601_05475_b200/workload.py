@@ -122,6 +122,9 @@ CONFIGS: Dict[str, Config] = {
     # long-reasoning rollouts (extended-thinking critiques)
     "cfg4": Config("cfg4", "bf16", 4, 32, 64, 8, 128, ("fixed", 4096), ("uniform", 16384, 32768),
                    permute_pages=True, append_steps=64),
+    # cfg4 over an e4m3 cache with per-(page, kv head) scales: half the bytes per cached token
+    "cfg4_fp8": Config("cfg4_fp8", "fp8", 4, 32, 64, 8, 128, ("fixed", 4096), ("uniform", 16384, 32768),
+                       permute_pages=True, append_steps=64),
     # one of cfg4's four prompt groups alone (3.2 GB): the same chunk geometry at a size a profiler can replay
     "cfg4g1": Config("cfg4g1", "bf16", 1, 32, 64, 8, 128, ("fixed", 4096), ("uniform", 16384, 32768),
                      permute_pages=True, append_steps=64),

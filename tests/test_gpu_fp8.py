@@ -65,18 +65,50 @@ CASES = {
 }
 
 
+@pytest.mark.parametrize("tc", ["1", "0"])
 @pytest.mark.parametrize("name", list(CASES))
-def test_fp8_decode_matches_oracle(name):
+def test_fp8_decode_matches_oracle(name, tc, monkeypatch):
+    """tc = 1: the prefix levels run on the tensor-core pass over their widened copy (where the shape allows it);
+    tc = 0: every candidate streams its group's e4m3 pages itself."""
+    monkeypatch.setenv("MC_PREFIX_TC", tc)
     cfg, outer = CASES[name]
     fp = make_fp8(cfg, outer)
     dp = device_problem(fp)
     scratch = torch.empty(fp.tables.num_pages, dtype=torch.int32, device="cuda")
     assert mc.mc_kv_layout_validate(dp.layout, scratch, scratch.numel() * 4) == mc.MC_OK
+    assert (dp.geom.prefix_ctas > 0) == (tc == "1")
     q = wl.draw_q(cfg, 0)
     o, lse = dp.decode(to_device(cfg, q))
     torch.cuda.synchronize()
     assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
     check(o, lse, *oracle(fp, q))
+    dp.close()
+
+
+def test_fp8_prefix_changes_take_effect_after_a_refresh():
+    """The tensor-core prefix pass reads a widened copy of the prefix made when the layout was created: after the
+    prefix pages change, mc_kv_layout_refresh_prefix brings the copy up to date."""
+    cfg, _ = CASES["cfg2s"]
+    fp = make_fp8(cfg)
+    dp = device_problem(fp)
+    assert dp.geom.prefix_ctas > 0
+    q = wl.draw_q(cfg, 0)
+    qd = to_device(cfg, q)
+    dp.decode(qd)
+    torch.cuda.synchronize()
+    check(dp.o, dp.lse, *oracle(fp, q))
+    # the first three prefix pages get V = 0 (code 0) and K scales twice as large
+    for i in range(3):
+        pid = int(fp.tables.prefix_pages[0, i])
+        dp.v_pool[pid] = 0
+        dp.k_scale[pid] *= 2
+        fp.v_prefix[0][16 * i:16 * i + 16] = 0.0
+        fp.k_prefix[0][16 * i:16 * i + 16] *= 2.0
+    mc.mc_kv_layout_refresh_prefix(dp.layout)
+    dp.decode(qd)
+    torch.cuda.synchronize()
+    assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+    check(dp.o, dp.lse, *oracle(fp, q))
     dp.close()
 
 
