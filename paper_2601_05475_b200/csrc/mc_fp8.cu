@@ -29,7 +29,9 @@ namespace {
 
 constexpr int D = 128;
 constexpr int kW = 2;                      // warps (items) per CTA
-constexpr int kStages = 8;                 // page stages per warp: two being computed, six in flight
+constexpr int kStages = 4;                 // page stages per warp: two being computed, two in flight (32 KB a CTA, six CTAs
+                                           // = twelve warps per SM; measured against 6 and 8 stages with 4 and 3 CTAs:
+                                           // cfg4 suffix pass 951 : 968 : 962 us, whole step 1003 : 1018 : 1095 us)
 constexpr uint32_t kSlabBytes = kPage * D;           // one (page, kv head) slab of K or of V: 2 KB
 constexpr uint32_t kStageBytes = 2 * kSlabBytes;
 constexpr long long kDrainCycles = 2000000ll;        // ~1 ms: what a warp that gives up grants its copies in flight
