@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # 4096-token chunks on a small problem of cfg4's shape; the traffic grows in proportion to the tokens streamed,
 # so the ratio is scaled by the units of the timed workload).  A ratio is only reported while the kernel source
 # still has the hash it had when the counters were taken.
-SUFFIX_TRAFFIC_RATIO = {"short_chunks": None, "long_chunks": None}
-SUFFIX_KERNEL_SHA1 = ""
+SUFFIX_TRAFFIC_RATIO = {"short_chunks": 1.0130, "long_chunks": 1.0025}
+SUFFIX_KERNEL_SHA1 = "071b4e65961c357d4e4d7980d6c287aa4388286a"
 
 
 def suffix_traffic(algorithmic_bytes, suffix_part_tokens):
@@ -524,6 +524,9 @@ def run_gpu(args):
 
     if args.pass_only:         # profiling aid: one pass alone on the launching stream, one small JSON line
         cfg = wl.CONFIGS[args.workload]
+        if args.kv_dtype:
+            import dataclasses
+            cfg = dataclasses.replace(cfg, dtype=args.kv_dtype)
         dp = make_device_problem(cfg, headroom_tokens=1)
         g = dp.geom
         lse_off = (g.rows * g.n_parts * g.head_dim * 4 + 255) // 256 * 256
@@ -555,7 +558,7 @@ def run_gpu(args):
             print(json.dumps({"scoring_attention": measure_scoring()}))
         return 0
 
-    main = measure(args.workload, args.steps, args.warmup, True, min_seconds=1.0)
+    main = measure(args.workload, args.steps, args.warmup, True, min_seconds=args.min_seconds)
     others = {}
     cold = None
     if args.all_configs:
@@ -673,6 +676,10 @@ def main():
     ap.add_argument("--scoring-only", action="store_true", help="run only the scoring pass (profiling aid)")
     ap.add_argument("--pass-only", choices=["suffix", "prefix"], default=None,
                     help="run only that pass of --workload, alone (profiling aid)")
+    ap.add_argument("--kv-dtype", choices=["bf16", "fp8"], default=None,
+                    help="with --pass-only: the cache type, if not the workload's own")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="repeat the block of --steps steps until this much device time has been timed (0: one block)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
                     help="time only --workload (default: also cfg2/cfg3/cfg4 summaries under per_config)")
     args = ap.parse_args()

@@ -187,6 +187,23 @@ mc_status_t mc_kv_append(mc_kv_layout_t *layout, const void *k_new, const void *
 mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const void *v_new, void *q,
                               const int32_t *pos_offset, double theta_base, void *stream);
 
+/* Appends up to n_max tokens per candidate in one call (ingesting a prompt or a candidate's whole continuation
+ * before it is scored - the value model of Section 2.3, "Generative Value Function Guided Search", reads every
+ * candidate in full - or storing several speculated tokens):
+ *   k_new, v_new  device [B][n_max][Hkv][d], of the type mc_kv_append takes
+ *   n_new         device int32 [B] or NULL: candidate b gets its first min(max(n_new[b], 0), n_max) tokens; NULL: n_max
+ * Token t of candidate b lands at suffix position suffix_len[b] + t; then suffix_len[b] grows by the count, on the
+ * device.  A candidate whose tokens do not all fit its page row is left unchanged and MC_ERR_INVALID_ARG is latched.
+ * theta_base > 0 rotates the keys as mc_kv_append_rope does, token t to position (tokens in front of the candidate's
+ * suffix, or pos_offset[b]) + suffix_len[b] + t, and, when q (device [B][n_max][Hq][d]) is given, the query rows of
+ * the same tokens in place; theta_base = 0 stores the keys as they are (q and pos_offset must then be NULL).
+ * An MC_FP8_E4M3 cache is written as by successive mc_kv_append calls (a page's scales come from the token that
+ * opens it, whether that token is part of this call or was stored before); the rotation is not available on it.
+ * n_max <= 65535.  Two launches; asynchronous on `stream`. */
+mc_status_t mc_kv_append_tokens(mc_kv_layout_t *layout, const void *k_new, const void *v_new, int32_t n_max,
+                                const int32_t *n_new, void *q, const int32_t *pos_offset, double theta_base,
+                                void *stream);
+
 /* Prefix pass: for every group and kv head, the stacked queries of all the group's candidates attend
  * to the group's prefix; writes parts [0, n_prefix_parts) of every row.  q: device [B][Hq][d]. */
 mc_status_t mc_prefix_attn(mc_kv_layout_t *layout, const void *q, float scale,

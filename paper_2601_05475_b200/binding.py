@@ -45,6 +45,8 @@ EXPORTS = {
     "mc_workspace_bytes": (c_size_t, [c_void_p]),
     "mc_kv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
     "mc_kv_append_rope": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_double, c_void_p]),
+    "mc_kv_append_tokens": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_double,
+                                      c_void_p]),
     "mc_prefix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
     "mc_suffix_attn": (c_int32, [c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p]),
     "mc_merge_lse": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -156,6 +158,12 @@ def mc_kv_append(layout: int, k_new, v_new, stream: int = 0) -> None:
 def mc_kv_append_rope(layout: int, k_new, v_new, q, pos_offset, theta_base: float, stream: int = 0) -> None:
     _check(lib().mc_kv_append_rope(layout, _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(pos_offset), theta_base, stream),
            "mc_kv_append_rope")
+
+
+def mc_kv_append_tokens(layout: int, k_new, v_new, n_max: int, n_new=None, q=None, pos_offset=None,
+                        theta_base: float = 0.0, stream: int = 0) -> None:
+    _check(lib().mc_kv_append_tokens(layout, _ptr(k_new), _ptr(v_new), n_max, _ptr(n_new), _ptr(q), _ptr(pos_offset),
+                                     theta_base, stream), "mc_kv_append_tokens")
 
 
 def mc_prefix_attn(layout: int, q, scale: float, o_part, lse_part, stream: int = 0) -> None:

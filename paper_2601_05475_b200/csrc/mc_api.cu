@@ -172,6 +172,101 @@ __global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels l
 }
 
 // ------------------------------------------------------------------------------------------------
+// append of several tokens per candidate (prompt ingestion, speculated tokens): block (t, b) stores token t of
+// candidate b at suffix position suffix_len[b] + t, rotated or not; the lengths move in a second launch, once every
+// row is in place.  A candidate whose tokens do not all fit its page row is left alone and reported.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int tokens_of(const int32_t *n_new, int b, int n_max) {
+  if (!n_new) return n_max;
+  const int n = __ldg(n_new + b);
+  return n < 0 ? 0 : n > n_max ? n_max : n;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) append_tokens_kernel(Params p, RopeLevels lv, const T *__restrict__ k_new,
+                                                            const T *__restrict__ v_new, T *q, int n_max,
+                                                            const int32_t *__restrict__ n_new,
+                                                            const int32_t *__restrict__ pos_offset, double log2_base,
+                                                            const int32_t *__restrict__ suffix_len) {
+  const int t = blockIdx.x, b = blockIdx.y;
+  const int n = tokens_of(n_new, b, n_max);
+  if (t >= n) return;
+  const int s0 = __ldg(suffix_len + b);
+  if (s0 < 0 || (long long)s0 + n > (long long)p.max_sp * kPage) {   // (reported by the kernel that moves the lengths)
+    return;
+  }
+  const int s = s0 + t;
+  const int page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + (s >> 4));
+  if ((unsigned)page >= (unsigned)p.num_pages) {
+    if (threadIdx.x == 0) latch(p, kDevBadPage);
+    return;
+  }
+  const size_t tok = (size_t)b * n_max + t;
+  const int row_vec = p.d * (int)sizeof(T) / 16, n_vec = p.Hkv * row_vec;
+  uint4 *vp = reinterpret_cast<uint4 *>(const_cast<void *>(p.v_pool));
+  const uint4 *vsrc = reinterpret_cast<const uint4 *>(v_new) + tok * n_vec;
+  for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
+    const int h = j / row_vec, cc = j % row_vec;
+    vp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = vsrc[j];
+  }
+  if (log2_base == 0.0) {   // keys as they are
+    uint4 *kp = reinterpret_cast<uint4 *>(const_cast<void *>(p.k_pool));
+    const uint4 *ksrc = reinterpret_cast<const uint4 *>(k_new) + tok * n_vec;
+    for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
+      const int h = j / row_vec, cc = j % row_vec;
+      kp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = ksrc[j];
+    }
+    return;
+  }
+  // rotary position embedding, as in append_rope_kernel: position = the tokens in front of this one
+  long long pos = s;
+  if (pos_offset) {
+    pos += __ldg(pos_offset + b);
+  } else {
+    for (int k = 0; k < lv.n; ++k) {
+      int lo = 0, hi = lv.G[k];
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(lv.group_offsets[k] + mid) <= b) lo = mid; else hi = mid;
+      }
+      pos += max(__ldg(lv.prefix_len[k] + lo), 0);
+    }
+  }
+  const int half = p.d / 2, lanes = blockDim.x / half;
+  const int i = threadIdx.x % half, h0 = threadIdx.x / half;
+  double sn, cs;
+  sincos((double)pos * exp2(-2.0 * i / p.d * log2_base), &sn, &cs);
+  const float c = (float)cs, sf = (float)sn;
+  T *kp = reinterpret_cast<T *>(const_cast<void *>(p.k_pool));
+  for (int h = h0; h < p.Hkv; h += lanes) {
+    const T *src = k_new + (tok * p.Hkv + h) * p.d;
+    T *dst = kp + (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * p.d;
+    const float re = rope_load(src + i), im = rope_load(src + i + half);
+    rope_store(dst + i, re * c - im * sf);
+    rope_store(dst + i + half, re * sf + im * c);
+  }
+  if (q)
+    for (int h = h0; h < p.Hq; h += lanes) {
+      T *row = q + (tok * p.Hq + h) * p.d;
+      const float re = rope_load(row + i), im = rope_load(row + i + half);
+      rope_store(row + i, re * c - im * sf);
+      rope_store(row + i + half, re * sf + im * c);
+    }
+}
+
+__global__ void advance_len_kernel(Params p, int n_max, const int32_t *__restrict__ n_new, int32_t *suffix_len) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= p.B) return;
+  const int n = tokens_of(n_new, b, n_max), s0 = suffix_len[b];
+  if (n == 0) return;
+  if (s0 < 0 || (long long)s0 + n > (long long)p.max_sp * kPage) {
+    latch(p, kDevBadPage);
+    return;
+  }
+  suffix_len[b] = s0 + n;
+}
+
+// ------------------------------------------------------------------------------------------------
 // validation
 // ------------------------------------------------------------------------------------------------
 __global__ void validate_kernel(Params p, int32_t *refs, int with_suffix) {
@@ -702,6 +797,49 @@ mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const v
     mc::append_rope_kernel<__nv_bfloat16><<<L->p.B, 256, 0, st>>>(
         L->p, lv, reinterpret_cast<const __nv_bfloat16 *>(k_new), reinterpret_cast<const uint4 *>(v_new),
         reinterpret_cast<__nv_bfloat16 *>(q), pos_offset, l2b, L->desc.suffix_len);
+  mc::count_launch();
+  return mc::check_launch();
+}
+
+mc_status_t mc_kv_append_tokens(mc_kv_layout_t *layout, const void *k_new, const void *v_new, int32_t n_max,
+                                const int32_t *n_new, void *q, const int32_t *pos_offset, double theta_base,
+                                void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !k_new || !v_new || !mc::aligned16(k_new) || !mc::aligned16(v_new) || (q && !mc::aligned16(q)))
+    return MC_ERR_INVALID_ARG;
+  if (!L->has_suffix || n_max < 0 || n_max > 65535 || theta_base < 0.0) return MC_ERR_INVALID_ARG;
+  if (theta_base == 0.0 && (q || pos_offset)) return MC_ERR_INVALID_ARG;   // they belong to the rotation
+  if (theta_base > 0.0 && (L->p.d % 2 != 0 || 256 % (L->p.d / 2) != 0)) return MC_ERR_INVALID_ARG;
+  if (n_max == 0) return MC_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (L->fp8) {
+    if (theta_base > 0.0) return MC_ERR_UNSUPPORTED;   // the rotary append does not quantise
+    const mc_status_t s = mc::launch_append_tokens_fp8(L->p, k_new, v_new, n_max, n_new, L->desc.suffix_len, st);
+    if (s != MC_OK) return s;
+  } else {
+    mc::RopeLevels lv;
+    lv.n = 1 + L->n_outer;
+    for (int k = 0; k < lv.n; ++k) {
+      const mc::Params &pk = k == 0 ? L->p : L->outer_p[k - 1];
+      lv.G[k] = pk.G;
+      lv.group_offsets[k] = pk.group_offsets;
+      lv.prefix_len[k] = pk.prefix_len;
+    }
+    const double l2b = theta_base > 0.0 ? std::log2(theta_base) : 0.0;
+    if (theta_base == 1.0) return MC_ERR_INVALID_ARG;   // log2 = 0 is the "no rotation" mark (and base 1 rotates every pair alike)
+    const dim3 grid((unsigned)n_max, (unsigned)L->p.B);
+    if (L->desc.dtype == MC_F32)
+      mc::append_tokens_kernel<float><<<grid, 256, 0, st>>>(L->p, lv, reinterpret_cast<const float *>(k_new),
+                                                            reinterpret_cast<const float *>(v_new),
+                                                            reinterpret_cast<float *>(q), n_max, n_new, pos_offset, l2b,
+                                                            L->desc.suffix_len);
+    else
+      mc::append_tokens_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+          L->p, lv, reinterpret_cast<const __nv_bfloat16 *>(k_new), reinterpret_cast<const __nv_bfloat16 *>(v_new),
+          reinterpret_cast<__nv_bfloat16 *>(q), n_max, n_new, pos_offset, l2b, L->desc.suffix_len);
+    mc::count_launch();
+  }
+  mc::advance_len_kernel<<<(L->p.B + 255) / 256, 256, 0, st>>>(L->p, n_max, n_new, L->desc.suffix_len);
   mc::count_launch();
   return mc::check_launch();
 }

@@ -510,6 +510,60 @@ __global__ void __launch_bounds__(256) append_fp8_kernel(Params p, const __nv_bf
   if (threadIdx.x == 0) suffix_len[b] = s + 1;
 }
 
+// Several tokens per candidate: block (t, b) quantises token t of candidate b for suffix position s = len + t.  The
+// scale of its page is the one the page's opening token fixes: its own row when it opens the page (it also stores
+// the scale), the row of the batch's token that does when that token is part of this call, else the stored one.  The
+// lengths move in a second launch.
+__global__ void __launch_bounds__(256)
+append_tokens_fp8_kernel(Params p, const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
+                         int n_max, const int32_t *__restrict__ n_new, const int32_t *__restrict__ suffix_len,
+                         float *k_scale, float *v_scale) {
+  const int t = blockIdx.x, b = blockIdx.y;
+  int n = n_max;
+  if (n_new) {
+    n = __ldg(n_new + b);
+    n = n < 0 ? 0 : n > n_max ? n_max : n;
+  }
+  if (t >= n) return;
+  const int s0 = __ldg(suffix_len + b);
+  if (s0 < 0 || (long long)s0 + n > (long long)p.max_sp * kPage) return;   // (reported when the lengths move)
+  const int s = s0 + t, slot = s & 15;
+  const int page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + (s >> 4));
+  if ((unsigned)page >= (unsigned)p.num_pages) {
+    if (threadIdx.x == 0) latch(p, kDevBadPage);
+    return;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t_open = t - slot;   // the batch's token that opens this page, if it is in the batch
+  uint8_t *kp = reinterpret_cast<uint8_t *>(const_cast<void *>(p.k_pool));
+  uint8_t *vp = reinterpret_cast<uint8_t *>(const_cast<void *>(p.v_pool));
+  for (int h = warp; h < p.Hkv; h += 8) {
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+      const __nv_bfloat16 *base = (which ? v_new : k_new) + ((size_t)b * n_max * p.Hkv + h) * D + 4 * lane;
+      const uint2 w = *reinterpret_cast<const uint2 *>(base + (size_t)t * p.Hkv * D);
+      const float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
+      const float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
+      float *scale_ptr = (which ? v_scale : k_scale) + (size_t)page * p.Hkv + h;
+      float scale;
+      if (t_open >= 0) {
+        const uint2 o = *reinterpret_cast<const uint2 *>(base + (size_t)t_open * p.Hkv * D);
+        float amax = fmaxf(fmaxf(fabsf(__uint_as_float(o.x << 16)), fabsf(__uint_as_float(o.x & 0xffff0000u))),
+                           fmaxf(fabsf(__uint_as_float(o.y << 16)), fabsf(__uint_as_float(o.y & 0xffff0000u))));
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, sh));
+        scale = amax > 0.f ? __fdiv_rn(amax * 2.f, 448.f) : 1.f;
+        if (slot == 0 && lane == 0) *scale_ptr = scale;
+      } else {
+        scale = *scale_ptr;
+      }
+      const uint32_t codes = encode4(__fdiv_rn(x0, scale), __fdiv_rn(x1, scale), __fdiv_rn(x2, scale), __fdiv_rn(x3, scale));
+      uint8_t *dst = (which ? vp : kp) + (((size_t)page * p.Hkv + h) * kPage + slot) * D + 4 * lane;
+      *reinterpret_cast<uint32_t *>(dst) = codes;
+    }
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -653,6 +707,15 @@ mc_status_t launch_fp8(const Params &p, const Fp8Plan *plan, int mode, const voi
                                            plan->wait_cycles);
   count_launch();
   return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
+}
+
+mc_status_t launch_append_tokens_fp8(const Params &p, const void *k_new, const void *v_new, int n_max,
+                                     const int32_t *n_new, const int32_t *suffix_len, cudaStream_t stream) {
+  append_tokens_fp8_kernel<<<dim3((unsigned)n_max, (unsigned)p.B), 256, 0, stream>>>(
+      p, reinterpret_cast<const __nv_bfloat16 *>(k_new), reinterpret_cast<const __nv_bfloat16 *>(v_new), n_max, n_new,
+      suffix_len, const_cast<float *>(p.k_scale), const_cast<float *>(p.v_scale));
+  count_launch();
+  return check_launch();
 }
 
 mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_new, int32_t *suffix_len,

@@ -148,5 +148,7 @@ const float *fp8_expanded_k_scale(const Fp8Plan *plan);
 mc_status_t fp8_expand_launch(const Fp8Plan *plan, const Params *levels, int n_levels, cudaStream_t stream);
 mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_new, int32_t *suffix_len,
                               cudaStream_t stream);
+mc_status_t launch_append_tokens_fp8(const Params &p, const void *k_new, const void *v_new, int n_max,
+                                     const int32_t *n_new, const int32_t *suffix_len, cudaStream_t stream);
 
 }  // namespace mc
