@@ -193,7 +193,8 @@ mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const v
  *   k_new, v_new  device [B][n_max][Hkv][d], of the type mc_kv_append takes
  *   n_new         device int32 [B] or NULL: candidate b gets its first min(max(n_new[b], 0), n_max) tokens; NULL: n_max
  * Token t of candidate b lands at suffix position suffix_len[b] + t; then suffix_len[b] grows by the count, on the
- * device.  A candidate whose tokens do not all fit its page row is left unchanged and MC_ERR_INVALID_ARG is latched.
+ * device.  A candidate whose tokens do not all fit its page row, or whose row lacks a valid page id for one of them,
+ * keeps its length (rows of it may have been written beyond that length) and MC_ERR_INVALID_ARG is latched.
  * theta_base > 0 rotates the keys as mc_kv_append_rope does, token t to position (tokens in front of the candidate's
  * suffix, or pos_offset[b]) + suffix_len[b] + t, and, when q (device [B][n_max][Hq][d]) is given, the query rows of
  * the same tokens in place; theta_base = 0 stores the keys as they are (q and pos_offset must then be NULL).

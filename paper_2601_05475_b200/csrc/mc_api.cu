@@ -259,7 +259,10 @@ __global__ void advance_len_kernel(Params p, int n_max, const int32_t *__restric
   if (b >= p.B) return;
   const int n = tokens_of(n_new, b, n_max), s0 = suffix_len[b];
   if (n == 0) return;
-  if (s0 < 0 || (long long)s0 + n > (long long)p.max_sp * kPage) {
+  bool fits = s0 >= 0 && (long long)s0 + n <= (long long)p.max_sp * kPage;
+  for (int pg = s0 >> 4; fits && pg <= (s0 + n - 1) >> 4; ++pg)   // every page the new tokens need is there
+    fits = (unsigned)__ldg(p.suffix_pages + (size_t)b * p.max_sp + pg) < (unsigned)p.num_pages;
+  if (!fits) {
     latch(p, kDevBadPage);
     return;
   }

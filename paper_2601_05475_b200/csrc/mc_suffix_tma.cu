@@ -52,12 +52,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false once `limit` cycles have passed (MC_ERR_TIMEOUT is latched).
+// The same test without suspension: returns at once.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false once `limit` cycles have passed (MC_ERR_TIMEOUT is latched).  A limit shorter than the
+// time the hardware may keep a thread suspended inside try_wait is honoured by polling without suspension.
 __device__ __forceinline__ bool mbar_wait(const Params &p, uint64_t *bar, uint32_t parity, long long limit) {
-  if (mbar_try_wait(bar, parity)) return true;
+  const bool polled = limit < 2000000ll;
+  if (polled ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (polled ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if (clock64() - t0 > limit) {
       latch(p, kDevTimeout);
       return false;

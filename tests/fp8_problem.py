@@ -45,21 +45,26 @@ class Fp8HostProblem:
             scale[pid] = sc[pg]
         return fp8.dequantise_sequence(codes, sc)
 
+    def append_one(self, b, k_row, v_row):
+        """One token of candidate b (k_row, v_row [Hkv][d]), as the library stores it: slot 0 of a page fixes the
+        page's scales."""
+        s = int(self.suffix_len[b])
+        pid, slot = int(self.tables.suffix_pages[b, s // wl.PAGE]), s % wl.PAGE
+        for new, pool, scale, logical in ((k_row, self.k_pool, self.k_scale, self.k_suffix),
+                                          (v_row, self.v_pool, self.v_scale, self.v_suffix)):
+            row = np.zeros((1, self.cfg.Hkv, self.cfg.d), dtype=np.float64)
+            for h in range(self.cfg.Hkv):
+                if slot == 0:
+                    scale[pid, h] = fp8.page_scale(new[h])
+                pool[pid, h, slot] = fp8.quantise_rows(new[h][None], scale[pid, h])[0]
+                row[0, h] = fp8.dequantise(pool[pid, h, slot], scale[pid, h])
+            logical[b] = np.concatenate([logical[b], row], axis=0)
+        self.suffix_len[b] = s + 1
+
     def append(self, k_new, v_new):
-        """One token per candidate, as mc_kv_append stores it: slot 0 of a page fixes the page's scales."""
+        """One token per candidate (k_new, v_new [B][Hkv][d]), as mc_kv_append stores it."""
         for b in range(self.cfg.B):
-            s = int(self.suffix_len[b])
-            pid, slot = int(self.tables.suffix_pages[b, s // wl.PAGE]), s % wl.PAGE
-            for new, pool, scale, logical in ((k_new, self.k_pool, self.k_scale, self.k_suffix),
-                                              (v_new, self.v_pool, self.v_scale, self.v_suffix)):
-                row = np.zeros((1, self.cfg.Hkv, self.cfg.d), dtype=np.float64)
-                for h in range(self.cfg.Hkv):
-                    if slot == 0:
-                        scale[pid, h] = fp8.page_scale(new[b, h])
-                    pool[pid, h, slot] = fp8.quantise_rows(new[b, h][None], scale[pid, h])[0]
-                    row[0, h] = fp8.dequantise(pool[pid, h, slot], scale[pid, h])
-                logical[b] = np.concatenate([logical[b], row], axis=0)
-            self.suffix_len[b] = s + 1
+            self.append_one(b, k_new[b], v_new[b])
 
 
 def make(cfg: wl.Config, outer=(), **kw) -> Fp8HostProblem:
