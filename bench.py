@@ -452,9 +452,10 @@ def run_gpu(args):
 
     def measure_search():
         """The search bookkeeping on 2^17 problems x 8 trajectories x 8 steps (Section 3.1: K = 8, depth 8): one pass
-        = rewards / best-so-far / value targets / labels / returns, value head, selection of tau* and of the state
-        to expand.  Algorithmic bytes per (trajectory, step): 5 read + 10 written; per trajectory 4 (length) +
-        4 (return) + 20 (logits) + 4 (expected) + 2 x 4 re-read by the two selections."""
+        = rewards / best-so-far / value targets / labels / returns (mc_search_returns), then value head, selection of
+        tau* and of the state to expand in one launch (mc_search_select).  Algorithmic bytes per (trajectory, step):
+        5 read + 10 written; per trajectory 4 (length) + 4 (return, written) + 20 (logits) + 4 (expected) + 4 (return,
+        read by the selection)."""
         b = wl.draw_search_batch(problems=1 << 17, K=8, T=8, seed=0)
         N, T, P = b["N"], b["T"], b["P"]
         dev = lambda a: torch.from_numpy(a).cuda()
@@ -467,25 +468,34 @@ def run_gpu(args):
         s1, s2, s3 = wl.SEARCH_THRESHOLDS
         stream = torch.cuda.current_stream().cuda_stream
 
-        def one():
+        def returns():
             mc.mc_search_returns(sp, ok, ln, N, T, s1, s2, s3, 0.95, r, u, v, lab, G, stream)
-            mc.mc_search_value_head(lg, N, None, ev, stream)
-            mc.mc_search_group_argmax(G, go, P, best_t, stream)
-            mc.mc_search_group_argmax(ev, go, P, best_s, stream)
 
-        for _ in range(3):
-            one()
-        total, reps = 0.0, 10
-        for _ in range(reps):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            one()
-            e1.record()
-            torch.cuda.synchronize()
-            total += e0.elapsed_time(e1)
-        ms = total / reps
-        nbytes = N * T * 15 + N * (4 + 4 + 20 + 4 + 8) + 2 * P * 8
+        def select():
+            mc.mc_search_select(lg, G, go, P, None, ev, best_t, best_s, stream)
+
+        def one():
+            returns()
+            select()
+
+        def timed(fn, reps=10):
+            for _ in range(3):
+                fn()
+            total = 0.0
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                total += e0.elapsed_time(e1)
+            return total / reps
+
+        ms, ms_returns, ms_select = timed(one), timed(returns), timed(select)
+        nbytes = N * T * 15 + N * (4 + 4 + 20 + 4 + 4) + 2 * P * 8
         return {"trajectories": N, "steps": T, "ms": round(ms, 5), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                "launches": 2, "ms_returns_alone": round(ms_returns, 5), "ms_select_alone": round(ms_select, 5),
+                "gbs_returns_alone": round((N * T * 15 + N * 8) / (ms_returns * 1e-3) / 1e9, 1),
                 "algorithmic_bytes": nbytes, "trajectory_steps_per_s": round(N * T / (ms * 1e-3), 1),
                 "l2": "arrays of one pass (170 MB) larger than L2, no flush"}
 

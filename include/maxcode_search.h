@@ -55,6 +55,17 @@ mc_status_t mc_search_value_head(const float *logits, int32_t N, float *prob, fl
 mc_status_t mc_search_group_argmax(const float *values, const int32_t *group_offsets, int32_t P, int32_t *best,
                                    void *stream);
 
+/* mc_search_value_head and both uses of mc_search_group_argmax as ONE launch over groups (Section 2.3, "Generative
+ * Value Function Guided Search": the state with the highest mean value is expanded; Section 2.1: tau* has the highest
+ * return).  For every group j = entries group_offsets[j] .. group_offsets[j+1]-1:
+ *   logits        float [N][5]  ->  prob float [N][5] (may be NULL), expected float [N] (may be NULL)
+ *   best_expected int32 [P]     index of the group's largest mean (may be NULL)
+ *   traj_return   float [N]     ->  best_return int32 [P]: index of the group's largest return (both NULL or both given)
+ * Ties go to the smaller index, NaN is never selected, an empty group gives -1.  Entries outside every group are
+ * not visited (their prob / expected are not written).  group_offsets int32 [P+1], increasing. */
+mc_status_t mc_search_select(const float *logits, const float *traj_return, const int32_t *group_offsets, int32_t P,
+                             float *prob, float *expected, int32_t *best_return, int32_t *best_expected, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -65,6 +65,8 @@ EXPORTS = {
                                     c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "mc_search_value_head": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p, c_void_p]),
     "mc_search_group_argmax": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "mc_search_select": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   c_void_p]),
 }
 
 
@@ -228,3 +230,9 @@ def mc_search_value_head(logits, N: int, prob, expected, stream: int = 0) -> Non
 def mc_search_group_argmax(values, group_offsets, P: int, best, stream: int = 0) -> None:
     _check(lib().mc_search_group_argmax(_ptr(values), _ptr(group_offsets), P, _ptr(best), stream),
            "mc_search_group_argmax")
+
+
+def mc_search_select(logits, traj_return, group_offsets, P: int, prob=None, expected=None, best_return=None,
+                     best_expected=None, stream: int = 0) -> None:
+    _check(lib().mc_search_select(_ptr(logits), _ptr(traj_return), _ptr(group_offsets), P, _ptr(prob), _ptr(expected),
+                                  _ptr(best_return), _ptr(best_expected), stream), "mc_search_select")

@@ -1,4 +1,4 @@
-// bf16, d = 128, g <= 8: split-KV attention with one warp per (candidate, kv head, part).
+// bf16, d = 128 or 64, g <= 8: split-KV attention with one warp per (candidate, kv head, part).
 //
 // A warp streams its token range page by page (16 tokens).  Per page and kv head it reads the 4 KB K
 // slab and the 4 KB V slab exactly once with 128-bit loads straight into the register fragments of
@@ -19,7 +19,6 @@ namespace mc {
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int D = 128;
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -51,7 +50,8 @@ __device__ __forceinline__ uint64_t l2_stream_policy() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
   return pol;
 }
-// Asks L2 to fetch one 4 KB (page, kv head) slab; costs no registers and no shared memory.
+// Asks L2 to fetch one (page, kv head) slab; costs no registers and no shared memory.
+template <int D>
 __device__ __forceinline__ void l2_prefetch_slab(const void *p) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(p), "r"(kPage * D * 2) : "memory");
 }
@@ -67,24 +67,28 @@ __device__ __forceinline__ uint4 ld16(const uint4 *p, uint64_t policy) {
   return v;
 }
 
+// A row of D elements is D / 8 chunks of 16 bytes; NJ = D / 32 chunks per lane of a K row, NH = D / 64 of a V row.
+template <int D>
 struct PageRegs {
-  uint4 k[8];  // k[j]: row gid, chunk tig+4j;  k[4+j]: row gid+8, same chunk
-  uint4 v[8];  // v[2x], v[2x+1]: token {2tig, 2tig+1, 2tig+8, 2tig+9}[x], chunks gid and gid+8
+  static constexpr int NJ = D / 32, NH = D / 64;
+  uint4 k[2 * NJ];  // k[j]: row gid, chunk tig+4j;  k[NJ+j]: row gid+8, same chunk
+  uint4 v[4 * NH];  // v[NH x + half]: token {2tig, 2tig+1, 2tig+8, 2tig+9}[x], chunk gid + 8 half
 };
 
-template <bool STREAM>
-__device__ __forceinline__ void issue_loads(PageRegs &r, const uint4 *kslab, const uint4 *vslab, int gid, int tig,
+template <bool STREAM, int D>
+__device__ __forceinline__ void issue_loads(PageRegs<D> &r, const uint4 *kslab, const uint4 *vslab, int gid, int tig,
                                             uint64_t pol) {
+  constexpr int NJ = D / 32, NH = D / 64, ROW = D / 8;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    r.k[j] = ld16<STREAM>(kslab + gid * 16 + tig + 4 * j, pol);
-    r.k[4 + j] = ld16<STREAM>(kslab + (gid + 8) * 16 + tig + 4 * j, pol);
+  for (int j = 0; j < NJ; ++j) {
+    r.k[j] = ld16<STREAM>(kslab + gid * ROW + tig + 4 * j, pol);
+    r.k[NJ + j] = ld16<STREAM>(kslab + (gid + 8) * ROW + tig + 4 * j, pol);
   }
 #pragma unroll
   for (int x = 0; x < 4; ++x) {
     const int tok = 2 * tig + (x & 1) + (x >> 1) * 8;
-    r.v[2 * x] = ld16<STREAM>(vslab + tok * 16 + gid, pol);
-    r.v[2 * x + 1] = ld16<STREAM>(vslab + tok * 16 + gid + 8, pol);
+#pragma unroll
+    for (int half = 0; half < NH; ++half) r.v[NH * x + half] = ld16<STREAM>(vslab + tok * ROW + gid + 8 * half, pol);
   }
 }
 
@@ -92,19 +96,22 @@ __device__ __forceinline__ uint32_t word(const uint4 &v, int i) {
   return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
+template <int D>
 struct State {
   float m0, m1, l0, l1;  // heads 2tig and 2tig+1 (l: this lane's share)
-  float o[8][4];         // o[i]: head-dim tile i; [0],[1]: d = D_gid[2i], heads 2tig, 2tig+1; [2],[3]: D_gid[2i+1]
+  float o[D / 16][4];    // o[i]: head-dim tile i; [0],[1]: d = D_gid[2i], heads 2tig, 2tig+1; [2],[3]: D_gid[2i+1]
 };
 
 // One page: tokens [tok_base, tok_base+16), those at or beyond `hi` masked.
-__device__ __forceinline__ void compute_page(State &st, const PageRegs &r, const uint32_t (&qf)[4][4], float sl2,
-                                             int tok_base, int hi, int gid, int tig) {
+template <int D>
+__device__ __forceinline__ void compute_page(State<D> &st, const PageRegs<D> &r, const uint32_t (&qf)[D / 32][4],
+                                             float sl2, int tok_base, int hi, int gid, int tig) {
+  constexpr int NJ = D / 32, NH = D / 64;
   float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    mma16816(c, r.k[j].x, r.k[4 + j].x, r.k[j].y, r.k[4 + j].y, qf[j][0], qf[j][1]);
-    mma16816(c, r.k[j].z, r.k[4 + j].z, r.k[j].w, r.k[4 + j].w, qf[j][2], qf[j][3]);
+  for (int j = 0; j < NJ; ++j) {
+    mma16816(c, r.k[j].x, r.k[NJ + j].x, r.k[j].y, r.k[NJ + j].y, qf[j][0], qf[j][1]);
+    mma16816(c, r.k[j].z, r.k[NJ + j].z, r.k[j].w, r.k[NJ + j].w, qf[j][2], qf[j][3]);
   }
   const bool v0 = tok_base + gid < hi, v1 = tok_base + gid + 8 < hi;
   const float s00 = v0 ? c[0] * sl2 : -INFINITY, s01 = v0 ? c[1] * sl2 : -INFINITY;
@@ -125,24 +132,24 @@ __device__ __forceinline__ void compute_page(State &st, const PageRegs &r, const
   st.m0 = mn0;
   st.m1 = mn1;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
+  for (int i = 0; i < D / 16; ++i) {
     st.o[i][0] *= a0; st.o[i][1] *= a1; st.o[i][2] *= a0; st.o[i][3] *= a1;
   }
   const uint32_t pb0 = transpose8x8(pack_bf16x2(p00, p01));
   const uint32_t pb1 = transpose8x8(pack_bf16x2(p10, p11));
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
+  for (int half = 0; half < NH; ++half) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint32_t x0 = word(r.v[0 + half], i), y0 = word(r.v[2 + half], i);
-      const uint32_t x1 = word(r.v[4 + half], i), y1 = word(r.v[6 + half], i);
+      const uint32_t x0 = word(r.v[0 * NH + half], i), y0 = word(r.v[1 * NH + half], i);
+      const uint32_t x1 = word(r.v[2 * NH + half], i), y1 = word(r.v[3 * NH + half], i);
       mma16816(st.o[half * 4 + i], __byte_perm(x0, y0, 0x5410), __byte_perm(x0, y0, 0x7632),
                __byte_perm(x1, y1, 0x5410), __byte_perm(x1, y1, 0x7632), pb0, pb1);
     }
   }
 }
 
-template <int MODE>
+template <int MODE, int D>
 __device__ __forceinline__ void
 attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
               float *__restrict__ lse_part, int prefetch_pages) {
@@ -174,9 +181,9 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
     if (first_pg < p.max_sp) pid_first = __ldg(row_pages + first_pg);
     if (first_pg + 1 < p.max_sp) pid_second = __ldg(row_pages + first_pg + 1);
   }
-  uint32_t qf[4][4];
+  uint32_t qf[D / 32][4];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int j = 0; j < D / 32; ++j) {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (gid < p.g) v = __ldg(reinterpret_cast<const uint4 *>(q + ((size_t)b * p.Hq + (size_t)h * p.g + gid) * D) + tig + 4 * j);
     qf[j][0] = v.x; qf[j][1] = v.y; qf[j][2] = v.z; qf[j][3] = v.w;
@@ -188,11 +195,11 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
     if (lane < g) lse_part[(row0 + lane) * p.n_parts + sp.part] = -INFINITY;
     return;
   }
-  State st;
+  State<D> st;
   st.m0 = st.m1 = -INFINITY;
   st.l0 = st.l1 = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) st.o[i][0] = st.o[i][1] = st.o[i][2] = st.o[i][3] = 0.f;
+  for (int i = 0; i < D / 16; ++i) st.o[i][0] = st.o[i][1] = st.o[i][2] = st.o[i][3] = 0.f;
 
   const uint4 *kpool = reinterpret_cast<const uint4 *>(p.k_pool);
   const uint4 *vpool = reinterpret_cast<const uint4 *>(p.v_pool);
@@ -211,11 +218,11 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
   };
 
   const uint64_t pol = l2_stream_policy();
-  PageRegs ra, rb;
+  PageRegs<D> ra, rb;
   int hi_a, hi_b = 0;
   {
     const size_t s = slab_of(MODE == kSuffix ? pid_first : __ldg(sp.pages + pg_first), hi_a);
-    issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
+    issue_loads<STREAM, D>(ra, kpool + s, vpool + s, gid, tig, pol);
   }
   int pid_next = 0;
   if (pg_first + 1 < pg_end) pid_next = MODE == kSuffix ? pid_second : __ldg(sp.pages + pg_first + 1);
@@ -225,8 +232,8 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
   auto prefetch_page = [&](int pgi, int pid) {
     if (pgi < pg_end && (unsigned)pid < (unsigned)p.num_pages) {
       const size_t s = ((size_t)pid * p.Hkv + h) * kSlab;
-      l2_prefetch_slab(kpool + s);
-      l2_prefetch_slab(vpool + s);
+      l2_prefetch_slab<D>(kpool + s);
+      l2_prefetch_slab<D>(vpool + s);
     }
   };
   if (STREAM && lane < kPrefetch) {   // kPrefetch <= 32
@@ -241,14 +248,14 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
     if (STREAM && pf_pg < pg_end) pf_pid = __ldg(sp.pages + pf_pg);   // used at the end of the iteration
     if (has_b) {
       const size_t s = slab_of(pid_next, hi_b);
-      issue_loads<STREAM>(rb, kpool + s, vpool + s, gid, tig, pol);
+      issue_loads<STREAM, D>(rb, kpool + s, vpool + s, gid, tig, pol);
       if (pg + 2 < pg_end) pid_next2 = __ldg(sp.pages + pg + 2);
     }
     compute_page(st, ra, qf, sl2, pg * kPage, hi_a, gid, tig);
     if (has_b) {
       if (pg + 2 < pg_end) {
         const size_t s = slab_of(pid_next2, hi_a);
-        issue_loads<STREAM>(ra, kpool + s, vpool + s, gid, tig, pol);
+        issue_loads<STREAM, D>(ra, kpool + s, vpool + s, gid, tig, pol);
         if (pg + 3 < pg_end) pid_next = __ldg(sp.pages + pg + 3);
       }
       compute_page(st, rb, qf, sl2, (pg + 1) * kPage, hi_b, gid, tig);
@@ -273,7 +280,7 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
       const float inv = 1.f / l;
       float *dst = o_part + slot * D + 8 * gid;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      for (int half = 0; half < D / 64; ++half) {
         const float(*t)[4] = st.o + half * 4;
         float4 w0 = make_float4(t[0][e] * inv, t[0][e + 2] * inv, t[1][e] * inv, t[1][e + 2] * inv);
         float4 w1 = make_float4(t[2][e] * inv, t[2][e + 2] * inv, t[3][e] * inv, t[3][e + 2] * inv);
@@ -284,11 +291,11 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
   }
 }
 
-template <int MODE>
+template <int MODE, int D>
 __global__ void __launch_bounds__(kWarps * 32, 2)
 attn_mma_kernel(Params p, const __nv_bfloat16 *__restrict__ q, float sl2, float *__restrict__ o_part,
                 float *__restrict__ lse_part, int prefetch_pages) {
-  attn_mma_body<MODE>(p, q, sl2, o_part, lse_part, prefetch_pages);
+  attn_mma_body<MODE, D>(p, q, sl2, o_part, lse_part, prefetch_pages);
   // As the programmatic dependent of the prefix pass the suffix grid starts before that one ends; one thread of the
   // grid waits for the prerequisite grid before it exits, so that this grid - and the merge behind it - cannot
   // complete earlier.  Without a prerequisite the instruction returns at once.
@@ -312,7 +319,9 @@ static int suffix_prefetch_pages() {
 
 int mma_items_per_cta() { return kWarps; }
 
-bool mma_supported(const Params &p, int dtype) { return dtype == MC_BF16 && p.d == 128 && p.g >= 1 && p.g <= 8; }
+bool mma_supported(const Params &p, int dtype) {
+  return dtype == MC_BF16 && (p.d == 128 || p.d == 64) && p.g >= 1 && p.g <= 8;
+}
 
 mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, float *o_part, float *lse_part,
                        cudaStream_t stream, bool beside_previous) {
@@ -323,7 +332,8 @@ mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, fl
   const float sl2 = scale * kLog2e;
   const __nv_bfloat16 *qb = reinterpret_cast<const __nv_bfloat16 *>(q);
   if (mode == kPrefix) {
-    attn_mma_kernel<kPrefix><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, 0);
+    if (p.d == 128) attn_mma_kernel<kPrefix, 128><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, 0);
+    else attn_mma_kernel<kPrefix, 64><<<grid, kWarps * 32, 0, stream>>>(p, qb, sl2, o_part, lse_part, 0);
   } else {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -334,8 +344,8 @@ mc_status_t launch_mma(const Params &p, int mode, const void *q, float scale, fl
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = beside_previous ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, attn_mma_kernel<kSuffix>, p, qb, sl2, o_part, lse_part, suffix_prefetch_pages()) !=
-        cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, p.d == 128 ? attn_mma_kernel<kSuffix, 128> : attn_mma_kernel<kSuffix, 64>, p, qb, sl2,
+                           o_part, lse_part, suffix_prefetch_pages()) != cudaSuccess) {
       count_launch();
       return MC_ERR_CUDA;
     }

@@ -236,6 +236,66 @@ group_argmax_kernel(const float *__restrict__ values, const int32_t *__restrict_
   if (active && sub == 0) best[j] = bi;
 }
 
+// Value head and both selections of a group in one pass: eight lanes per group; every lane forms the value head of
+// its entries (softmax over the five class logits, its mean), keeps the best mean and the best return it has seen,
+// and the eight lanes reduce both (value, index) pairs.  Nothing is read twice and nothing needs a second launch.
+__device__ __forceinline__ void take_better(float &bv, int &bi, float v, int i) {
+  if (i >= 0 && (bi < 0 ? v == v : (v > bv || (v == bv && i < bi)))) {
+    bv = v;
+    bi = i;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+select_kernel(const float *__restrict__ logits, const float *__restrict__ traj_return,
+              const int32_t *__restrict__ group_offsets, int P, float *__restrict__ prob, float *__restrict__ expected,
+              int32_t *__restrict__ best_return, int32_t *__restrict__ best_expected) {
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long j = tid / kLanesPerGroup;
+  const int sub = (int)(tid % kLanesPerGroup);
+  const bool active = j < P;   // whole warps stay in the shuffles below
+  const int lo = active ? __ldg(group_offsets + j) : 0, hi = active ? __ldg(group_offsets + j + 1) : 0;
+  float ev = -INFINITY, gv = -INFINITY;
+  int ei = -1, gi = -1;
+  for (int i = lo + sub; i < hi; i += kLanesPerGroup) {
+    float z[5];
+#pragma unroll
+    for (int q = 0; q < 5; ++q) z[q] = __ldg(logits + (size_t)i * 5 + q);
+    const float mx = fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), z[4]);
+    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < 5; ++q) {
+      z[q] = expf(z[q] - mx);
+      sum += z[q];
+    }
+    const float inv = 1.f / sum;
+    float e = 0.f;
+#pragma unroll
+    for (int q = 0; q < 5; ++q) {
+      const float pq = z[q] * inv;
+      if (prob) prob[(size_t)i * 5 + q] = pq;
+      e = fmaf((float)q, pq, e);
+    }
+    if (expected) expected[i] = e;
+    if (e == e) take_better(ev, ei, e, i);                        // (indices rise: an equal value never replaces)
+    if (traj_return) {
+      const float g = __ldg(traj_return + i);
+      if (g == g) take_better(gv, gi, g, i);
+    }
+  }
+#pragma unroll
+  for (int sh = kLanesPerGroup / 2; sh >= 1; sh >>= 1) {
+    const float oev = __shfl_xor_sync(0xffffffffu, ev, sh), ogv = __shfl_xor_sync(0xffffffffu, gv, sh);
+    const int oei = __shfl_xor_sync(0xffffffffu, ei, sh), ogi = __shfl_xor_sync(0xffffffffu, gi, sh);
+    take_better(ev, ei, oev, oei);
+    take_better(gv, gi, ogv, ogi);
+  }
+  if (active && sub == 0) {
+    if (best_expected) best_expected[j] = ei;
+    if (best_return) best_return[j] = gi;
+  }
+}
+
 }  // namespace
 }  // namespace mc
 
@@ -284,6 +344,17 @@ mc_status_t mc_search_group_argmax(const float *values, const int32_t *group_off
   const long long threads = (long long)P * mc::kLanesPerGroup;
   mc::group_argmax_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       values, group_offsets, P, best);
+  mc::count_launch();
+  return mc::check_launch();
+}
+
+mc_status_t mc_search_select(const float *logits, const float *traj_return, const int32_t *group_offsets, int32_t P,
+                             float *prob, float *expected, int32_t *best_return, int32_t *best_expected, void *stream) {
+  if (!logits || !group_offsets || P < 1 || (!best_expected && !expected && !prob)) return MC_ERR_INVALID_ARG;
+  if ((best_return != nullptr) != (traj_return != nullptr)) return MC_ERR_INVALID_ARG;
+  const long long threads = (long long)P * mc::kLanesPerGroup;
+  mc::select_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      logits, traj_return, group_offsets, P, prob, expected, best_return, best_expected);
   mc::count_launch();
   return mc::check_launch();
 }

@@ -326,6 +326,28 @@ def test_several_row_tiles_and_several_prefix_splits(monkeypatch, root):
     dp.close()
 
 
+@pytest.mark.parametrize("g", [4, 8, 1])
+def test_bf16_head_dim_64_on_the_warp_level_tensor_path(g):
+    """bf16 with d = 64 runs both passes on the warp-level MMA kernel (the tcgen05 and TMA-fed kernels are d = 128
+    only): ragged prefixes, permuted pages, suffixes over several chunks, appends."""
+    cfg = wl.Config("d64", "bf16", 3, 4, 2 * g, 2, 64, ("loguniform", 90, 1500), ("uniform", 0, 700), permute_pages=True,
+                    append_steps=2, seed=21)
+    hp = wl.make_host_problem(cfg)
+    dp = DeviceProblem.from_host(hp)
+    assert dp.geom.prefix_ctas == 0
+    for step in range(3):
+        q = wl.draw_q(cfg, step)
+        if step:
+            k_new, v_new = wl.draw_append(cfg, step)
+            mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
+            hp.append(k_new, v_new)
+        o, lse = dp.decode(to_device(cfg, q))
+        torch.cuda.synchronize()
+        assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+        check_close(cfg, o, lse, *oracle_full(hp, q))
+    dp.close()
+
+
 def test_unequal_group_sizes():
     cfg = wl.Config("unequal", "bf16", 2, 2, 8, 2, 128, ("fixed", 0), ("fixed", (5, 40, 0, 100)), seed=4)
     hp = wl.make_host_problem(cfg, prefix_len=np.array([64, 200], dtype=np.int32))

@@ -119,6 +119,52 @@ def test_value_head_and_selection_match_oracle():
         assert ref_ev[best[j]] >= ref_ev[ref_best[j]] - 2e-5
 
 
+def test_fused_selection_matches_oracle_and_the_separate_calls():
+    """mc_search_select: value head, selection by mean value and selection by return in one launch."""
+    batch = wl.draw_search_batch(problems=70, K=8, T=8, seed=6)
+    N, P = batch["N"], batch["P"]
+    rng = np.random.default_rng(2)
+    G_np = (rng.integers(0, 5, size=N) * 0.9 ** rng.integers(0, 8, size=N)).astype(np.float32)             # many ties
+    go_np = batch["group_offsets"].copy()
+    go_np[3] = go_np[2]                                        # an empty group
+    logits, G, go = (torch.from_numpy(a).cuda() for a in (batch["logits"], G_np, go_np))
+    prob = torch.full((N, 5), -7.0, device="cuda")
+    ev = torch.full((N,), -7.0, device="cuda")
+    best_g, best_e = (torch.full((P,), -9, dtype=torch.int32, device="cuda") for _ in range(2))
+    mc.mc_search_select(logits, G, go, P, prob, ev, best_g, best_e)
+    torch.cuda.synchronize()
+    prob, ev_h = prob.cpu().numpy(), ev.cpu().numpy()
+    inside = np.zeros(N, dtype=bool)
+    for j in range(P):
+        inside[go_np[j]:go_np[j + 1]] = True
+    for n in range(N):
+        if inside[n]:
+            p, e = orc.value_head(batch["logits"][n].astype(np.float64))
+            np.testing.assert_allclose(prob[n], p, rtol=1e-5, atol=1e-7)
+            assert abs(ev_h[n] - e) <= 1e-5
+        else:                                                  # entries outside every group are not visited
+            assert ev_h[n] == -7.0
+    assert best_g.cpu().tolist() == orc.group_argmax(G_np, go_np).tolist()           # exact: the inputs are given
+    assert best_e.cpu().tolist() == orc.group_argmax(np.where(inside, ev_h, np.nan), go_np).tolist()
+    assert best_g.cpu().tolist()[2] == -1
+    # the separate calls give the same
+    ev2 = torch.empty((N,), device="cuda")
+    b2 = torch.empty((P,), dtype=torch.int32, device="cuda")
+    mc.mc_search_value_head(logits, N, None, ev2)
+    mc.mc_search_group_argmax(ev2, go, P, b2)
+    torch.cuda.synchronize()
+    assert torch.equal(b2, best_e) and torch.equal(ev2[torch.from_numpy(inside).cuda()], ev[torch.from_numpy(inside).cuda()])
+    # only the selection, nothing stored; and the host checks
+    best_only = torch.full((P,), -9, dtype=torch.int32, device="cuda")
+    mc.mc_search_select(logits, None, go, P, None, None, None, best_only)
+    torch.cuda.synchronize()
+    assert torch.equal(best_only, best_e)
+    with pytest.raises(mc.McError):
+        mc.mc_search_select(logits, G, go, P, None, ev, None, best_only)            # a return array without its output
+    with pytest.raises(mc.McError):
+        mc.mc_search_select(logits, None, go, P)                                     # nothing asked for
+
+
 def test_group_argmax_edge_cases():
     vals = torch.tensor([1.0, 3.0, 3.0, 2.0, float("nan"), -1.0, float("-inf")] + [0.5] * 70 + [9.0], device="cuda")
     go = torch.tensor([0, 4, 4, 6, 7, 78], dtype=torch.int32, device="cuda")
