@@ -1118,6 +1118,28 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
       if (lpt_assign(by_cost, cost, mid, nullptr) <= target_us) hi = mid; else lo = mid + 1;
     }
     grid = lo;
+    // A prefix pass that outlasts the suffix pass even on its full share of the SMs (long shared prompts, short
+    // private suffixes: the first steps of a round of rollouts) is what the step waits for: it may then have more
+    // CTAs, up to every SM.  Estimate of the step with g prefix CTAs: the prefix pass beside the suffix stream (a
+    // third longer than alone) against the suffix pass on the SMs that are left (it needs sm_count - cap of them to
+    // saturate HBM and slows in proportion below that); with every SM taken the two passes run one after the other.
+    const double suffix_us = target_us / 0.09;   // target_us is a tenth of nine tenths of the suffix pass's time
+    if (grid == cap && most > cap && target_us > 0.0) {
+      double best = lpt_assign(by_cost, cost, cap, nullptr) * 1.3;
+      if (best > suffix_us) {
+        const int step = most - cap > 32 ? 4 : 1;
+        for (int g = cap + step; g <= most; g = (g < most && g + step > most) ? most : g + step) {
+          const double load = lpt_assign(by_cost, cost, g, nullptr);
+          const double left = (double)(sm_count - g), sat = (double)(sm_count - cap);
+          const double est = left < 1.0 ? load + suffix_us
+                                        : std::max(load * 1.3, suffix_us * (left >= sat ? 1.0 : sat / left));
+          if (est < best * 0.98) {   // (a larger grid must earn its SMs)
+            best = est;
+            grid = g;
+          }
+        }
+      }
+    }
   }
   plan->grid = grid;
   plan->one_part_per_row = (n_levels == 1 && levels[0].n_prefix_parts == 1) || fine >= 0;
