@@ -350,7 +350,8 @@ mc_status_t mc_search_group_argmax(const float *values, const int32_t *group_off
 
 mc_status_t mc_search_select(const float *logits, const float *traj_return, const int32_t *group_offsets, int32_t P,
                              float *prob, float *expected, int32_t *best_return, int32_t *best_expected, void *stream) {
-  if (!logits || !group_offsets || P < 1 || (!best_expected && !expected && !prob)) return MC_ERR_INVALID_ARG;
+  if (!logits || !group_offsets || P < 1 || (!best_expected && !best_return && !expected && !prob))
+    return MC_ERR_INVALID_ARG;
   if ((best_return != nullptr) != (traj_return != nullptr)) return MC_ERR_INVALID_ARG;
   const long long threads = (long long)P * mc::kLanesPerGroup;
   mc::select_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(

@@ -161,6 +161,10 @@ def test_fused_selection_matches_oracle_and_the_separate_calls():
     assert torch.equal(best_only, best_e)
     with pytest.raises(mc.McError):
         mc.mc_search_select(logits, G, go, P, None, ev, None, best_only)            # a return array without its output
+    only_g = torch.full((P,), -9, dtype=torch.int32, device="cuda")
+    mc.mc_search_select(logits, G, go, P, None, None, only_g, None)                  # only tau*
+    torch.cuda.synchronize()
+    assert torch.equal(only_g, best_g)
     with pytest.raises(mc.McError):
         mc.mc_search_select(logits, None, go, P)                                     # nothing asked for
 
