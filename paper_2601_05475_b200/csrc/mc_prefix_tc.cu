@@ -23,6 +23,7 @@
 #include <algorithm>
 #include <cstdlib>
 #include <functional>
+#include <type_traits>
 #include <queue>
 #include <utility>
 #include <vector>
@@ -244,7 +245,8 @@ struct Item {
   const int32_t *pages2, *limits2;
 };
 
-__device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs, int item) {
+// `cand_per_unit`: candidates in one item's rows (one 128-row tile: 128 / g; a pair of row tiles: twice that)
+__device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs, int item, int cand_per_unit) {
   int l = 0;
   while (l + 1 < lvs.n && item >= lvs.lv[l].item_end) ++l;
   const TcLevel &L = lvs.lv[l];
@@ -272,9 +274,8 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
   if (L.row_limit) {
     // the limits do not decrease inside a group: no row of this tile sees beyond the limit of its last candidate
     it.limits = L.row_limit + it.b0;
-    const int cand_per_tile = kTileM / p.g;
-    const int last = min((it.mt + 1) * cand_per_tile, it.n_cand) - 1;
-    if (last >= it.mt * cand_per_tile) it.hi = min(it.hi, max(__ldg(it.limits + last), 0));
+    const int last = min((it.mt + 1) * cand_per_unit, it.n_cand) - 1;
+    if (last >= it.mt * cand_per_unit) it.hi = min(it.hi, max(__ldg(it.limits + last), 0));
   }
   it.lo2 = it.hi2 = 0;
   it.part2 = -1;
@@ -297,9 +298,8 @@ __device__ __forceinline__ Item decode_item(const Params &p, const TcLevels &lvs
     it.pages2 = C.prefix_pages + (size_t)lo * C.max_pp;
     if (C.row_limit) {
       it.limits2 = C.row_limit + it.b0;
-      const int cand_per_tile = kTileM / p.g;
-      const int last = min((it.mt + 1) * cand_per_tile, it.n_cand) - 1;
-      if (last >= it.mt * cand_per_tile) it.hi2 = min(it.hi2, max(__ldg(it.limits2 + last), 0));
+      const int last = min((it.mt + 1) * cand_per_unit, it.n_cand) - 1;
+      if (last >= it.mt * cand_per_unit) it.hi2 = min(it.hi2, max(__ldg(it.limits2 + last), 0));
     }
   }
   return it;
@@ -394,7 +394,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 
     auto next_item = [&](int from, Item &out) -> int {
       for (int k = from; k < k_end; ++k) {
-        out = decode_item(p, lvs, __ldg(item_list + k));
+        out = decode_item(p, lvs, __ldg(item_list + k), cand_per_tile);
         if (item_has_work(out, cand_per_tile)) return k;
       }
       return k_end;
@@ -514,7 +514,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
     if (lane == 0) {
       uint32_t team_tiles[kTeams] = {0u, 0u};   // tiles of each team whose P has been taken (all items)
       for (int k = k_begin; k < k_end && !sm.abort; ++k) {
-        const Item it = decode_item(p, lvs, __ldg(item_list + k));
+        const Item it = decode_item(p, lvs, __ldg(item_list + k), cand_per_tile);
         if (!item_has_work(it, cand_per_tile)) continue;
         const int qb = it_n & 1;
         if (!mbar_wait(sm, p, &sm.q_ready[qb], (it_n >> 1) & 1)) break;
@@ -591,7 +591,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       int k0 = k_begin;
       Item qi;
       for (; k0 < k_end; ++k0) {
-        qi = decode_item(p, lvs, __ldg(item_list + k0));
+        qi = decode_item(p, lvs, __ldg(item_list + k0), cand_per_tile);
         if (item_has_work(qi, cand_per_tile)) break;
       }
       if (k0 < k_end) {
@@ -619,7 +619,7 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
       }
     }
     for (int k = k_begin; k < k_end && !sm.abort; ++k) {
-      const Item it = decode_item(p, lvs, __ldg(item_list + k));
+      const Item it = decode_item(p, lvs, __ldg(item_list + k), cand_per_tile);
       if (it.mt * cand_per_tile >= it.n_cand) continue;
       const int cand = it.mt * cand_per_tile + r / g;
       const bool row_ok = cand < it.n_cand;
@@ -880,6 +880,498 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
 
 static_assert(sizeof(Smem) <= 232448, "shared memory of one CTA");
 
+// ================================================================================================
+// Row-pair variant.  Where a (group, kv head) has at least two 128-row tiles of stacked queries, an item covers
+// TWO of them and the CTA's two teams are the two row tiles: every K/V tile is copied into shared memory once and
+// read by both teams' products (half the copies and half the L2 reads of the variant above, where each row tile
+// streams the K/V tiles on its own), an item is twice as long (half the per-item cost), and each team owns its rows
+// from the first product to the stores (no merging of two streams in the epilogue).  The query tiles arrive by TMA
+// through a tensor map laid over q (box = 128 / g candidates x g heads x 64 elements, which IS the stacked row
+// order), so no thread stages them.  Per team the order on the tensor pipe is the same chain as above - S(t),
+// O += P(t) V(t), S(t+1) - and the other team's products fill the gaps.  With per-candidate limits (scoring) the
+// teams see different numbers of tiles; a tile's slot is released by the product of its last user.
+// ================================================================================================
+struct __align__(1024) SmemRp {
+  uint8_t q[kTeams][kTileBytes];      // team T's stacked query tile, [d half][128 rows][64], 128-byte swizzle
+  uint8_t k[kKSlots][kTileBytes];
+  uint8_t v[kVSlots][kTileBytes];
+  uint64_t full_k[kKSlots], empty_k[kKSlots], full_v[kVSlots], empty_v[kVSlots];
+  uint64_t q_full[kTeams], q_free[kTeams], s_full[kTeams], p_full[kTeams], pv_done[kTeams];
+  uint32_t page_ok[8];
+  float kscale[8][8];
+  uint32_t tmem_base;
+  volatile int abort;
+  long long wait_cycles;
+};
+
+__device__ __forceinline__ bool mbar_wait_rp(SmemRp &sm, const Params &p, uint64_t *bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(32);
+    if (sm.abort) return false;
+    if (clock64() - t0 > sm.wait_cycles) {
+      sm.abort = 1;
+      latch(p, kDevTimeout);
+      return false;
+    }
+  }
+}
+
+// One d half (64 elements) of a stacked query tile: 128 / g candidates x g heads x 64 elements, 16 KB.
+__device__ __forceinline__ void tma_load_q_half(void *dst, const CUtensorMap *map, int x, int head, int cand,
+                                                uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(head), "r"(cand), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// What one team (row tile 2 mp + T of the item's pair) sees of the item.
+struct TeamView {
+  bool rows;        // the row tile has candidates
+  int hi1, hi2;     // ends of the two token ranges for this tile's rows (its last candidate's limits applied)
+  int n1, n2;       // its tiles in the two ranges
+};
+__device__ __forceinline__ TeamView team_view(const Item &u, int T, int cand_per_tile) {
+  TeamView v;
+  const int first = (2 * u.mt + T) * cand_per_tile;
+  v.rows = first < u.n_cand;
+  const int last = min(first + cand_per_tile, u.n_cand) - 1;
+  v.hi1 = u.hi;
+  v.hi2 = u.hi2;
+  if (v.rows && u.limits) v.hi1 = min(v.hi1, max(__ldg(u.limits + last), 0));
+  if (v.rows && u.limits2) v.hi2 = min(v.hi2, max(__ldg(u.limits2 + last), 0));
+  v.n1 = v.rows ? tiles_of(u.lo, v.hi1) : 0;
+  v.n2 = v.rows ? tiles_of(u.lo2, v.hi2) : 0;
+  return v;
+}
+
+template <bool KSCALE>
+__global__ void __maxnreg__(168)
+prefix_rp_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_constant__ CUtensorMap k_map,
+                 const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap q_map, float sl2,
+                 float *__restrict__ o_part, float *__restrict__ lse_part, const int32_t *__restrict__ item_list,
+                 const int32_t *__restrict__ cta_begin, __nv_bfloat16 *__restrict__ o_final,
+                 float *__restrict__ lse_final, long long wait_cycles, const float *__restrict__ k_scale) {
+  const bool direct = o_final != nullptr;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  SmemRp &sm = *reinterpret_cast<SmemRp *>(smem_raw);
+  if ((smem_u32(smem_raw) & 1023u) != 0) {
+    if (threadIdx.x == 0) latch(p, MC_ERR_CUDA);
+    return;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = p.g, cand_per_tile = kTileM / g, cand_per_unit = 2 * cand_per_tile;
+  const int k_begin = __ldg(cta_begin + blockIdx.x), k_end = __ldg(cta_begin + blockIdx.x + 1);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kKSlots; ++s) {
+      mbar_init(&sm.full_k[s], 2);
+      mbar_init(&sm.empty_k[s], 1);
+    }
+    for (int s = 0; s < kVSlots; ++s) {
+      mbar_init(&sm.full_v[s], 1);
+      mbar_init(&sm.empty_v[s], 1);
+    }
+    for (int t = 0; t < kTeams; ++t) {
+      mbar_init(&sm.q_full[t], 1);
+      mbar_init(&sm.q_free[t], 1);
+      mbar_init(&sm.s_full[t], 1);
+      mbar_init(&sm.p_full[t], kSoftmaxThreads);
+      mbar_init(&sm.pv_done[t], 1);
+    }
+    sm.abort = 0;
+    sm.wait_cycles = wait_cycles;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+  if (threadIdx.x == kThreads - 1) {   // (see the kernel above: the append's completion, then the word to the suffix pass)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  }
+
+  // `kt` counts the K/V tiles of the CTA's stream (an item adds the tiles of the union of its two teams' ranges);
+  // every role advances it alike.
+  uint32_t kt = 0;
+
+  if (warp == 0 || warp >= 2 + kTeams * (kSoftmaxThreads / 32)) {
+    // ---------------------------------------------------------------- producers (three warps)
+    const int prole = warp == 0 ? 0 : warp - (1 + kTeams * (kSoftmaxThreads / 32));   // 0, 1: K d half; 2: V
+    const uint64_t policy = l2_keep_policy();
+    bool ok = true;
+    uint32_t q_n[kTeams] = {0u, 0u};   // items in which each team had tiles
+    for (int k = k_begin; k < k_end && ok && !sm.abort; ++k) {
+      const Item u = decode_item(p, lvs, __ldg(item_list + k), cand_per_unit);
+      const TeamView tv0 = team_view(u, 0, cand_per_tile), tv1 = team_view(u, 1, cand_per_tile);
+      const int n1 = max(tv0.n1, tv1.n1), n2 = max(tv0.n2, tv1.n2);
+      if (n1 + n2 == 0) continue;
+      // the teams' query tiles: two boxes each, as soon as the tile's previous tenant has been read for the last time
+      if (prole == 0) {
+#pragma unroll
+        for (int T = 0; T < kTeams; ++T) {
+          if (!ok || (T ? tv1.n1 + tv1.n2 : tv0.n1 + tv0.n2) == 0) continue;
+          if (q_n[T] > 0) {
+            ok = mbar_wait_rp(sm, p, &sm.q_free[T], (q_n[T] - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) continue;
+          }
+          if (lane == 0) {
+            mbar_expect_tx(&sm.q_full[T], kTileBytes);
+            const int cand0 = u.b0 + (2 * u.mt + T) * cand_per_tile;
+            tma_load_q_half(sm.q[T], &q_map, 0, u.h * g, cand0, &sm.q_full[T]);
+            tma_load_q_half(sm.q[T] + kHalfBytes, &q_map, 64, u.h * g, cand0, &sm.q_full[T]);
+          }
+          ++q_n[T];
+        }
+        if (!ok) break;
+      }
+      for (int seg = 0; seg < 2 && ok; ++seg) {
+        const int seg_lo = seg ? u.lo2 : u.lo;
+        const int seg_hi = seg ? max(tv0.hi2, tv1.hi2) : max(tv0.hi1, tv1.hi1);
+        const int32_t *seg_pages = seg ? u.pages2 : u.pages;
+        if ((seg ? n2 : n1) == 0) continue;
+        const int last_pg = (seg_hi - 1) >> 4;
+        auto load_ids = [&](int blk) -> int { return __ldg(seg_pages + min((seg_lo >> 4) + blk * 32 + lane, last_pg)); };
+        int ids_cur = load_ids(0), ids_next = load_ids(1);
+        int tile = 0;
+        for (int t0 = seg_lo; t0 < seg_hi; t0 += kTileN, ++kt, ++tile) {
+          int pid = __shfl_sync(0xffffffffu, ids_cur, (tile & 3) * 8 + (lane & 7));
+          if ((tile & 3) == 3) {
+            ids_cur = ids_next;
+            ids_next = load_ids((tile >> 2) + 2);
+          }
+          const bool in_range = t0 + (lane & 7) * kPage < seg_hi, good = (unsigned)pid < (unsigned)p.num_pages;
+          if (lane < 8 && in_range && !good && prole == 0) latch(p, kDevBadPage);
+          if (!good) pid = 0;
+          const uint32_t okmask = __ballot_sync(0xffffffffu, in_range && good) & 0xffu;
+          if (prole < 2) {
+            const int sk = kt % kKSlots;
+            ok = mbar_wait_rp(sm, p, &sm.empty_k[sk], ((kt / kKSlots) & 1) ^ 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (KSCALE && prole == 0) {
+              if (lane < 8) sm.kscale[kt & 7][lane] = in_range && good ? __ldg(k_scale + (size_t)pid * p.Hkv + u.h) : 1.f;
+              __syncwarp();
+            }
+            if (lane == 0) {
+              if (prole == 0) sm.page_ok[kt & 7] = okmask;
+              mbar_expect_tx(&sm.full_k[sk], kHalfBytes);
+            }
+            __syncwarp();
+            if (lane < 8)
+              tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64, u.h, pid,
+                                 &sm.full_k[sk], policy);
+          } else {
+            const int sv = kt % kVSlots;
+            ok = mbar_wait_rp(sm, p, &sm.empty_v[sv], ((kt / kVSlots) & 1) ^ 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(&sm.full_v[sv], kTileBytes);
+            __syncwarp();
+            if (lane < 8) tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, u.h, pid, &sm.full_v[sv], policy);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      uint32_t tt0 = 0u, tt1 = 0u;   // tiles of each team whose P has been taken (all items)
+      uint32_t qn0 = 0u, qn1 = 0u;   // items in which each team had tiles
+      for (int k = k_begin; k < k_end && !sm.abort; ++k) {
+        const Item u = decode_item(p, lvs, __ldg(item_list + k), cand_per_unit);
+        const TeamView tv0 = team_view(u, 0, cand_per_tile), tv1 = team_view(u, 1, cand_per_tile);
+        const int n1 = max(tv0.n1, tv1.n1), n_all = n1 + max(tv0.n2, tv1.n2);
+        if (n_all == 0) continue;
+        // The products follow the CTA's K/V stream tile by tile: at tile t, for each team that uses it, the second
+        // product of t and then that team's first product of tile t + 1 (so a team's chain is S, P V, S, ... as in the
+        // kernel above and no product ever asks for a tile outside the slots in flight).  Team 1 is issued after
+        // team 0, so a tile's last user is team 1 where it uses the tile.
+        const int n1_0 = tv0.n1, n2_0 = tv0.n2, n1_1 = tv1.n1, n2_1 = tv1.n2;
+        auto uses0 = [&](int t) -> bool { return t < n1 ? t < n1_0 : t - n1 < n2_0; };
+        auto uses1 = [&](int t) -> bool { return t < n1 ? t < n1_1 : t - n1 < n2_1; };
+        const int cnt0 = n1_0 + n2_0, cnt1 = n1_1 + n2_1;
+        int s_left0 = cnt0, s_left1 = cnt1, pv0 = 0, pv1 = 0;   // first products still to issue; second products issued
+        bool ok = true;
+        uint64_t q_desc0 = 0, q_desc1 = 0;
+        if (cnt0 > 0) {
+          ok = mbar_wait_rp(sm, p, &sm.q_full[0], qn0 & 1);
+          ++qn0;
+          q_desc0 = smem_desc(smem_u32(sm.q[0]), 16, 1024);
+        }
+        if (ok && cnt1 > 0) {
+          ok = mbar_wait_rp(sm, p, &sm.q_full[1], qn1 & 1);
+          ++qn1;
+          q_desc1 = smem_desc(smem_u32(sm.q[1]), 16, 1024);
+        }
+        if (!ok) break;
+        tc_fence_after();
+        // first product of team T (compile-time) on stream tile t
+        auto issue_qk = [&](auto Tc, int t, bool last_user, bool last_of_team) -> bool {
+          constexpr int T = decltype(Tc)::value;
+          const uint32_t ktq = kt + t;
+          const int s = ktq % kKSlots;
+          if (!mbar_wait_rp(sm, p, &sm.full_k[s], (ktq / kKSlots) & 1)) return false;
+          tc_fence_after();
+          const uint32_t tmem_s = tmem + (uint32_t)T * 256u;
+          const uint64_t k_desc = smem_desc(smem_u32(sm.k[s]), 16, 1024), q_desc = T ? q_desc1 : q_desc0;
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+            umma_ss(tmem_s, q_desc + off, k_desc + off, kIdescQK, kk > 0);
+          }
+          if (last_user) umma_commit(&sm.empty_k[s]);   // K(t) is free once its last user's product has read it
+          umma_commit(&sm.s_full[T]);
+          if (last_of_team) umma_commit(&sm.q_free[T]);  // last reader of this team's query tile
+          return true;
+        };
+        auto issue_pv = [&](auto Tc, int t, bool first_of_team, bool last_user, uint32_t done_before) -> bool {
+          constexpr int T = decltype(Tc)::value;
+          const uint32_t ktp = kt + t;
+          const int s = ktp % kVSlots;
+          if (!(mbar_wait_rp(sm, p, &sm.p_full[T], done_before & 1) &&
+                mbar_wait_rp(sm, p, &sm.full_v[s], (ktp / kVSlots) & 1)))
+            return false;
+          tc_fence_after();
+          const uint32_t tmem_s = tmem + (uint32_t)T * 256u, tmem_o = tmem_s + kTileN;
+          const uint64_t v_desc = smem_desc(smem_u32(sm.v[s]), kPageBytes / 2, 1024);
+#pragma unroll
+          for (int kk = 0; kk < kTileN / 16; ++kk)
+            umma_ts(tmem_o, tmem_s + (kk >> 2) * 64 + (kk & 3) * 8, v_desc + (uint64_t)((kk * kPageBytes) >> 4), kIdescPV,
+                    !first_of_team || (kk > 0));
+          if (last_user) umma_commit(&sm.empty_v[s]);
+          umma_commit(&sm.pv_done[T]);
+          return true;
+        };
+        using T0 = std::integral_constant<int, 0>;
+        using T1 = std::integral_constant<int, 1>;
+        // (both teams use stream tile 0 unless a team's first range is empty; the general rule covers it)
+        if (uses0(0)) ok = issue_qk(T0{}, 0, !uses1(0), --s_left0 == 0);
+        if (ok && uses1(0)) ok = issue_qk(T1{}, 0, true, --s_left1 == 0);
+        for (int t = 0; t < n_all && ok; ++t) {
+          const bool u0 = uses0(t), u1 = uses1(t), nx = t + 1 < n_all;
+          const bool v0 = nx && uses0(t + 1), v1 = nx && uses1(t + 1);
+          if (u0) {
+            ok = issue_pv(T0{}, t, pv0 == 0, !u1, tt0);
+            ++tt0;
+            ++pv0;
+          }
+          if (ok && v0) ok = issue_qk(T0{}, t + 1, !v1, --s_left0 == 0);
+          if (ok && u1) {
+            ok = issue_pv(T1{}, t, pv1 == 0, true, tt1);
+            ++tt1;
+            ++pv1;
+          }
+          if (ok && v1) ok = issue_qk(T1{}, t + 1, true, --s_left1 == 0);
+        }
+        if (!ok) break;
+        kt += n_all;
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax / epilogue: team T = row tile 2 mp + T
+    const int team = (warp - 2) >> 2;
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tmem_s = tmem + (uint32_t)team * 256u, tmem_o = tmem_s + kTileN;
+    uint32_t team_tiles = 0;
+    for (int k = k_begin; k < k_end && !sm.abort; ++k) {
+      const Item u = decode_item(p, lvs, __ldg(item_list + k), cand_per_unit);
+      const TeamView me = team_view(u, team, cand_per_tile), other = team_view(u, team ^ 1, cand_per_tile);
+      const int n1 = max(me.n1, other.n1), n_all = n1 + max(me.n2, other.n2);
+      if (me.rows) {
+        const int cand = (2 * u.mt + team) * cand_per_tile + r / g;
+        const bool row_ok = cand < u.n_cand;
+        const size_t qrow = (size_t)(u.b0 + cand) * p.Hq + (size_t)u.h * g + (r % g);
+        const size_t slot = qrow * p.n_parts + u.part;
+        if (!direct && row_ok && u.part2 >= 0) lse_part[qrow * p.n_parts + u.part2] = -INFINITY;
+        const int my_tiles = me.n1 + me.n2;
+        if (my_tiles == 0) {   // no tokens for these rows in this split
+          if (direct && row_ok) {
+            uint4 *dst = reinterpret_cast<uint4 *>(o_final + qrow * D);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+            lse_final[qrow] = -INFINITY;
+          } else if (row_ok) {
+            lse_part[slot] = -INFINITY;
+          }
+        } else {
+          float m = -INFINITY, l = 0.f;
+          const int hi_row1 = u.limits && row_ok ? min(me.hi1, __ldg(u.limits + cand)) : me.hi1;
+          const int hi_row2 = u.limits2 && row_ok ? min(me.hi2, __ldg(u.limits2 + cand)) : me.hi2;
+          bool alive = true;
+          for (int c = 0; c < my_tiles && alive; ++c, ++team_tiles) {
+            const int t = c < me.n1 ? c : n1 + (c - me.n1);                  // tile of the CTA's K/V stream
+            const int t0 = c < me.n1 ? u.lo + c * kTileN : u.lo2 + (c - me.n1) * kTileN;
+            const int hi_row = c < me.n1 ? hi_row1 : hi_row2;
+            alive = mbar_wait_rp(sm, p, &sm.s_full[team], team_tiles & 1);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) break;
+            tc_fence_after();
+            const uint32_t page_ok = sm.page_ok[(kt + t) & 7];
+            const bool full_tile = page_ok == 0xffu && t0 + kTileN <= hi_row;
+            float ck[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ck[i] = KSCALE ? sl2 * sm.kscale[(kt + t) & 7][i] : sl2;
+            uint32_t sv[kTileN];
+            auto load_row = [&]() {
+#pragma unroll
+              for (int cc = 0; cc < kTileN / 32; ++cc)
+                tmem_ld32(tmem_s + lane_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[cc * 32]));
+              tmem_wait_ld();
+              if (!full_tile) {
+                const uint32_t masked = __float_as_uint(sl2 >= 0.f ? -INFINITY : INFINITY);
+#pragma unroll
+                for (int col = 0; col < kTileN; ++col) {
+                  const bool okc = ((page_ok >> (col >> 4)) & 1u) && (t0 + col < hi_row);
+                  if (!okc) sv[col] = masked;
+                }
+              }
+            };
+            load_row();
+            float mx = -INFINITY;
+#pragma unroll
+            for (int pg = 0; pg < 8; ++pg) {
+              float e4[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) e4[i] = __uint_as_float(sv[16 * pg + i]);
+              if (sl2 >= 0.f) {
+#pragma unroll
+                for (int i = 4; i < 16; ++i) e4[i & 3] = fmaxf(e4[i & 3], __uint_as_float(sv[16 * pg + i]));
+                e4[0] = fmaxf(fmaxf(e4[0], e4[1]), fmaxf(e4[2], e4[3]));
+              } else {
+#pragma unroll
+                for (int i = 4; i < 16; ++i) e4[i & 3] = fminf(e4[i & 3], __uint_as_float(sv[16 * pg + i]));
+                e4[0] = fminf(fminf(e4[0], e4[1]), fminf(e4[2], e4[3]));
+              }
+              if (e4[0] != INFINITY && e4[0] != -INFINITY) mx = fmaxf(mx, e4[0] * ck[pg]);
+            }
+            float m_use = m;
+            bool rescale = false;
+            if (mx > m + 8.f) {
+              m_use = mx;
+              rescale = c > 0 && m > -INFINITY;
+            }
+            const float alpha = rescale ? fast_exp2(m - m_use) : 1.f;
+            if (__any_sync(0xffffffffu, rescale)) {
+              alive = mbar_wait_rp(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
+              alive = __all_sync(0xffffffffu, alive);
+              if (!alive) break;
+              tc_fence_after();
+#pragma unroll 1
+              for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t v[32];
+                tmem_ld32(tmem_o + lane_addr + cc * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                tmem_st32(tmem_o + lane_addr + cc * 32, v);
+              }
+              tmem_wait_st();
+              load_row();
+            }
+            l *= alpha;
+            m = m_use;
+            const float neg_m = m == -INFINITY ? 0.f : -m;
+            float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int cc = 0; cc < kTileN / 32; ++cc) {
+              uint32_t pw[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float cf = ck[(cc * 32 + 2 * j) >> 4];
+                const float p0 = fast_exp2(fmaf(__uint_as_float(sv[cc * 32 + 2 * j]), cf, neg_m));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(sv[cc * 32 + 2 * j + 1]), cf, neg_m));
+                lsum[j & 1] += p0;
+                lsum[2 + (j & 1)] += p1;
+                pw[j] = pack_bf16x2(p0, p1);
+              }
+              tmem_st16(tmem_s + lane_addr + (cc >> 1) * 64 + (cc & 1) * 16, pw);
+            }
+            l += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm.p_full[team]);
+          }
+          if (!alive) break;
+          // ---- epilogue of this team's rows: its own accumulator, nothing to merge
+          alive = mbar_wait_rp(sm, p, &sm.pv_done[team], (team_tiles - 1) & 1);
+          if (!__all_sync(0xffffffffu, alive)) break;
+          tc_fence_after();
+          const float inv = l > 0.f ? 1.f / l : 0.f;
+          const uint32_t store_mask = __ballot_sync(0xffffffffu, row_ok && (direct || l > 0.f));
+#pragma unroll 1
+          for (int cc = 0; cc < D / 32; ++cc) {
+            const int col0 = cc * 32;
+            const unsigned long long my_off = (unsigned long long)(direct ? qrow : slot) * D + col0;
+            uint32_t v[32];
+            tmem_ld32(tmem_o + lane_addr + col0, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * inv);
+#pragma unroll
+            for (int s = 4; s >= 1; s >>= 1) {   // transpose 8 x 8 blocks of 16-byte pieces inside each group of 8 lanes
+              const bool up = (lane & s) != 0;
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) {
+                if (kk & s) continue;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                  const uint32_t send = up ? v[4 * kk + w] : v[4 * (kk | s) + w];
+                  const uint32_t got = __shfl_xor_sync(0xffffffffu, send, s);
+                  if (up) v[4 * kk + w] = got; else v[4 * (kk | s) + w] = got;
+                }
+              }
+            }
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const int src = (lane & 24) + kk;
+              const unsigned long long off = __shfl_sync(0xffffffffu, my_off, src);
+              if (!((store_mask >> src) & 1u)) continue;
+              if (direct)
+                *reinterpret_cast<uint2 *>(o_final + off + 4 * (lane & 7)) =
+                    make_uint2(pack_bf16x2(__uint_as_float(v[4 * kk]), __uint_as_float(v[4 * kk + 1])),
+                               pack_bf16x2(__uint_as_float(v[4 * kk + 2]), __uint_as_float(v[4 * kk + 3])));
+              else
+                *reinterpret_cast<float4 *>(o_part + off + 4 * (lane & 7)) =
+                    make_float4(__uint_as_float(v[4 * kk]), __uint_as_float(v[4 * kk + 1]), __uint_as_float(v[4 * kk + 2]),
+                                __uint_as_float(v[4 * kk + 3]));
+            }
+          }
+          if (row_ok) (direct ? lse_final[qrow] : lse_part[slot]) = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+          tc_fence_before();
+        }
+      }
+      kt += n_all;
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (sm.abort && warp == 0 && lane == 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < kDrainCycles) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+static_assert(sizeof(SmemRp) <= 232448, "shared memory of one CTA");
+
 }  // namespace
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -934,6 +1426,26 @@ bool encode_kv_pair_map(CUtensorMap *map, const void *lower_pool, unsigned long 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// q [B][Hq][128] (bf16) as boxes of 128 / g candidates x g heads x 64 elements, 128-byte swizzle.
+bool encode_q_map(CUtensorMap *map, const void *q, int B, int Hq, int g) {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !sym)
+      return false;
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)B};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hq * D * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)g, (cuuint32_t)(kTileM / g)};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(q), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct PrefixTcPlan {
   CUtensorMap k_map, v_map;
   TcLevels levels;
@@ -941,6 +1453,7 @@ struct PrefixTcPlan {
   bool one_part_per_row;   // every row gets exactly one part from this pass: one single-split level, or two chained
   long long wait_cycles;   // limit of every device-side wait
   const float *k_scale;    // non-null: the pools are an expanded e4m3 cache, one K scale per (page, kv head)
+  bool row_pairs;          // items are pairs of row tiles: the row-pair kernel runs the pass
   int32_t *dev_lists;   // device: cta_begin[grid + 1], then item_list[n_items]
 };
 
@@ -956,6 +1469,10 @@ namespace {
 
 bool env_chain_levels() {
   const char *e = std::getenv("MC_PREFIX_CHAIN");
+  return !(e && *e == '0');
+}
+bool env_row_pairs() {
+  const char *e = std::getenv("MC_PREFIX_PAIRS");
   return !(e && *e == '0');
 }
 
@@ -1002,6 +1519,12 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   long long items = 0;
   plan->levels.n = n_levels;
   std::vector<double> cost;
+  // Where every level stacks at least two 128-row tiles per (group, kv head), an item is a pair of row tiles (the
+  // row-pair kernel); otherwise one row tile (MC_PREFIX_PAIRS=0: always one).
+  bool pairs = env_row_pairs();
+  for (int k = 0; k < n_levels; ++k) pairs = pairs && (max_group[k] * levels[k].g + kTileM - 1) / kTileM >= 2;
+  plan->row_pairs = pairs;
+  const int unit_rows = pairs ? 2 * kTileM : kTileM;
   // Two single-split levels of which one's groups nest in the other's, with as many 128-row tiles: the finer level's
   // items take the coarser level's tokens along (one item, one accumulator, one part per row tile instead of two
   // items and two parts), and the coarser level gets no items of its own.
@@ -1027,8 +1550,8 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
         while (i < go[f].size() && go[f][i] < go[c][(size_t)j]) ++i;
         nested = i < go[f].size() && go[f][i] == go[c][(size_t)j];
       }
-      for (int j = 0; j < levels[f].G; ++j) tiles_f += ((long long)(go[f][(size_t)j + 1] - go[f][(size_t)j]) * p.g + kTileM - 1) / kTileM;
-      for (int j = 0; j < levels[c].G; ++j) tiles_c += ((long long)(go[c][(size_t)j + 1] - go[c][(size_t)j]) * p.g + kTileM - 1) / kTileM;
+      for (int j = 0; j < levels[f].G; ++j) tiles_f += ((long long)(go[f][(size_t)j + 1] - go[f][(size_t)j]) * p.g + unit_rows - 1) / unit_rows;
+      for (int j = 0; j < levels[c].G; ++j) tiles_c += ((long long)(go[c][(size_t)j + 1] - go[c][(size_t)j]) * p.g + unit_rows - 1) / unit_rows;
       if (nested && tiles_f <= tiles_c) {
         coarse_len.resize((size_t)levels[c].G);
         if (cudaMemcpy(coarse_len.data(), levels[c].prefix_len, sizeof(int32_t) * coarse_len.size(),
@@ -1054,7 +1577,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
     lv.part_tokens = pk.prefix_part_tokens;
     lv.n_groups = pk.G;
     lv.chain = k == fine ? coarse : -1;
-    lv.n_mt = (max_group[k] * pk.g + kTileM - 1) / kTileM;
+    lv.n_mt = (max_group[k] * pk.g + unit_rows - 1) / unit_rows;   // row units (tiles, or pairs of tiles) per (group, kv head, split)
     const long long level_items = (long long)pk.G * pk.Hkv * lv.n_splits * lv.n_mt;
     items += level_items;
     if (items > (1ll << 24)) {
@@ -1068,7 +1591,7 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
         cudaMemcpy(go.data(), pk.group_offsets, sizeof(int32_t) * go.size(), cudaMemcpyDeviceToHost) == cudaSuccess &&
         cudaMemcpy(len.data(), pk.prefix_len, sizeof(int32_t) * len.size(), cudaMemcpyDeviceToHost) == cudaSuccess;
     (void)cudaGetLastError();
-    const int cand_per_tile = kTileM / pk.g;
+    const int cand_per_tile = unit_rows / pk.g;   // candidates per row unit
     for (long long it = 0; it < level_items; ++it) {
       const int mt = (int)(it % lv.n_mt);
       long long r = it / lv.n_mt;
@@ -1091,7 +1614,10 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
         tiles += (l2 + kTileN - 1) / kTileN;
       }
       double c = 0.0;
-      if (k != coarse && tiles > 0 && mt * cand_per_tile < n_cand) c = (double)tiles * tile_us + item_us;
+      if (k != coarse && tiles > 0 && mt * cand_per_tile < n_cand) {
+        const int row_tiles = pairs && (long long)(n_cand - mt * cand_per_tile) * pk.g > kTileM ? 2 : 1;
+        c = (double)tiles * row_tiles * tile_us + item_us;
+      }
       cost.push_back(c);
     }
   }
@@ -1157,6 +1683,10 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
                            (int)sizeof(Smem)) != cudaSuccess ||
       cudaFuncSetAttribute(prefix_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sizeof(Smem)) != cudaSuccess ||
+      cudaFuncSetAttribute(prefix_rp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sizeof(SmemRp)) != cudaSuccess ||
+      cudaFuncSetAttribute(prefix_rp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sizeof(SmemRp)) != cudaSuccess ||
       cudaMalloc(&plan->dev_lists, sizeof(int32_t) * lists.size()) != cudaSuccess ||
       cudaMemcpy(plan->dev_lists, lists.data(), sizeof(int32_t) * lists.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -1184,18 +1714,30 @@ mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const vo
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)plan->grid);
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = sizeof(Smem);
+  cfg.dynamicSmemBytes = plan->row_pairs ? sizeof(SmemRp) : sizeof(Smem);
   cfg.stream = stream;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = beside_previous ? 1 : 0;
-  const cudaError_t e = cudaLaunchKernelEx(
-      &cfg, plan->k_scale ? prefix_tc_kernel<true> : prefix_tc_kernel<false>, p, plan->levels, plan->k_map, plan->v_map,
-      reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
-      (const int32_t *)(plan->dev_lists + plan->grid + 1), (const int32_t *)plan->dev_lists,
-      reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles, plan->k_scale);
+  cudaError_t e;
+  if (plan->row_pairs) {
+    // the stacked query tiles come by TMA: a map over this call's q, [B][Hq][d] seen as boxes of 128 / g candidates x
+    // g heads x 64 elements (rows of the box = the stacked row order); candidates beyond B read as zeros
+    CUtensorMap q_map;
+    if (!encode_q_map(&q_map, q, p.B, p.Hq, p.g)) return MC_ERR_CUDA;
+    e = cudaLaunchKernelEx(&cfg, plan->k_scale ? prefix_rp_kernel<true> : prefix_rp_kernel<false>, p, plan->levels,
+                           plan->k_map, plan->v_map, q_map, scale * kLog2e, o_part, lse_part,
+                           (const int32_t *)(plan->dev_lists + plan->grid + 1), (const int32_t *)plan->dev_lists,
+                           reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles, plan->k_scale);
+  } else {
+    e = cudaLaunchKernelEx(
+        &cfg, plan->k_scale ? prefix_tc_kernel<true> : prefix_tc_kernel<false>, p, plan->levels, plan->k_map, plan->v_map,
+        reinterpret_cast<const __nv_bfloat16 *>(q), scale * kLog2e, o_part, lse_part,
+        (const int32_t *)(plan->dev_lists + plan->grid + 1), (const int32_t *)plan->dev_lists,
+        reinterpret_cast<__nv_bfloat16 *>(o_final), lse_final, plan->wait_cycles, plan->k_scale);
+  }
   count_launch();
   return e == cudaSuccess ? check_launch() : MC_ERR_CUDA;
 }

@@ -21,11 +21,16 @@ pytestmark = pytest.mark.gpu
 if not torch.cuda.is_available():
     pytest.skip("no CUDA device", allow_module_level=True)
 
-CFG = wl.scaled_down(wl.CONFIGS["cfg2"], "timeout", C=8, prefix=("fixed", 1040), suffix=("uniform", 0, 600))
+# 8 candidates: one 128-row tile per (group, kv head), the prefix kernel with two tile streams; 40 candidates: three
+# row tiles, the row-pair prefix kernel
+CFGS = {"one-tile": wl.scaled_down(wl.CONFIGS["cfg2"], "timeout", C=8, prefix=("fixed", 1040), suffix=("uniform", 0, 600)),
+        "row-pairs": wl.scaled_down(wl.CONFIGS["cfg2"], "timeout-rp", C=40, prefix=("fixed", 1040), suffix=("uniform", 0, 300))}
 
 
-@pytest.mark.parametrize("passes", ["prefix", "suffix", "step"])
-def test_expired_wait_is_reported_and_the_next_call_is_correct(passes, monkeypatch):
+@pytest.mark.parametrize("passes,shape", [("prefix", "one-tile"), ("suffix", "one-tile"), ("step", "one-tile"),
+                                          ("prefix", "row-pairs"), ("step", "row-pairs")])
+def test_expired_wait_is_reported_and_the_next_call_is_correct(passes, shape, monkeypatch):
+    CFG = CFGS[shape]
     hp = wl.make_host_problem(CFG)
     q_np = wl.draw_q(CFG, 0)
     q = to_device(CFG, q_np)
