@@ -300,12 +300,15 @@ def test_other_scales(scale):
     dp.close()
 
 
+@pytest.mark.parametrize("pairs", ["1", "0"])
 @pytest.mark.parametrize("root", [0, 300])
-def test_several_row_tiles_and_several_prefix_splits(monkeypatch, root):
+def test_several_row_tiles_and_several_prefix_splits(monkeypatch, root, pairs):
     """44 candidates x 8 heads per kv head = 352 stacked rows (three 128-row tiles, the last partly filled) over a
     ragged 613-token prefix cut into three splits, every row checked; `root` > 0 puts a prompt shared by all
-    candidates in front (a two-level cascade whose levels have different splits)."""
+    candidates in front (a two-level cascade whose levels have different splits).  pairs = 1: the row-pair prefix
+    kernel (the second pair of row tiles has one tile only); pairs = 0: one row tile per item."""
     monkeypatch.setenv("MC_PREFIX_PART_TOKENS", "256")
+    monkeypatch.setenv("MC_PREFIX_PAIRS", pairs)
     cfg = wl.Config("tiles", "bf16", 1, 44, 64, 8, 128, ("fixed", 613), ("uniform", 0, 90), permute_pages=True, seed=11)
     hp = wl.make_host_problem(cfg)
     if root:

@@ -26,7 +26,7 @@ CASES = {
 }
 
 
-@pytest.mark.parametrize("suffix_storage", [False, True])
+@pytest.mark.parametrize("suffix_storage", [False, True, "one-row-tile-items"])
 @pytest.mark.parametrize("name", list(CASES))
 def test_scoring_matches_oracle(name, suffix_storage, monkeypatch):
     """suffix_storage True also runs the two levels as separate items (MC_PREFIX_CHAIN=0) instead of chained ones.
@@ -35,6 +35,9 @@ def test_scoring_matches_oracle(name, suffix_storage, monkeypatch):
     cfg, prefix_len, seq_len = CASES[name]
     hp = wl.make_scoring_host_problem(cfg, prefix_len, seq_len)
     q = wl.draw_scoring_q(cfg, seq_len)
+    if suffix_storage == "one-row-tile-items":      # the prefix kernel that gives each 128-row tile an item of its own
+        monkeypatch.setenv("MC_PREFIX_PAIRS", "0")
+        suffix_storage = False
     if suffix_storage:
         monkeypatch.setenv("MC_PREFIX_CHAIN", "0")
     dp = ScoringDeviceProblem(hp, suffix_storage=suffix_storage)
