@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # 4096-token chunks on a small problem of cfg4's shape; the traffic grows in proportion to the tokens streamed,
 # so the ratio is scaled by the units of the timed workload).  A ratio is only reported while the kernel source
 # still has the hash it had when the counters were taken.
-SUFFIX_TRAFFIC_RATIO = {"short_chunks": 1.0126, "long_chunks": 1.0025}
-SUFFIX_KERNEL_SHA1 = "67aa78f27892d8ec82ccc8a2311d5a268e7c5771"
+SUFFIX_TRAFFIC_RATIO = {"short_chunks": 1.0122, "long_chunks": 1.0024}
+SUFFIX_KERNEL_SHA1 = "b1c5d052742adae3d483a7572013b2a9de2a4403"
 
 
 def suffix_traffic(algorithmic_bytes, suffix_part_tokens):

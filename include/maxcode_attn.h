@@ -18,8 +18,9 @@
  * token chunks) and a log-sum-exp merge of the partial results.
  *
  * Memory layout (all DEVICE memory, owned by the caller, borrowed by the layout object):
- *   k_pool, v_pool  [num_pages][Hkv][16][d]   elements of `dtype`; 16-byte aligned.  One (page, kv head)
- *                                              slab is 16*d contiguous elements.
+ *   k_pool, v_pool  [num_pages][Hkv][page_size][d]   elements of `dtype`; 16-byte aligned.  One (page, kv head)
+ *                                              slab is page_size*d contiguous elements; page_size is 16 (the
+ *                                              layout the kernels walk directly), 32 or 64 tokens.
  *   prefix_pages    int32 [G][max_prefix_pages]   physical page ids of group j's prefix, in token order
  *   prefix_len      int32 [G]                     tokens (the last page may be partially filled)
  *   suffix_pages    int32 [B][max_suffix_pages]   physical page ids of candidate b's suffix
@@ -31,6 +32,10 @@
  * Page-table entries beyond a sequence's pages are never dereferenced.  Slots of a page beyond the
  * sequence length may hold any finite values.  A page id outside [0, num_pages) makes the kernels skip
  * that page and latch MC_ERR_INVALID_ARG in the device status word (see mc_get_last_status).
+ * With page_size 32 or 64 the kernels still move 16-token blocks (a page is 2 or 4 of them, contiguous per kv head)
+ * and read page tables that the layout object derives from the caller's once, at create time: after changing entries
+ * of prefix_pages, suffix_pages or an outer level's pages call mc_kv_layout_refresh_tables.  With page_size 16 the
+ * caller's tables are read at every call and there is nothing to refresh.
  *
  * Partial results ("parts").  rows = B*Hq, row = b*Hq + hq.  Each row has n_parts slots:
  *   parts [0, n_prefix_parts)            prefix splits of prefix_part_tokens tokens each
@@ -80,7 +85,7 @@ typedef struct {
   int32_t num_q_heads;           /* Hq, a multiple of Hkv */
   int32_t num_kv_heads;          /* Hkv */
   int32_t head_dim;              /* d: 64 or 128 */
-  int32_t page_size;             /* must be 16 */
+  int32_t page_size;             /* tokens per page: 16, 32 or 64 (MC_FP8_E4M3 and mc_decode_attn_static: 16) */
   int32_t num_pages;             /* pages in each pool */
   int32_t max_prefix_pages;      /* row stride of prefix_pages */
   int32_t max_suffix_pages;      /* row stride of suffix_pages; 0: no private tokens at all (scoring whole
@@ -148,7 +153,8 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout);
 
 /* Debug aid: checks on the device that group_offsets is increasing and ends at B, that lengths fit the
  * table strides, that every referenced page id lies in [0, num_pages) and that no page is referenced
- * twice.  Synchronises `stream`.  `scratch` is device memory of at least num_pages*4 bytes. */
+ * twice.  Synchronises `stream`.  `scratch` is device memory of at least num_pages * (page_size / 16) * 4 bytes.
+ * With page_size 32 or 64 it first re-derives the layout's tables from the caller's (mc_kv_layout_refresh_tables). */
 mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t scratch_bytes, void *stream);
 
 /* MC_FP8_E4M3 layouts whose prefix pass runs on the tensor cores keep the prefix levels widened to 16-bit pools of
@@ -157,6 +163,13 @@ mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t 
  * changing prefix pages, their scales, the prefix tables or prefix_len of such a layout, call this to widen them
  * again (asynchronous on `stream`).  On every other layout it does nothing and returns MC_OK. */
 mc_status_t mc_kv_layout_refresh_prefix(mc_kv_layout_t *layout, void *stream);
+
+/* page_size 32 or 64: rewrites the layout's own page tables (in 16-token blocks: entry e of a caller's table becomes
+ * blocks e * page_size / 16 + 0, 1, ...) from the caller's prefix_pages, suffix_pages and outer-level pages as they
+ * are now; one small launch per table, asynchronous on `stream`, order it before the next attention or append call.
+ * Needed after the caller changes a table entry (assigning a page to a growing suffix, swapping a prefix); lengths
+ * are always read live and need no refresh.  page_size 16: does nothing and returns MC_OK. */
+mc_status_t mc_kv_layout_refresh_tables(mc_kv_layout_t *layout, void *stream);
 
 /* Part geometry chosen at create time (needed to size and index o_part / lse_part). */
 mc_status_t mc_kv_layout_geometry(const mc_kv_layout_t *layout, mc_part_geometry_t *out);

@@ -41,6 +41,7 @@ EXPORTS = {
     "mc_kv_layout_destroy": (c_int32, [c_void_p]),
     "mc_kv_layout_validate": (c_int32, [c_void_p, c_void_p, c_size_t, c_void_p]),
     "mc_kv_layout_refresh_prefix": (c_int32, [c_void_p, c_void_p]),
+    "mc_kv_layout_refresh_tables": (c_int32, [c_void_p, c_void_p]),
     "mc_kv_layout_geometry": (c_int32, [c_void_p, POINTER(PartGeometry)]),
     "mc_workspace_bytes": (c_size_t, [c_void_p]),
     "mc_kv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -137,6 +138,10 @@ def mc_kv_layout_destroy(layout: int) -> None:
 
 def mc_kv_layout_refresh_prefix(layout: int, stream: int = 0) -> None:
     _check(lib().mc_kv_layout_refresh_prefix(layout, stream), "mc_kv_layout_refresh_prefix")
+
+
+def mc_kv_layout_refresh_tables(layout: int, stream: int = 0) -> None:
+    _check(lib().mc_kv_layout_refresh_tables(layout, stream), "mc_kv_layout_refresh_tables")
 
 
 def mc_kv_layout_geometry(layout: int) -> PartGeometry:

@@ -32,6 +32,12 @@ struct Layout {
   PrefixTcPlan *tc_plan;      // non-null: every prefix level runs on the tcgen05 kernel, as one launch
   int n_outer;                // outer prefix levels of a cascade (shared by more candidates than the base level)
   Params outer_p[kMaxOuterLevels];
+  // Cache pages of 32 or 64 tokens: every kernel walks 16-token unit pages through tables the layout derives from
+  // the caller's (entry e of a table becomes the units e * r .. e * r + r - 1, r = page_size / 16).
+  struct UnitTable { const int32_t *src; int32_t *dst; long long n; };
+  UnitTable unit_tab[2 + kMaxOuterLevels];
+  int n_unit_tab;
+  int32_t *unit_buf;          // the derived tables, one allocation; null with 16-token pages
   cudaStream_t side_stream;   // the suffix pass of mc_decode_attn runs here, beside the prefix pass
   cudaEvent_t fork_ev, join_ev;
   bool pdl;                   // suffix pass launched as the prefix pass's programmatic dependent (MC_PDL=0: off)
@@ -86,7 +92,7 @@ __global__ void __launch_bounds__(256) append_kernel(Params p, const uint4 *__re
   for (int i = threadIdx.x; i < 2 * n_vec; i += blockDim.x) {
     const int which = i >= n_vec, j = which ? i - n_vec : i;
     const int h = j / row_vec, c = j % row_vec;
-    const size_t dst = (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + c;
+    const size_t dst = (slab_index(p, page, h) * kPage + (s & 15)) * row_vec + c;
     const size_t src = ((size_t)b * p.Hkv + h) * row_vec + c;
     if (which) vp[dst] = v_new[src]; else kp[dst] = k_new[src];
   }
@@ -149,7 +155,7 @@ __global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels l
   T *kp = reinterpret_cast<T *>(const_cast<void *>(p.k_pool));
   for (int h = h0; h < p.Hkv; h += lanes) {
     const T *src = k_new + ((size_t)b * p.Hkv + h) * p.d;
-    T *dst = kp + (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * p.d;
+    T *dst = kp + (slab_index(p, page, h) * kPage + (s & 15)) * p.d;
     const float re = rope_load(src + i), im = rope_load(src + i + half);
     rope_store(dst + i, re * c - im * sf);
     rope_store(dst + i + half, re * sf + im * c);
@@ -165,7 +171,7 @@ __global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels l
   uint4 *vp = reinterpret_cast<uint4 *>(const_cast<void *>(p.v_pool));
   for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
     const int h = j / row_vec, cc = j % row_vec;
-    vp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = v_new[((size_t)b * p.Hkv + h) * row_vec + cc];
+    vp[(slab_index(p, page, h) * kPage + (s & 15)) * row_vec + cc] = v_new[((size_t)b * p.Hkv + h) * row_vec + cc];
   }
   __syncthreads();  // every thread has read s and issued its stores before the length moves
   if (threadIdx.x == 0) suffix_len[b] = s + 1;
@@ -207,14 +213,14 @@ __global__ void __launch_bounds__(256) append_tokens_kernel(Params p, RopeLevels
   const uint4 *vsrc = reinterpret_cast<const uint4 *>(v_new) + tok * n_vec;
   for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
     const int h = j / row_vec, cc = j % row_vec;
-    vp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = vsrc[j];
+    vp[(slab_index(p, page, h) * kPage + (s & 15)) * row_vec + cc] = vsrc[j];
   }
   if (log2_base == 0.0) {   // keys as they are
     uint4 *kp = reinterpret_cast<uint4 *>(const_cast<void *>(p.k_pool));
     const uint4 *ksrc = reinterpret_cast<const uint4 *>(k_new) + tok * n_vec;
     for (int j = threadIdx.x; j < n_vec; j += blockDim.x) {
       const int h = j / row_vec, cc = j % row_vec;
-      kp[(((size_t)page * p.Hkv + h) * kPage + (s & 15)) * row_vec + cc] = ksrc[j];
+      kp[(slab_index(p, page, h) * kPage + (s & 15)) * row_vec + cc] = ksrc[j];
     }
     return;
   }
@@ -240,7 +246,7 @@ __global__ void __launch_bounds__(256) append_tokens_kernel(Params p, RopeLevels
   T *kp = reinterpret_cast<T *>(const_cast<void *>(p.k_pool));
   for (int h = h0; h < p.Hkv; h += lanes) {
     const T *src = k_new + (tok * p.Hkv + h) * p.d;
-    T *dst = kp + (((size_t)page * p.Hkv + h) * kPage + (s & 15)) * p.d;
+    T *dst = kp + (slab_index(p, page, h) * kPage + (s & 15)) * p.d;
     const float re = rope_load(src + i), im = rope_load(src + i + half);
     rope_store(dst + i, re * c - im * sf);
     rope_store(dst + i + half, re * sf + im * c);
@@ -268,6 +274,22 @@ __global__ void advance_len_kernel(Params p, int n_max, const int32_t *__restric
   }
   suffix_len[b] = s0 + n;
 }
+
+// ------------------------------------------------------------------------------------------------
+// page tables of a cache with 32- or 64-token pages, rewritten in 16-token unit pages: entry e of the
+// caller's table gives the 2^lr units e * 2^lr + 0 .. 2^lr - 1; a negative entry stays -1, any other entry
+// outside the pool becomes an id that no pool has
+// ------------------------------------------------------------------------------------------------
+__global__ void unit_table_kernel(const int32_t *__restrict__ src, int32_t *__restrict__ dst, long long n_src, int lr,
+                                  int src_pages) {
+  const long long n = n_src << lr, nth = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nth) {
+    const int e = __ldg(src + (i >> lr));
+    dst[i] = e < 0 ? -1 : e >= src_pages ? 0x7fffffff : (e << lr) + (int)(i & ((1 << lr) - 1));
+  }
+}
+
+mc_status_t launch_unit_tables(const Layout *L, cudaStream_t st);
 
 // ------------------------------------------------------------------------------------------------
 // validation
@@ -359,6 +381,17 @@ mc_status_t run_pass(Layout *L, int mode, const void *q, float scale, float *o_p
     }
   }
   return run_level(L, L->p, mode, q, scale, o_part, lse_part, st);
+}
+
+mc_status_t launch_unit_tables(const Layout *L, cudaStream_t st) {
+  for (int i = 0; i < L->n_unit_tab; ++i) {
+    const Layout::UnitTable &t = L->unit_tab[i];
+    const long long n = t.n << L->p.lr;
+    const int blocks = (int)(n / 256 + 1 > 1184 ? 1184 : n / 256 + 1);
+    unit_table_kernel<<<blocks, 256, 0, st>>>(t.src, t.dst, t.n, L->p.lr, L->desc.num_pages);
+    count_launch();
+  }
+  return check_launch();
 }
 
 // Splits and persistent-CTA count of one prefix level (see the comment in mc_kv_layout_create_cascade).
@@ -463,7 +496,14 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     if (outer[k].num_groups < 1 || outer[k].num_groups > d->batch || outer[k].max_pages < 1 ||
         !outer[k].group_offsets || !outer[k].pages || !outer[k].len)
       return MC_ERR_INVALID_ARG;
-  if (d->page_size != mc::kPage) return MC_ERR_UNSUPPORTED;
+  if (d->page_size != 16 && d->page_size != 32 && d->page_size != 64) return MC_ERR_UNSUPPORTED;
+  const int lr = d->page_size == 16 ? 0 : d->page_size == 32 ? 1 : 2, upp = 1 << lr;   // unit pages per cache page
+  if ((long long)d->num_pages * upp >= 0x7fffffffLL || (long long)d->max_prefix_pages * upp * mc::kPage > 0x7fffffffLL ||
+      (long long)d->max_suffix_pages * upp * mc::kPage > 0x7fffffffLL)
+    return MC_ERR_UNSUPPORTED;
+  for (int k = 0; k < n_outer; ++k)
+    if ((long long)outer[k].max_pages * upp * mc::kPage > 0x7fffffffLL) return MC_ERR_UNSUPPORTED;
+  if (d->dtype == MC_FP8_E4M3 && lr != 0) return MC_ERR_UNSUPPORTED;   // page scales are per 16-token page
   if (d->dtype != MC_F32 && d->dtype != MC_BF16 && d->dtype != MC_FP8_E4M3) return MC_ERR_UNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return MC_ERR_UNSUPPORTED;
   if ((long long)d->batch * d->num_q_heads > (1ll << 30)) return MC_ERR_UNSUPPORTED;
@@ -480,13 +520,16 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   L->io_dtype = fp8 ? MC_BF16 : d->dtype;
   L->fp8 = nullptr;
   L->x_n = 0;
+  L->n_unit_tab = 0;
+  L->unit_buf = nullptr;
   mc::Params &p = L->p;
   p.k_pool = d->k_pool; p.v_pool = d->v_pool;
   p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
   p.suffix_pages = d->suffix_pages; p.suffix_len = d->suffix_len;
   p.G = d->num_groups; p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.d = d->head_dim;
   p.g = d->num_q_heads / d->num_kv_heads;
-  p.num_pages = d->num_pages; p.max_pp = d->max_prefix_pages; p.max_sp = d->max_suffix_pages;
+  p.lr = lr;
+  p.num_pages = d->num_pages * upp; p.max_pp = d->max_prefix_pages * upp; p.max_sp = d->max_suffix_pages * upp;
   p.row_limit = nullptr;
   p.k_scale = fp8 ? d->k_scale : nullptr;
   p.v_scale = fp8 ? d->v_scale : nullptr;
@@ -497,8 +540,38 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     po.group_offsets = outer[k].group_offsets;
     po.prefix_pages = outer[k].pages;
     po.prefix_len = outer[k].len;
-    po.max_pp = outer[k].max_pages;
+    po.max_pp = outer[k].max_pages * upp;
     po.row_limit = outer[k].row_limit;
+  }
+  if (lr > 0) {   // tables in unit pages, filled before anything below reads them
+    long long total = 0;
+    auto add = [&](const int32_t *src, long long n) {
+      L->unit_tab[L->n_unit_tab++] = {src, reinterpret_cast<int32_t *>((uintptr_t)total), n};   // dst: offset for now
+      total += ((n << lr) + 63) & ~63ll;
+    };
+    add(d->prefix_pages, (long long)d->num_groups * d->max_prefix_pages);
+    if (d->max_suffix_pages > 0) add(d->suffix_pages, (long long)d->batch * d->max_suffix_pages);
+    for (int k = 0; k < n_outer; ++k) add(outer[k].pages, (long long)outer[k].num_groups * outer[k].max_pages);
+    if (cudaMalloc(&L->unit_buf, sizeof(int32_t) * (size_t)total) != cudaSuccess) {
+      (void)cudaGetLastError();
+      delete L;
+      return MC_ERR_OUT_OF_MEMORY;
+    }
+    for (int i = 0; i < L->n_unit_tab; ++i)
+      L->unit_tab[i].dst = L->unit_buf + reinterpret_cast<uintptr_t>(L->unit_tab[i].dst);
+    int i = 0;
+    p.prefix_pages = L->unit_tab[i++].dst;
+    if (d->max_suffix_pages > 0) p.suffix_pages = L->unit_tab[i++].dst;
+    for (int k = 0; k < n_outer; ++k) {
+      L->outer_p[k].prefix_pages = L->unit_tab[i++].dst;
+      L->outer_p[k].suffix_pages = p.suffix_pages;
+    }
+    if (mc::launch_unit_tables(L, nullptr) != MC_OK || cudaStreamSynchronize(nullptr) != cudaSuccess) {
+      (void)cudaGetLastError();
+      cudaFree(L->unit_buf);
+      delete L;
+      return MC_ERR_CUDA;
+    }
   }
 
   // Part geometry.  Suffix chunks come from the table stride (the lengths live on the device and may grow).
@@ -506,7 +579,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   // are now.  The prefix pass runs beside the suffix pass and should end well inside the suffix pass's HBM time;
   // every work item (one token range of one 128-row tile) pays a fixed prologue/epilogue, so items should be
   // long: as few splits as still let one item fit that time.  Constants are measured for this kernel pair.
-  const int max_s = d->max_suffix_pages * mc::kPage;
+  const int max_s = p.max_sp * mc::kPage;
   double suffix_us = 0.0, suffix_tokens_now = -1.0;
   int32_t *sl = nullptr;
   {
@@ -574,6 +647,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
   L->sfx_plan = L->has_suffix && L->use_mma && mc::env_int("MC_SUFFIX_TMA", 1) ? mc::suffix_tma_plan(p, d->dtype) : nullptr;
   if (fp8 && !(L->fp8 = mc::fp8_plan(p))) {
     delete[] sl;
+    cudaFree(L->unit_buf);
     delete L;
     return MC_ERR_UNSUPPORTED;
   }
@@ -622,6 +696,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
 
   if (cudaMalloc(&L->dev_status, 256) != cudaSuccess) {
     cudaFree(L->suffix_order);
+    cudaFree(L->unit_buf);
     mc::suffix_tma_plan_free(L->sfx_plan);
     mc::fp8_plan_free(L->fp8);
     delete L;
@@ -631,6 +706,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
       cudaMallocHost(&L->host_status, sizeof(int32_t)) != cudaSuccess) {
     cudaFree(L->dev_status);
     cudaFree(L->suffix_order);
+    cudaFree(L->unit_buf);
     mc::suffix_tma_plan_free(L->sfx_plan);
     mc::fp8_plan_free(L->fp8);
     delete L;
@@ -704,9 +780,17 @@ mc_status_t mc_kv_layout_destroy(mc_kv_layout_t *layout) {
   mc::fp8_plan_free(L->fp8);
   cudaFree(L->dev_status);
   cudaFree(L->suffix_order);
+  cudaFree(L->unit_buf);
   cudaFreeHost(L->host_status);
   delete L;
   return MC_OK;
+}
+
+mc_status_t mc_kv_layout_refresh_tables(mc_kv_layout_t *layout, void *stream) {
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L) return MC_ERR_INVALID_ARG;
+  if (L->n_unit_tab == 0) return MC_OK;   // 16-token pages: the kernels read the caller's tables themselves
+  return mc::launch_unit_tables(L, reinterpret_cast<cudaStream_t>(stream));
 }
 
 mc_status_t mc_kv_layout_refresh_prefix(mc_kv_layout_t *layout, void *stream) {
@@ -751,6 +835,7 @@ mc_status_t mc_kv_layout_validate(mc_kv_layout_t *layout, void *scratch, size_t 
   if (!L || !scratch) return MC_ERR_INVALID_ARG;
   if (scratch_bytes < (size_t)L->p.num_pages * sizeof(int32_t)) return MC_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (L->n_unit_tab && mc::launch_unit_tables(L, st) != MC_OK) return MC_ERR_CUDA;   // check the tables as they are now
   if (cudaMemsetAsync(scratch, 0, (size_t)L->p.num_pages * sizeof(int32_t), st) != cudaSuccess) return MC_ERR_CUDA;
   mc::validate_kernel<<<148, 256, 0, st>>>(L->p, reinterpret_cast<int32_t *>(scratch), 1);
   mc::count_launch();

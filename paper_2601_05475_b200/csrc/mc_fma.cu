@@ -94,7 +94,7 @@ attn_fma_kernel(Params p, const T *__restrict__ q, float scale_log2, float *__re
         ok = false;
       }
       if (ok) {
-        const size_t off = (((size_t)page * p.Hkv + h) * kPage + (t & 15)) * D + lane * VEC;
+        const size_t off = (slab_index(p, page, h) * kPage + (t & 15)) * D + lane * VEC;
         float kv[VEC];
         RowLoad<T, VEC>::ld(kp + off, kv);
         RowLoad<T, VEC>::ld(vp + off, vv[u]);

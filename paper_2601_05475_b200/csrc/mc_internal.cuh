@@ -23,7 +23,8 @@ struct Params {
   const void *k_pool, *v_pool;
   const int32_t *group_offsets, *prefix_pages, *prefix_len, *suffix_pages, *suffix_len;
   int32_t G, B, Hq, Hkv, d, g;
-  int32_t num_pages, max_pp, max_sp;
+  int32_t num_pages, max_pp, max_sp;                 // in 16-token UNIT pages (a cache page of 32 / 64 tokens is 2 / 4 of them)
+  int32_t lr;                                        // log2 of the unit pages per cache page (0, 1, 2)
   int32_t n_parts;                                   // part slots per row (all prefix levels + suffix chunks)
   int32_t n_prefix_parts, prefix_part_base;          // this prefix level's splits and its first part slot
   int32_t suffix_part_base;                          // first part slot of the suffix chunks
@@ -53,6 +54,13 @@ __device__ __forceinline__ int group_of(const Params &p, int b) {
 }
 
 __device__ __forceinline__ void latch(const Params &p, int code) { atomicCAS(p.status, 0, code); }
+
+// The kernels walk tables of 16-token unit pages.  Unit id u = cache page id * units per page + unit inside the page;
+// the pool is [cache page][kv head][page_size tokens][d], so the 16-token slab of (u, kv head h) is slab number
+// ((u >> lr) * Hkv + h) * 2^lr + (u & (2^lr - 1)) in units of 16 * d elements.  With 16-token cache pages: u * Hkv + h.
+__device__ __forceinline__ size_t slab_index(const Params &p, int unit, int h) {
+  return ((((size_t)(unit >> p.lr)) * p.Hkv + h) << p.lr) + (size_t)(unit & ((1 << p.lr) - 1));
+}
 
 template <int MODE>
 __device__ __forceinline__ Span resolve_span(const Params &p, int b, int part) {
@@ -119,9 +127,10 @@ mc_status_t launch_prefix_tc(const Params &p, const PrefixTcPlan *plan, const vo
                              bool beside_previous = false);
 
 
-// Tensor map over a paged pool [page][kv head][16 tokens][128] (bf16) for TMA copies with the 128-byte swizzle:
-// `whole_page`: one 4 KB box per (page, kv head) slab that lands as [d half][16 tokens][64];
-// otherwise one 2 KB box per (page, kv head, d half).
+// Tensor map over a paged pool seen as num_pages * Hkv slabs of [16 tokens][128] (bf16; num_pages counts 16-token
+// unit pages; slab_index orders them) for TMA copies with the 128-byte swizzle:
+// `whole_page`: one 4 KB box per slab that lands as [d half][16 tokens][64];
+// otherwise one 2 KB box per (slab, d half).
 bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv, bool whole_page);
 bool encode_kv_pair_map(CUtensorMap *map, const void *lower_pool, unsigned long long distance, int num_pages, int Hkv);
 

@@ -214,7 +214,7 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
       pid = 0;
       hi_eff = 0;
     }
-    return ((size_t)pid * p.Hkv + h) * kSlab;
+    return slab_index(p, pid, h) * kSlab;
   };
 
   const uint64_t pol = l2_stream_policy();
@@ -231,7 +231,7 @@ attn_mma_body(const Params &p, const __nv_bfloat16 *__restrict__ q, float sl2, f
   const int kPrefetch = prefetch_pages;
   auto prefetch_page = [&](int pgi, int pid) {
     if (pgi < pg_end && (unsigned)pid < (unsigned)p.num_pages) {
-      const size_t s = ((size_t)pid * p.Hkv + h) * kSlab;
+      const size_t s = slab_index(p, pid, h) * kSlab;
       l2_prefetch_slab<D>(kpool + s);
       l2_prefetch_slab<D>(vpool + s);
     }

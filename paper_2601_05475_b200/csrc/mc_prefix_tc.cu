@@ -108,23 +108,23 @@ __device__ __forceinline__ uint64_t l2_keep_policy() {
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
   return pol;
 }
-// One (page, kv head) slab of V: both 64-element halves of its 16 token rows, 4 KB, one box.
-__device__ __forceinline__ void tma_load_page(void *dst, const CUtensorMap *map, int head, int page, uint64_t *bar,
-                                              uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
-      "[%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;\n"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(0), "r"(0), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
-      : "memory");
-}
-// One d half (64 elements) of the 16 token rows of a (page, kv head) slab of K: 2 KB.  The swizzle span caps
-// a box at 64 elements per row, and the K-major operand wants each half's 128 token rows contiguous.
-__device__ __forceinline__ void tma_load_half_page(void *dst, const CUtensorMap *map, int x, int head, int page,
-                                                   uint64_t *bar, uint64_t policy) {
+// One 16-token slab of V (a unit page of one kv head): both 64-element halves of its 16 token rows, 4 KB, one box.
+// `slab` counts 16-token slabs of the pool (slab_index).
+__device__ __forceinline__ void tma_load_page(void *dst, const CUtensorMap *map, int slab, uint64_t *bar, uint64_t policy) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%2, %3, %4, %5}], [%6], %7;\n"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(0), "r"(head), "r"(page), "r"(smem_u32(bar)), "l"(policy)
+      ::"r"(smem_u32(dst)), "l"(map), "r"(0), "r"(0), "r"(0), "r"(slab), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+// One d half (64 elements) of the 16 token rows of a slab of K: 2 KB.  The swizzle span caps a box at 64 elements per
+// row, and the K-major operand wants each half's 128 token rows contiguous.
+__device__ __forceinline__ void tma_load_half_page(void *dst, const CUtensorMap *map, int x, int slab, uint64_t *bar,
+                                                   uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4}], [%5], %6;\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(0), "r"(slab), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
 
@@ -486,8 +486,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           }
           __syncwarp();
           if (lane < 8)
-            tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64, it.h, pid,
-                               &sm.full_k[sk], policy);
+            tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64,
+                               (int)slab_index(p, pid, it.h), &sm.full_k[sk], policy);
         } else {
           // ---- V(t): 8 boxes of 4 KB
           const int sv = kt % kVSlots;
@@ -496,7 +496,8 @@ prefix_tc_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
           if (!ok) break;
           if (lane == 0) mbar_expect_tx(&sm.full_v[sv], kTileBytes);
           __syncwarp();
-          if (lane < 8) tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, it.h, pid, &sm.full_v[sv], policy);
+          if (lane < 8)
+            tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, (int)slab_index(p, pid, it.h), &sm.full_v[sv], policy);
         }
         if (round <= kQRounds) {
           ok = q_step(nxt, it_n + 1, round);
@@ -1069,8 +1070,8 @@ prefix_rp_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
             }
             __syncwarp();
             if (lane < 8)
-              tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64, u.h, pid,
-                                 &sm.full_k[sk], policy);
+              tma_load_half_page(sm.k[sk] + prole * kHalfBytes + lane * (kPageBytes / 2), &k_map, prole * 64,
+                                 (int)slab_index(p, pid, u.h), &sm.full_k[sk], policy);
           } else {
             const int sv = kt % kVSlots;
             ok = mbar_wait_rp(sm, p, &sm.empty_v[sv], ((kt / kVSlots) & 1) ^ 1);
@@ -1078,7 +1079,8 @@ prefix_rp_kernel(Params p, const __grid_constant__ TcLevels lvs, const __grid_co
             if (!ok) break;
             if (lane == 0) mbar_expect_tx(&sm.full_v[sv], kTileBytes);
             __syncwarp();
-            if (lane < 8) tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, u.h, pid, &sm.full_v[sv], policy);
+            if (lane < 8)
+              tma_load_page(sm.v[sv] + lane * kPageBytes, &v_map, (int)slab_index(p, pid, u.h), &sm.full_v[sv], policy);
           }
         }
       }
@@ -1388,21 +1390,23 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int Hkv,
       return false;
     fn = reinterpret_cast<EncodeTiledFn>(sym);
   }
-  // pool[page][head][token][d] seen as [page][head][token][d half][64]; dimensions innermost first, with the
-  // half before the token so that a box lands as [d half][16 tokens][64 elements]
-  const cuuint64_t dims[5] = {64, (cuuint64_t)kPage, 2, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
-  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, 128, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
-  const cuuint32_t box[5] = {64, (cuuint32_t)kPage, 2, 1, 1};
-  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  if (!whole_page) {   // K: pool[page][head][token][d], one box = 64 elements x 16 tokens
-    const cuuint64_t dims4[4] = {(cuuint64_t)D, (cuuint64_t)kPage, (cuuint64_t)Hkv, (cuuint64_t)num_pages};
-    const cuuint64_t strides4[3] = {(cuuint64_t)D * 2, (cuuint64_t)kPage * D * 2, (cuuint64_t)Hkv * kPage * D * 2};
-    const cuuint32_t box4[4] = {64, (cuuint32_t)kPage, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims4, strides4, box4, estr,
+  // The pool is a sequence of 16-token slabs of 16 x 128 elements (num_pages counts 16-token unit pages, so there
+  // are num_pages * Hkv of them, whatever the cache's page size).  V: a slab seen as [token][d half][64]; dimensions
+  // innermost first, with the half before the token so that a box lands as [d half][16 tokens][64 elements].
+  const cuuint64_t n_slabs = (cuuint64_t)num_pages * (cuuint64_t)Hkv;
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  if (!whole_page) {   // K: one box = 64 elements x 16 tokens of one slab
+    const cuuint64_t dims3[3] = {(cuuint64_t)D, (cuuint64_t)kPage, n_slabs};
+    const cuuint64_t strides3[2] = {(cuuint64_t)D * 2, (cuuint64_t)kPage * D * 2};
+    const cuuint32_t box3[3] = {64, (cuuint32_t)kPage, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims3, strides3, box3, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
   }
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(pool), dims, strides, box, estr,
+  const cuuint64_t dims[4] = {64, (cuuint64_t)kPage, 2, n_slabs};
+  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, 128, (cuuint64_t)kPage * D * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)kPage, 2, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1511,7 +1515,8 @@ PrefixTcPlan *prefix_tc_plan(const Params *levels, const int *max_group, int n_l
   plan->k_scale = k_scale;
   plan->wait_cycles = wait_limit_cycles();
   const Params &p = levels[0];
-  if (!encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
+  if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||
+      !encode_pool_map(&plan->k_map, p.k_pool, p.num_pages, p.Hkv, false) ||
       !encode_pool_map(&plan->v_map, p.v_pool, p.num_pages, p.Hkv, true)) {
     delete plan;
     return nullptr;

@@ -70,6 +70,7 @@ mc_status_t mc_decode_attn_static(const mc_kv_layout_desc_t *d, const void *q, f
   p.suffix_order = nullptr;
   p.row_limit = nullptr;
   p.k_scale = p.v_scale = nullptr;
+  p.lr = 0;
   p.k_pool = d->k_pool; p.v_pool = d->v_pool;
   p.group_offsets = d->group_offsets; p.prefix_pages = d->prefix_pages; p.prefix_len = d->prefix_len;
   p.suffix_pages = d->suffix_pages; p.suffix_len = d->suffix_len;

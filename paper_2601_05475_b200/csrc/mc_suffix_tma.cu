@@ -207,7 +207,7 @@ suffix_tma_body(const Params &p, const CUtensorMap &kv_map, uint32_t k_off, uint
     if ((unsigned)id >= (unsigned)p.num_pages) id = 0;
     const int s = o % kStages;
     mbar_expect_tx(&full[s], kStageBytes);
-    tma_load_stage(smem_u32(ring[s]), &kv_map, id * p.Hkv + h, &full[s], pol);
+    tma_load_stage(smem_u32(ring[s]), &kv_map, (int)slab_index(p, id, h), &full[s], pol);
   };
 #pragma unroll 1
   for (int o = 0; o < kStages && o < n_ord; o += 2) issue_pair(o);
@@ -393,7 +393,7 @@ SuffixTmaPlan *suffix_tma_plan(const Params &p, int dtype) {
   plan->k_off = ka < va ? 0u : kSlabBytes;
   plan->v_off = ka < va ? kSlabBytes : 0u;
   plan->wait_cycles = wait_limit_cycles();
-  if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||
+  if ((long long)p.num_pages * p.Hkv > 0x7fffffffLL ||   // (num_pages counts 16-token unit pages: the map's slabs)
       !encode_kv_pair_map(&plan->kv_map, ka < va ? p.k_pool : p.v_pool, (unsigned long long)(ka < va ? va - ka : ka - va),
                           p.num_pages, p.Hkv) ||
       cudaFuncSetAttribute(suffix_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(Smem)) !=

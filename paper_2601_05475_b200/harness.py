@@ -42,7 +42,7 @@ class DeviceProblem:
         self.group_offsets = i32(tables.group_offsets)
         d = mc.LayoutDesc()
         d.num_groups, d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = cfg.G, cfg.B, cfg.Hq, cfg.Hkv, cfg.d
-        d.page_size, d.num_pages = wl.PAGE, tables.num_pages
+        d.page_size, d.num_pages = cfg.page, tables.num_pages
         d.max_prefix_pages, d.max_suffix_pages = tables.max_prefix_pages, tables.max_suffix_pages
         d.dtype = {"f32": mc.MC_F32, "bf16": mc.MC_BF16, "fp8": mc.MC_FP8_E4M3}[cfg.dtype]
         d.k_pool, d.v_pool = k_pool.data_ptr(), v_pool.data_ptr()
@@ -110,7 +110,7 @@ def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, d
     outer_np = []
     for (go, lens) in outer:
         lens = np.asarray(lens, dtype=np.int32)
-        npp = (lens.astype(np.int64) + wl.PAGE - 1) // wl.PAGE
+        npp = (lens.astype(np.int64) + cfg.page - 1) // cfg.page
         pages = np.full((len(lens), max(1, int(npp.max(initial=0)))), -1, dtype=np.int32)
         for j in range(len(lens)):
             pages[j, :int(npp[j])] = np.arange(tables.num_pages, tables.num_pages + int(npp[j]), dtype=np.int32)
@@ -119,19 +119,19 @@ def make_device_problem(cfg: wl.Config, headroom_tokens: Optional[int] = None, d
     tdtype = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
     gen = torch.Generator(device=device)
     gen.manual_seed(cfg.seed * 1000003 + 17)
-    shape = (tables.num_pages, cfg.Hkv, wl.PAGE, cfg.d)
+    shape = (tables.num_pages, cfg.Hkv, cfg.page, cfg.d)
     fp8 = cfg.dtype == "fp8"
     k_pool = torch.empty(shape, dtype=torch.uint8 if fp8 else tdtype, device=device)
     v_pool = torch.empty(shape, dtype=torch.uint8 if fp8 else tdtype, device=device)
     k_scale = torch.empty((tables.num_pages, cfg.Hkv), dtype=torch.float32, device=device) if fp8 else None
     v_scale = torch.empty((tables.num_pages, cfg.Hkv), dtype=torch.float32, device=device) if fp8 else None
-    step = max(1, (1 << 28) // (cfg.Hkv * wl.PAGE * cfg.d))          # pages per chunk, bounds temporaries
+    step = max(1, (1 << 28) // (cfg.Hkv * cfg.page * cfg.d))          # pages per chunk, bounds temporaries
     for lo in range(0, tables.num_pages, step):
         hi = min(tables.num_pages, lo + step)
         k = torch.empty((hi - lo,) + shape[1:], dtype=tdtype, device=device).normal_(generator=gen)
         v = torch.empty((hi - lo,) + shape[1:], dtype=tdtype, device=device).normal_(generator=gen)
         if cfg.k_outlier_prob > 0.0:
-            mask = torch.rand((hi - lo, cfg.Hkv, wl.PAGE, 1), device=device, generator=gen) < cfg.k_outlier_prob
+            mask = torch.rand((hi - lo, cfg.Hkv, cfg.page, 1), device=device, generator=gen) < cfg.k_outlier_prob
             k = torch.where(mask, k * cfg.k_outlier_scale, k)
         if fp8:
             # an input generator, not the library's quantiser: every page gets the scale its first token would have
@@ -178,17 +178,17 @@ def logical_rows(dp: DeviceProblem, b: int, h: int, suffix_len_now: Optional[int
         jo = int(np.searchsorted(go, b, side="right") - 1)
         segments.append((pages[jo], int(lens[jo])))
     segments += [(dp.tables.prefix_pages[j], P), (dp.tables.suffix_pages[b], s)]
-    out = []
+    out, page = [], dp.cfg.page
     for pool, scale in ((dp.k_pool, dp.k_scale), (dp.v_pool, dp.v_scale)):
         parts, scales = [], []
         for pages_row, n in segments:
-            n_pages = (n + wl.PAGE - 1) // wl.PAGE
+            n_pages = (n + page - 1) // page
             if n_pages:
                 ids = torch.from_numpy(np.ascontiguousarray(pages_row[:n_pages], dtype=np.int64)).to(pool.device)
-                rows = pool[ids, h].reshape(n_pages * wl.PAGE, -1)[:n]
+                rows = pool[ids, h].reshape(n_pages * page, -1)[:n]
                 parts.append(rows.cpu().numpy() if pool.dtype == torch.uint8 else rows.float().cpu().numpy())
                 if scale is not None:
-                    scales.append(scale[ids, h].cpu().numpy().repeat(wl.PAGE)[:n])
+                    scales.append(scale[ids, h].cpu().numpy().repeat(page)[:n])
         empty = np.zeros((0, dp.cfg.d), dtype=np.uint8 if pool.dtype == torch.uint8 else np.float32)
         rows = np.concatenate(parts, axis=0) if parts else empty
         if scale is not None:      # an e4m3 cache: the codes and each token's scale, for the caller to decode

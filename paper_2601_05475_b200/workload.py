@@ -15,8 +15,9 @@ The five configurations below encode those shapes as G prompt groups x C
 candidates, one shared prefix per group and one private suffix per candidate.
 
 Storage layout produced here (and consumed by the CUDA library):
-  K pool, V pool : [num_pages][Hkv][16][d]   one (page, kv-head) slab is
-                                              16*d contiguous elements
+  K pool, V pool : [num_pages][Hkv][page][d] one (page, kv-head) slab is
+                                              page*d contiguous elements (page = 16
+                                              tokens unless the configuration says 32 or 64)
   prefix_pages   : int32 [G][max_prefix_pages]
   suffix_pages   : int32 [B][max_suffix_pages]
   prefix_len     : int32 [G]      tokens
@@ -84,6 +85,7 @@ class Config:
     k_outlier_scale: float = 1.0
     append_steps: int = 0           # extra decode steps, one appended token per candidate each
     seed: int = 0
+    page: int = PAGE                # tokens per cache page: 16, 32 or 64
 
     @property
     def B(self) -> int:
@@ -181,7 +183,7 @@ class PageTables:
 
 def build_page_tables(cfg: Config, prefix_len: np.ndarray, suffix_len: np.ndarray,
                       headroom_tokens: Optional[int] = None, permute: Optional[bool] = None) -> PageTables:
-    """Assign physical pages.  A prefix occupies ceil(P/16) pages (the last one possibly partial); every
+    """Assign physical pages.  A prefix occupies ceil(P/page) pages (the last one possibly partial); every
     candidate's suffix starts on a fresh page of its own and is pre-assigned enough pages for
     `headroom_tokens` appended tokens, so appends never need an allocator.  With `permute`, one uniform
     random permutation over all physical page ids of the pool is applied (Fisher-Yates, seeded)."""
@@ -189,8 +191,8 @@ def build_page_tables(cfg: Config, prefix_len: np.ndarray, suffix_len: np.ndarra
         headroom_tokens = cfg.append_steps + 1
     if permute is None:
         permute = cfg.permute_pages
-    npp = (prefix_len.astype(np.int64) + PAGE - 1) // PAGE
-    nsp = (suffix_len.astype(np.int64) + headroom_tokens + PAGE - 1) // PAGE
+    npp = (prefix_len.astype(np.int64) + cfg.page - 1) // cfg.page
+    nsp = (suffix_len.astype(np.int64) + headroom_tokens + cfg.page - 1) // cfg.page
     num_pages = int(npp.sum() + nsp.sum())
     max_pp = max(1, int(npp.max(initial=0)))
     max_sp = max(1, int(nsp.max(initial=0)))
@@ -280,7 +282,7 @@ class HostProblem:
     v_prefix: List[np.ndarray]
     k_suffix: List[np.ndarray]      # per candidate [s_b][Hkv][d] float32 (grows with append())
     v_suffix: List[np.ndarray]
-    k_pool: np.ndarray              # [num_pages][Hkv][16][d] storage dtype
+    k_pool: np.ndarray              # [num_pages][Hkv][page][d] storage dtype
     v_pool: np.ndarray
     outer: List["HostLevel"] = dataclasses.field(default_factory=list)   # outer cascade levels, if any
 
@@ -314,7 +316,7 @@ def add_outer_level(hp: "HostProblem", group_offsets: Sequence[int], lengths: Se
     lengths = np.asarray(lengths, dtype=np.int32)
     go = np.asarray(group_offsets, dtype=np.int32)
     n_groups = len(lengths)
-    npp = (lengths.astype(np.int64) + PAGE - 1) // PAGE
+    npp = (lengths.astype(np.int64) + cfg.page - 1) // cfg.page
     first = hp.k_pool.shape[0]
     extra = int(npp.sum())
     ids = np.arange(first, first + extra, dtype=np.int32)
@@ -346,10 +348,11 @@ def _scatter(pool: np.ndarray, pages_row: np.ndarray, tokens: np.ndarray, cfg: C
     """Write logical rows tokens[n][Hkv][d] into the pool through one page-table row."""
     n = tokens.shape[0]
     st = storage_array(cfg, tokens)
-    for p in range((n + PAGE - 1) // PAGE):
-        lo, hi = p * PAGE, min(n, (p + 1) * PAGE)
+    page = pool.shape[2]
+    for p in range((n + page - 1) // page):
+        lo, hi = p * page, min(n, (p + 1) * page)
         pid = int(pages_row[p])
-        # pool[pid] is [Hkv][16][d]; tokens are [t][Hkv][d]
+        # pool[pid] is [Hkv][page][d]; tokens are [t][Hkv][d]
         pool[pid, :, :hi - lo, :] = np.transpose(st[lo:hi], (1, 0, 2))
 
 
@@ -367,7 +370,7 @@ def make_host_problem(cfg: Config, *, headroom_tokens: Optional[int] = None, per
     k_suffix = [_draw_k(cfg, _T_KS, b, int(suffix_len[b])) for b in range(cfg.B)]
     v_suffix = [_round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_VS, b), (int(suffix_len[b]), cfg.Hkv, cfg.d)))
                 for b in range(cfg.B)]
-    shape = (tables.num_pages, cfg.Hkv, PAGE, cfg.d)
+    shape = (tables.num_pages, cfg.Hkv, cfg.page, cfg.d)
     fill = storage_array(cfg, np.full(1, SENTINEL, dtype=np.float32))[0]
     k_pool = np.full(shape, fill, dtype=fill.dtype)
     v_pool = np.full(shape, fill, dtype=fill.dtype)
@@ -404,11 +407,12 @@ def gather_logical(pool: np.ndarray, pages_row: Sequence[int], n_tokens: int, h:
     """Read n_tokens rows of kv head h back out of a pool image through a page-table row:
     returns [n_tokens][d] in the pool's storage dtype.  Plain indexing, used by tests that hold only the
     paged image (device-generated pools)."""
-    n_pages = (n_tokens + PAGE - 1) // PAGE
+    page = pool.shape[2]
+    n_pages = (n_tokens + page - 1) // page
     if n_pages == 0:
         return np.zeros((0, pool.shape[-1]), dtype=pool.dtype)
     ids = np.asarray(pages_row[:n_pages], dtype=np.int64)
-    return pool[ids, h].reshape(n_pages * PAGE, pool.shape[-1])[:n_tokens]
+    return pool[ids, h].reshape(n_pages * page, pool.shape[-1])[:n_tokens]
 
 
 # ----------------------------------------------------------------------------

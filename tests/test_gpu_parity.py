@@ -476,7 +476,7 @@ def test_host_errors_are_returned_immediately():
     assert L.mc_decode_attn(dp.layout, 0, cfg.scale, dp.o.data_ptr(), dp.lse.data_ptr(), dp.ws_ptr, dp.ws_bytes,
                             0) == mc.MC_ERR_INVALID_ARG
     bad = mc.LayoutDesc.from_buffer_copy(dp.desc)
-    bad.page_size = 32
+    bad.page_size = 48
     h = mc.c_void_p()
     assert L.mc_kv_layout_create(mc.byref(bad), mc.byref(h)) == mc.MC_ERR_UNSUPPORTED and not h.value
     bad = mc.LayoutDesc.from_buffer_copy(dp.desc)
