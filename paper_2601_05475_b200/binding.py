@@ -1,4 +1,4 @@
-"""ctypes binding of the C-ABI library (include/maxcode_attn.h): same names, argument marshalling only.
+"""ctypes binding of the C-ABI library (include/maxcode_attn.h, maxcode_search.h, maxcode_qkv.h): same names, argument marshalling only.
 
 Device buffers are torch tensors (torch is used for device memory and streams only); every entry point
 takes raw device pointers.  There is no fallback: if the shared library is missing or fails to load,
@@ -68,6 +68,10 @@ EXPORTS = {
     "mc_search_group_argmax": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
     "mc_search_select": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                    c_void_p]),
+    "mc_qkv_plan_create": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, POINTER(c_void_p)]),
+    "mc_qkv_plan_destroy": (c_int32, [c_void_p]),
+    "mc_qkv_plan_geometry": (c_int32, [c_void_p, POINTER(c_int32), POINTER(c_int32), POINTER(c_size_t)]),
+    "mc_qkv_append": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_double, c_void_p]),
 }
 
 
@@ -241,3 +245,24 @@ def mc_search_select(logits, traj_return, group_offsets, P: int, prob=None, expe
                      best_expected=None, stream: int = 0) -> None:
     _check(lib().mc_search_select(_ptr(logits), _ptr(traj_return), _ptr(group_offsets), P, _ptr(prob), _ptr(expected),
                                   _ptr(best_return), _ptr(best_expected), stream), "mc_search_select")
+
+
+def mc_qkv_plan_create(layout: int, w_qkv, bias, hidden: int) -> int:
+    h = c_void_p()
+    _check(lib().mc_qkv_plan_create(layout, _ptr(w_qkv), _ptr(bias), hidden, byref(h)), "mc_qkv_plan_create")
+    return h.value
+
+
+def mc_qkv_plan_destroy(plan: int) -> None:
+    _check(lib().mc_qkv_plan_destroy(plan), "mc_qkv_plan_destroy")
+
+
+def mc_qkv_plan_geometry(plan: int):
+    """(splits, ctas, workspace_bytes)"""
+    s, c, w = c_int32(), c_int32(), c_size_t()
+    _check(lib().mc_qkv_plan_geometry(plan, byref(s), byref(c), byref(w)), "mc_qkv_plan_geometry")
+    return s.value, c.value, w.value
+
+
+def mc_qkv_append(plan: int, x, q_out, pos_offset=None, theta_base: float = 0.0, stream: int = 0) -> None:
+    _check(lib().mc_qkv_append(plan, _ptr(x), _ptr(q_out), _ptr(pos_offset), theta_base, stream), "mc_qkv_append")

@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "maxcode_qkv.h"
 #include "mc_internal.cuh"
 
 namespace mc {
@@ -175,6 +176,84 @@ __global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels l
   }
   __syncthreads();  // every thread has read s and issued its stores before the length moves
   if (threadIdx.x == 0) suffix_len[b] = s + 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// the q/k/v projection's second half: one block per candidate adds up the pieces of the product (fp32 partial
+// sums [piece][row][feature], in piece order), adds the bias, rotates the query and key heads to the new token's
+// position exactly as append_rope_kernel does, writes q and stores k and v as the candidate's next suffix token.
+// Heads are 128 features wide: thread (i, lane) handles the pair (i, i + 64) of the heads lane, lane + 4, ...
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) qkv_finish_kernel(Params p, RopeLevels lv, const float *__restrict__ partial,
+                                                         int splits, int row_stride, int N,
+                                                         const __nv_bfloat16 *__restrict__ bias,
+                                                         __nv_bfloat16 *__restrict__ q_out,
+                                                         const int32_t *__restrict__ pos_offset, double log2_base,
+                                                         int32_t *suffix_len) {
+  // launched as the programmatic dependent of the product: nothing is read before that grid has completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  const int b = blockIdx.x;
+  const int s = suffix_len[b];
+  const int pg = s >> 4;
+  int page = -1;
+  if (s >= 0 && pg < p.max_sp) page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + pg);
+  const bool store_kv = (unsigned)page < (unsigned)p.num_pages;
+  if (!store_kv && threadIdx.x == 0) latch(p, kDevBadPage);   // row full, or a bad table entry: q only
+  long long pos = s < 0 ? 0 : s;
+  if (pos_offset) {
+    pos += __ldg(pos_offset + b);
+  } else {
+    for (int k = 0; k < lv.n; ++k) {
+      int lo = 0, hi = lv.G[k];
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(lv.group_offsets[k] + mid) <= b) lo = mid; else hi = mid;
+      }
+      pos += max(__ldg(lv.prefix_len[k] + lo), 0);
+    }
+  }
+  constexpr int kD = 128, kHalf = 64;
+  const int i = threadIdx.x % kHalf, h0 = threadIdx.x / kHalf, lanes = blockDim.x / kHalf;
+  float c = 1.f, sf = 0.f;
+  if (log2_base != 0.0) {
+    double sn, cs;
+    sincos((double)pos * exp2(-2.0 * i / kD * log2_base), &sn, &cs);
+    c = (float)cs;
+    sf = (float)sn;
+  }
+  __nv_bfloat16 *kp = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(p.k_pool));
+  __nv_bfloat16 *vp = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(p.v_pool));
+  const int heads = p.Hq + 2 * p.Hkv;
+  for (int head = h0; head < heads; head += lanes) {
+    const size_t n0 = (size_t)head * kD + i;
+    float re = 0.f, im = 0.f;
+    for (int piece = 0; piece < splits; ++piece) {
+      const float *src = partial + ((size_t)piece * row_stride + b) * N + n0;
+      re += src[0];
+      im += src[kHalf];
+    }
+    if (bias) {
+      re += __bfloat162float(bias[n0]);
+      im += __bfloat162float(bias[n0 + kHalf]);
+    }
+    if (head < p.Hq + p.Hkv) {   // queries and keys turn, values do not
+      const float r2 = re * c - im * sf, i2 = re * sf + im * c;
+      re = r2;
+      im = i2;
+    }
+    __nv_bfloat16 *dst;
+    if (head < p.Hq) {
+      dst = q_out + ((size_t)b * p.Hq + head) * kD;
+    } else {
+      if (!store_kv) continue;
+      const int h = head < p.Hq + p.Hkv ? head - p.Hq : head - p.Hq - p.Hkv;
+      dst = (head < p.Hq + p.Hkv ? kp : vp) + (slab_index(p, page, h) * kPage + (s & 15)) * kD;
+    }
+    dst[i] = __float2bfloat16_rn(re);
+    dst[i + kHalf] = __float2bfloat16_rn(im);
+  }
+  __syncthreads();  // every thread has read s and issued its stores before the length moves
+  if (threadIdx.x == 0 && store_kv) suffix_len[b] = s + 1;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -887,6 +966,87 @@ mc_status_t mc_kv_append_rope(mc_kv_layout_t *layout, const void *k_new, const v
         reinterpret_cast<__nv_bfloat16 *>(q), pos_offset, l2b, L->desc.suffix_len);
   mc::count_launch();
   return mc::check_launch();
+}
+
+struct mc_qkv_plan {
+  Layout *L;
+  mc::QkvPlan *gemm;
+  const void *bias;
+};
+
+mc_status_t mc_qkv_plan_create(mc_kv_layout_t *layout, const void *w_qkv, const void *bias, int32_t hidden,
+                               mc_qkv_plan_t **out) {
+  if (out) *out = nullptr;
+  Layout *L = reinterpret_cast<Layout *>(layout);
+  if (!L || !out || !w_qkv || !mc::aligned16(w_qkv) || (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)))
+    return MC_ERR_INVALID_ARG;
+  if (hidden < 64 || hidden % 64 != 0) return MC_ERR_INVALID_ARG;
+  if (L->desc.dtype != MC_BF16 || L->p.d != 128 || !L->has_suffix) return MC_ERR_UNSUPPORTED;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    sms = 148;
+  (void)cudaGetLastError();
+  mc_qkv_plan *pl = new (std::nothrow) mc_qkv_plan();
+  if (!pl) return MC_ERR_OUT_OF_MEMORY;
+  pl->L = L;
+  pl->bias = bias;
+  pl->gemm = mc::qkv_plan(L->p.B, L->p.Hq + 2 * L->p.Hkv, hidden, w_qkv, sms);
+  if (!pl->gemm) {
+    delete pl;
+    return MC_ERR_OUT_OF_MEMORY;
+  }
+  *out = pl;
+  return MC_OK;
+}
+
+mc_status_t mc_qkv_plan_destroy(mc_qkv_plan_t *plan) {
+  if (!plan) return MC_OK;
+  mc::qkv_plan_free(plan->gemm);
+  delete plan;
+  return MC_OK;
+}
+
+mc_status_t mc_qkv_plan_geometry(const mc_qkv_plan_t *plan, int32_t *splits, int32_t *ctas, size_t *workspace_bytes) {
+  if (!plan) return MC_ERR_INVALID_ARG;
+  if (splits) *splits = mc::qkv_splits(plan->gemm);
+  if (ctas) *ctas = mc::qkv_ctas(plan->gemm);
+  if (workspace_bytes) *workspace_bytes = mc::qkv_workspace_bytes(plan->gemm);
+  return MC_OK;
+}
+
+mc_status_t mc_qkv_append(mc_qkv_plan_t *plan, const void *x, void *q_out, const int32_t *pos_offset,
+                          double theta_base, void *stream) {
+  if (!plan || !x || !q_out || !mc::aligned16(x) || !mc::aligned16(q_out)) return MC_ERR_INVALID_ARG;
+  if (theta_base < 0.0 || (theta_base == 0.0 && pos_offset)) return MC_ERR_INVALID_ARG;
+  Layout *L = plan->L;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  mc_status_t s = mc::launch_qkv_gemm(plan->gemm, x, L->dev_status, st);
+  if (s != MC_OK) return s;
+  mc::RopeLevels lv;
+  lv.n = 1 + L->n_outer;
+  for (int k = 0; k < lv.n; ++k) {
+    const mc::Params &pk = k == 0 ? L->p : L->outer_p[k - 1];
+    lv.G[k] = pk.G;
+    lv.group_offsets[k] = pk.group_offsets;
+    lv.prefix_len[k] = pk.prefix_len;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)L->p.B);
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = mc::env_int("MC_PDL", 1) ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(
+      &cfg, mc::qkv_finish_kernel, L->p, lv, mc::qkv_partials(plan->gemm), mc::qkv_splits(plan->gemm),
+      mc::qkv_row_stride(plan->gemm), (L->p.Hq + 2 * L->p.Hkv) * 128, reinterpret_cast<const __nv_bfloat16 *>(plan->bias),
+      reinterpret_cast<__nv_bfloat16 *>(q_out), pos_offset, theta_base > 0.0 ? std::log2(theta_base) : 0.0,
+      L->desc.suffix_len);
+  mc::count_launch();
+  return e == cudaSuccess ? mc::check_launch() : MC_ERR_CUDA;
 }
 
 mc_status_t mc_kv_append_tokens(mc_kv_layout_t *layout, const void *k_new, const void *v_new, int32_t n_max,

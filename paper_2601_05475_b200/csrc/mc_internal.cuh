@@ -160,4 +160,16 @@ mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_
 mc_status_t launch_append_tokens_fp8(const Params &p, const void *k_new, const void *v_new, int n_max,
                                      const int32_t *n_new, const int32_t *suffix_len, cudaStream_t stream);
 
+// The q/k/v projection y = x W^T on the tensor cores (bf16, heads of 128 features): fp32 partial sums
+// [piece][row stride][N] of `splits` pieces of the hidden dimension, in a workspace the plan owns
+struct QkvPlan;
+QkvPlan *qkv_plan(int B, int heads, int hidden, const void *w, int sms);
+void qkv_plan_free(QkvPlan *plan);
+int qkv_splits(const QkvPlan *plan);
+int qkv_ctas(const QkvPlan *plan);
+int qkv_row_stride(const QkvPlan *plan);
+size_t qkv_workspace_bytes(const QkvPlan *plan);
+const float *qkv_partials(const QkvPlan *plan);
+mc_status_t launch_qkv_gemm(const QkvPlan *plan, const void *x, int32_t *status, cudaStream_t stream);
+
 }  // namespace mc

@@ -1,5 +1,5 @@
 // Log-sum-exp merge of the per-part partial results: one warp per output row, lanes split the head
-// dimension.  Reads only the parts whose lse is finite.
+// dimension.  Reads only the parts whose lse is finite, several of them at a time.
 #include "mc_internal.cuh"
 
 namespace mc {
@@ -54,21 +54,40 @@ merge_lse_kernel(int rows, int n_parts, const float *__restrict__ o_part, const 
   for (int c = 0; c < VEC; ++c) acc[c] = 0.f;
   float s = 0.f;
   if (m > -INFINITY) {
+    // Lane i of a batch holds the weight of part base + i; the rows of up to kBatch parts are then fetched together,
+    // so the merge pays one memory round trip per batch and not one per part.  An empty part has weight 0 and its
+    // row (which may hold anything) is not read.
+    constexpr int kBatch = 8;
     const float *op = o_part + (size_t)row * n_parts * D + lane * VEC;
-    for (int i = 0; i < n_parts; ++i) {
-      const float li = lp[i];  // same address in every lane: one broadcast load
-      if (li == -INFINITY) continue;
-      const float w = expf(li - m);
+    for (int base = 0; base < n_parts; base += 32) {
+      const float li = base + lane < n_parts ? lp[base + lane] : -INFINITY;
+      const float w = li == -INFINITY ? 0.f : expf(li - m);
       s += w;
-      if constexpr (VEC == 4) {
-        const float4 v = *reinterpret_cast<const float4 *>(op + (size_t)i * D);
-        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
-        acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
-      } else {
-        const float2 v = *reinterpret_cast<const float2 *>(op + (size_t)i * D);
-        acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+      const int cnt = min(32, n_parts - base);
+      for (int i0 = 0; i0 < cnt; i0 += kBatch) {
+        float wi[kBatch], v[kBatch][VEC];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          wi[k] = __shfl_sync(0xffffffffu, w, (i0 + k) & 31);   // lanes past the last part hold 0
+          const float *src = op + (size_t)(base + i0 + k) * D;
+          if constexpr (VEC == 4) {
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (wi[k] != 0.f) t = *reinterpret_cast<const float4 *>(src);
+            v[k][0] = t.x; v[k][1] = t.y; v[k][2] = t.z; v[k][3] = t.w;
+          } else {
+            float2 t = make_float2(0.f, 0.f);
+            if (wi[k] != 0.f) t = *reinterpret_cast<const float2 *>(src);
+            v[k][0] = t.x; v[k][1] = t.y;
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+          for (int c = 0; c < VEC; ++c) acc[c] = fmaf(wi[k], v[k][c], acc[c]);
       }
     }
+#pragma unroll
+    for (int sh = 16; sh >= 1; sh >>= 1) s += __shfl_xor_sync(0xffffffffu, s, sh);
     const float inv = 1.f / s;
 #pragma unroll
     for (int c = 0; c < VEC; ++c) acc[c] *= inv;

@@ -39,6 +39,7 @@ PAGE = 16
 
 # tensor ids for sub-stream derivation: (seed, tensor id, index) -> SeedSequence
 _T_PREFIX_LEN, _T_SUFFIX_LEN, _T_PERM, _T_Q, _T_KP, _T_VP, _T_KS, _T_VS, _T_OUTLIER, _T_KNEW, _T_VNEW = range(11)
+_T_HIDDEN, _T_WQKV, _T_BQKV = 11, 12, 13
 
 # Finite, large filler for page slots past a sequence's length: a kernel that
 # fails to mask them produces visibly wrong results instead of silently
@@ -257,6 +258,21 @@ def draw_append(cfg: Config, step: int) -> Tuple[np.ndarray, np.ndarray]:
     k = _round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_KNEW, step), (cfg.B, cfg.Hkv, cfg.d)))
     v = _round_to_dtype(cfg, _normal(_rng(cfg.seed, _T_VNEW, step), (cfg.B, cfg.Hkv, cfg.d)))
     return k, v
+
+
+def draw_hidden(cfg: Config, step: int, hidden: int) -> np.ndarray:
+    """Hidden states [B][hidden] entering the projection of decode step `step`: N(0, 1), bf16-representable float32."""
+    return bf16_bits_to_f32(f32_to_bf16_bits(_normal(_rng(cfg.seed, _T_HIDDEN, step), (cfg.B, hidden))))
+
+
+def draw_qkv_weights(cfg: Config, hidden: int, with_bias: bool = True) -> Tuple[np.ndarray, Optional[np.ndarray]]:
+    """Projection weights [(Hq + 2 Hkv) d][hidden], N(0, 1 / hidden) so that a projected feature is N(0, 1) like the
+    queries and keys of the other generators, and a bias [(Hq + 2 Hkv) d], N(0, 0.25); bf16-representable float32."""
+    n = (cfg.Hq + 2 * cfg.Hkv) * cfg.d
+    w = _normal(_rng(cfg.seed, _T_WQKV), (n, hidden)) * np.float32(1.0 / math.sqrt(hidden))
+    b = _normal(_rng(cfg.seed, _T_BQKV), (n,)) * np.float32(0.5) if with_bias else None
+    rnd = lambda a: bf16_bits_to_f32(f32_to_bf16_bits(np.ascontiguousarray(a, dtype=np.float32)))
+    return rnd(w), (rnd(b) if b is not None else None)
 
 
 def draw_single_head_history(cfg: Config, index: int, n_tokens: int) -> Tuple[np.ndarray, np.ndarray]:
