@@ -532,6 +532,57 @@ def run_gpu(args):
                 "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "flops": flops, "prefix_ctas": ctas, "n_parts": n_parts,
                 "launches_per_pass": int(launches), "scored_tokens_per_s": round(nv / (ms * 1e-3), 1), "status_ok": ok}
 
+    def measure_qkv():
+        """The decode layer's step in front of the attention (q/k/v projection + rotary embedding + append, fused):
+        configuration 4's 128 candidates, Hq 64 / Hkv 8 / d 128 and a hidden size of 8192 (the width of the 70B-class
+        models those head counts belong to): 168 MB of weights per call, streamed once.  Bytes = weights + hidden
+        states + the bf16 rows written; the plain library GEMM of the same shape (torch.matmul, no rotation, no
+        append) is timed beside it for context."""
+        qcfg = wl.scaled_down(wl.CONFIGS["cfg4"], "qkv", prefix=("fixed", 64), suffix=("fixed", (0,)), append_steps=0)
+        hidden, reps = 8192, 100
+        n = (qcfg.Hq + 2 * qcfg.Hkv) * qcfg.d
+        dp = make_device_problem(qcfg, headroom_tokens=4 * reps)
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(1234)
+        w = (torch.randn(n, hidden, device="cuda", generator=gen) * hidden ** -0.5).to(torch.bfloat16)
+        xs = [torch.randn(qcfg.B, hidden, device="cuda", generator=gen).to(torch.bfloat16) for _ in range(4)]
+        q_out = torch.empty(qcfg.B, qcfg.Hq, qcfg.d, dtype=torch.bfloat16, device="cuda")
+        plan = mc.mc_qkv_plan_create(dp.layout, w, None, hidden)
+        stream = torch.cuda.current_stream().cuda_stream
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn):
+            for i in range(5):
+                fn(i)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(reps):
+                fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        launches = mc.mc_launch_count()
+        ms = timed(lambda i: mc.mc_qkv_append(plan, xs[i % 4], q_out, None, 500000.0, stream))
+        launches = (mc.mc_launch_count() - launches) // (reps + 5)
+        ok = mc.mc_get_last_status(dp.layout) == mc.MC_OK
+        y = torch.empty(qcfg.B, n, dtype=torch.bfloat16, device="cuda")
+        ms_lib = timed(lambda i: torch.matmul(xs[i % 4], w.t(), out=y))
+        pieces, ctas, ws = mc.mc_qkv_plan_geometry(plan)
+        mc.mc_qkv_plan_destroy(plan)
+        dp.close()
+        nbytes = n * hidden * 2 + qcfg.B * hidden * 2 + qcfg.B * n * 2
+        return {"candidates": qcfg.B, "hidden": hidden, "features": n, "ms": round(ms, 5),
+                "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1), "tflops": round(2.0 * qcfg.B * n * hidden / (ms * 1e-3) / 1e12, 1),
+                "algorithmic_bytes": nbytes, "launches": int(launches), "ctas": ctas, "pieces": pieces,
+                "workspace_bytes": ws, "status_ok": ok, "library_gemm_alone_ms": round(ms_lib, 5),
+                "l2": "weights (168 MB) larger than L2, no flush"}
+
+    if args.qkv_only:          # profiling aid: only the fused projection, one small JSON line
+        if rank == 0:
+            print(json.dumps({"qkv_projection": measure_qkv()}))
+        return 0
+
     if args.pass_only:         # profiling aid: one pass alone on the launching stream, one small JSON line
         cfg = wl.CONFIGS[args.workload]
         if args.kv_dtype:
@@ -584,6 +635,7 @@ def run_gpu(args):
     read_peak = measure_read_peak() if args.all_configs else None
 
     scoring = measure_scoring() if args.all_configs else None
+    qkv = measure_qkv() if args.all_configs else None
 
     # max over ranks of the step time
     ms, e2e_ms = max_over_ranks([main["ms"], main["e2e_ms"]], device="cuda")
@@ -668,6 +720,7 @@ def run_gpu(args):
             "search_bookkeeping": (dict(search, frac_of_measured_hbm=round(search["gbs"] / peak, 4)) if search else None),
             "scoring_attention": (dict(scoring, bound="tensor", frac_of_measured_bf16=(
                 round(scoring["tflops"] / peaks["bf16_tflops"], 4) if peaks.get("bf16_tflops") else None)) if scoring else None),
+            "qkv_projection": (dict(qkv, bound="hbm", frac_of_measured_hbm=round(qkv["gbs"] / peak, 4)) if qkv else None),
         }
         print(json.dumps(line))
     if world > 1:
@@ -685,6 +738,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false",
                     help="skip the CPU-oracle leg (profiling runs only; the default run reports it)")
     ap.add_argument("--scoring-only", action="store_true", help="run only the scoring pass (profiling aid)")
+    ap.add_argument("--qkv-only", action="store_true", help="run only the fused q/k/v projection (profiling aid)")
     ap.add_argument("--pass-only", choices=["suffix", "prefix"], default=None,
                     help="run only that pass of --workload, alone (profiling aid)")
     ap.add_argument("--kv-dtype", choices=["bf16", "fp8"], default=None,

@@ -179,81 +179,131 @@ __global__ void __launch_bounds__(256) append_rope_kernel(Params p, RopeLevels l
 }
 
 // ------------------------------------------------------------------------------------------------
-// the q/k/v projection's second half: one block per candidate adds up the pieces of the product (fp32 partial
-// sums [piece][row][feature], in piece order), adds the bias, rotates the query and key heads to the new token's
-// position exactly as append_rope_kernel does, writes q and stores k and v as the candidate's next suffix token.
-// Heads are 128 features wide: thread (i, lane) handles the pair (i, i + 64) of the heads lane, lane + 4, ...
+// the q/k/v projection around its product.  Before it: one block per candidate looks up where the new token goes
+// (page and slot, from the length and the page table) and how far it turns (cosine and sine of every pair's angle,
+// formed in double precision as in append_rope_kernel), leaves both for the finishing kernel and moves the length;
+// the product, which needs none of this, runs meanwhile.  After it: block (b, y) adds up, for candidate b and four
+// heads, the pieces of the product (fp32 partial sums [piece][row][feature]; the pieces of a head pair are those of
+// the CTAs whose runs of k-blocks touch it, in CTA order), adds the bias, rotates the query and key heads, writes
+// q and stores k and v in the token's slot.  Heads are 128 features wide: a thread handles four neighbouring
+// pairs (i, i + 64) of one of the block's sixteen heads; all its loads (16 bytes each, up to eight pieces) are
+// independent of one another and in flight together.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) qkv_finish_kernel(Params p, RopeLevels lv, const float *__restrict__ partial,
-                                                         int splits, int row_stride, int N,
-                                                         const __nv_bfloat16 *__restrict__ bias,
-                                                         __nv_bfloat16 *__restrict__ q_out,
-                                                         const int32_t *__restrict__ pos_offset, double log2_base,
-                                                         int32_t *suffix_len) {
-  // launched as the programmatic dependent of the product: nothing is read before that grid has completed
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+struct QkvToken { int32_t page, s; };   // page < 0: the candidate has no room (or a bad table entry): q only
+
+__global__ void __launch_bounds__(64) qkv_prep_kernel(Params p, RopeLevels lv, const int32_t *__restrict__ pos_offset,
+                                                      double log2_base, int32_t *suffix_len, QkvToken *tok,
+                                                      float2 *rot) {
+  // the product is launched behind this kernel as its programmatic dependent and may start at once
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  constexpr int kD = 128;
   const int b = blockIdx.x;
   const int s = suffix_len[b];
   const int pg = s >> 4;
   int page = -1;
   if (s >= 0 && pg < p.max_sp) page = __ldg(p.suffix_pages + (size_t)b * p.max_sp + pg);
   const bool store_kv = (unsigned)page < (unsigned)p.num_pages;
-  if (!store_kv && threadIdx.x == 0) latch(p, kDevBadPage);   // row full, or a bad table entry: q only
-  long long pos = s < 0 ? 0 : s;
-  if (pos_offset) {
-    pos += __ldg(pos_offset + b);
-  } else {
-    for (int k = 0; k < lv.n; ++k) {
-      int lo = 0, hi = lv.G[k];
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(lv.group_offsets[k] + mid) <= b) lo = mid; else hi = mid;
-      }
-      pos += max(__ldg(lv.prefix_len[k] + lo), 0);
-    }
-  }
-  constexpr int kD = 128, kHalf = 64;
-  const int i = threadIdx.x % kHalf, h0 = threadIdx.x / kHalf, lanes = blockDim.x / kHalf;
-  float c = 1.f, sf = 0.f;
+  float2 r = make_float2(1.f, 0.f);
   if (log2_base != 0.0) {
-    double sn, cs;
-    sincos((double)pos * exp2(-2.0 * i / kD * log2_base), &sn, &cs);
-    c = (float)cs;
-    sf = (float)sn;
-  }
-  __nv_bfloat16 *kp = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(p.k_pool));
-  __nv_bfloat16 *vp = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(p.v_pool));
-  const int heads = p.Hq + 2 * p.Hkv;
-  for (int head = h0; head < heads; head += lanes) {
-    const size_t n0 = (size_t)head * kD + i;
-    float re = 0.f, im = 0.f;
-    for (int piece = 0; piece < splits; ++piece) {
-      const float *src = partial + ((size_t)piece * row_stride + b) * N + n0;
-      re += src[0];
-      im += src[kHalf];
-    }
-    if (bias) {
-      re += __bfloat162float(bias[n0]);
-      im += __bfloat162float(bias[n0 + kHalf]);
-    }
-    if (head < p.Hq + p.Hkv) {   // queries and keys turn, values do not
-      const float r2 = re * c - im * sf, i2 = re * sf + im * c;
-      re = r2;
-      im = i2;
-    }
-    __nv_bfloat16 *dst;
-    if (head < p.Hq) {
-      dst = q_out + ((size_t)b * p.Hq + head) * kD;
+    long long pos = s < 0 ? 0 : s;
+    if (pos_offset) {
+      pos += __ldg(pos_offset + b);
     } else {
-      if (!store_kv) continue;
-      const int h = head < p.Hq + p.Hkv ? head - p.Hq : head - p.Hq - p.Hkv;
-      dst = (head < p.Hq + p.Hkv ? kp : vp) + (slab_index(p, page, h) * kPage + (s & 15)) * kD;
+      for (int k = 0; k < lv.n; ++k) {
+        int lo = 0, hi = lv.G[k];
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (__ldg(lv.group_offsets[k] + mid) <= b) lo = mid; else hi = mid;
+        }
+        pos += max(__ldg(lv.prefix_len[k] + lo), 0);
+      }
     }
-    dst[i] = __float2bfloat16_rn(re);
-    dst[i + kHalf] = __float2bfloat16_rn(im);
+    double sn, cs;
+    sincos((double)pos * exp2(-2.0 * threadIdx.x / kD * log2_base), &sn, &cs);
+    r = make_float2((float)cs, (float)sn);
   }
-  __syncthreads();  // every thread has read s and issued its stores before the length moves
-  if (threadIdx.x == 0 && store_kv) suffix_len[b] = s + 1;
+  rot[(size_t)b * (kD / 2) + threadIdx.x] = r;
+  __syncthreads();   // every thread has read the length before it moves
+  if (threadIdx.x == 0) {
+    tok[b].page = store_kv ? page : -1;
+    tok[b].s = s;
+    if (store_kv) suffix_len[b] = s + 1; else latch(p, kDevBadPage);
+  }
+}
+
+__global__ void __launch_bounds__(256) qkv_finish_kernel(Params p, const float *__restrict__ partial, int ctas,
+                                                         int kb_per_pair, int n_pairs, int row_stride,
+                                                         int feature_stride, const __nv_bfloat16 *__restrict__ bias,
+                                                         __nv_bfloat16 *__restrict__ q_out,
+                                                         const QkvToken *__restrict__ tok,
+                                                         const float2 *__restrict__ rot, int rotate) {
+  // launched as the programmatic dependent of the product, which itself completes only after the kernel above has:
+  // nothing is read before that
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  constexpr int kD = 128, kHalf = 64, kBatch = 8;
+  const int b = blockIdx.x;
+  const int i = (threadIdx.x % 16) * 4, head = blockIdx.y * (blockDim.x / 16) + threadIdx.x / 16;
+  if (head >= p.Hq + 2 * p.Hkv) return;
+  // CTA c of the product holds k-blocks [c T / ctas, (c + 1) T / ctas) of the numbering pair * kb_per_pair + kb
+  const size_t n0 = (size_t)head * kD + i;
+  const long long total = (long long)n_pairs * kb_per_pair, u0 = (long long)(head >> 1) * kb_per_pair;
+  const int pieces = (int)(((u0 + kb_per_pair) * ctas - 1) / total) - (int)(((u0 + 1) * ctas - 1) / total) + 1;
+  const float *src = partial + (size_t)b * feature_stride + n0;
+  const size_t piece_stride = (size_t)row_stride * feature_stride;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 a[kBatch], c8[kBatch];
+#pragma unroll
+  for (int k = 0; k < kBatch; ++k) {
+    a[k] = k < pieces ? *reinterpret_cast<const float4 *>(src + (size_t)k * piece_stride) : zero;
+    c8[k] = k < pieces ? *reinterpret_cast<const float4 *>(src + (size_t)k * piece_stride + kHalf) : zero;
+  }
+  const QkvToken t = tok[b];
+  float re[4] = {0.f, 0.f, 0.f, 0.f}, im[4] = {0.f, 0.f, 0.f, 0.f};
+  float cs[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
+  if (rotate && head < p.Hq + p.Hkv) {   // queries and keys turn, values do not
+    const float4 r01 = *reinterpret_cast<const float4 *>(rot + (size_t)b * kHalf + i);
+    const float4 r23 = *reinterpret_cast<const float4 *>(rot + (size_t)b * kHalf + i + 2);
+    cs[0] = r01.x; sn[0] = r01.y; cs[1] = r01.z; sn[1] = r01.w;
+    cs[2] = r23.x; sn[2] = r23.y; cs[3] = r23.z; sn[3] = r23.w;
+  }
+#pragma unroll
+  for (int k = 0; k < kBatch; ++k) {   // pieces in order
+    re[0] += a[k].x; re[1] += a[k].y; re[2] += a[k].z; re[3] += a[k].w;
+    im[0] += c8[k].x; im[1] += c8[k].y; im[2] += c8[k].z; im[3] += c8[k].w;
+  }
+  for (int k = kBatch; k < pieces; ++k) {   // (more than eight pieces: a grid far wider than the stream is long)
+    const float4 x = *reinterpret_cast<const float4 *>(src + (size_t)k * piece_stride);
+    const float4 y = *reinterpret_cast<const float4 *>(src + (size_t)k * piece_stride + kHalf);
+    re[0] += x.x; re[1] += x.y; re[2] += x.z; re[3] += x.w;
+    im[0] += y.x; im[1] += y.y; im[2] += y.z; im[3] += y.w;
+  }
+  if (bias) {   // the sum of the pieces first, then the bias: one order, whatever the number of pieces
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      re[e] += __bfloat162float(bias[n0 + e]);
+      im[e] += __bfloat162float(bias[n0 + kHalf + e]);
+    }
+  }
+  __nv_bfloat16 *dst;
+  if (head < p.Hq) {
+    dst = q_out + ((size_t)b * p.Hq + head) * kD;
+  } else {
+    if (t.page < 0) return;
+    const bool is_k = head < p.Hq + p.Hkv;
+    const int h = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+    __nv_bfloat16 *pool = reinterpret_cast<__nv_bfloat16 *>(const_cast<void *>(is_k ? p.k_pool : p.v_pool));
+    dst = pool + (slab_index(p, t.page, h) * kPage + (t.s & 15)) * kD;
+  }
+  float o_re[4], o_im[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    o_re[e] = re[e] * cs[e] - im[e] * sn[e];
+    o_im[e] = re[e] * sn[e] + im[e] * cs[e];
+  }
+  __nv_bfloat162 w0 = __floats2bfloat162_rn(o_re[0], o_re[1]), w1 = __floats2bfloat162_rn(o_re[2], o_re[3]);
+  __nv_bfloat162 w2 = __floats2bfloat162_rn(o_im[0], o_im[1]), w3 = __floats2bfloat162_rn(o_im[2], o_im[3]);
+  *reinterpret_cast<uint2 *>(dst + i) = make_uint2(*reinterpret_cast<uint32_t *>(&w0), *reinterpret_cast<uint32_t *>(&w1));
+  *reinterpret_cast<uint2 *>(dst + i + kHalf) = make_uint2(*reinterpret_cast<uint32_t *>(&w2), *reinterpret_cast<uint32_t *>(&w3));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -972,6 +1022,8 @@ struct mc_qkv_plan {
   Layout *L;
   mc::QkvPlan *gemm;
   const void *bias;
+  void *token_info;       // device: per candidate, where its new token goes (QkvToken [B]) and, 256-byte aligned
+                          // behind that, the rotation of its 64 pairs (float2 [B][64])
 };
 
 mc_status_t mc_qkv_plan_create(mc_kv_layout_t *layout, const void *w_qkv, const void *bias, int32_t hidden,
@@ -992,7 +1044,11 @@ mc_status_t mc_qkv_plan_create(mc_kv_layout_t *layout, const void *w_qkv, const 
   pl->L = L;
   pl->bias = bias;
   pl->gemm = mc::qkv_plan(L->p.B, L->p.Hq + 2 * L->p.Hkv, hidden, w_qkv, sms);
-  if (!pl->gemm) {
+  pl->token_info = nullptr;
+  const size_t tok_bytes = mc::align_up(sizeof(mc::QkvToken) * (size_t)L->p.B, 256);
+  if (!pl->gemm || cudaMalloc(&pl->token_info, tok_bytes + sizeof(float2) * 64 * (size_t)L->p.B) != cudaSuccess) {
+    (void)cudaGetLastError();
+    mc::qkv_plan_free(pl->gemm);
     delete pl;
     return MC_ERR_OUT_OF_MEMORY;
   }
@@ -1003,14 +1059,15 @@ mc_status_t mc_qkv_plan_create(mc_kv_layout_t *layout, const void *w_qkv, const 
 mc_status_t mc_qkv_plan_destroy(mc_qkv_plan_t *plan) {
   if (!plan) return MC_OK;
   mc::qkv_plan_free(plan->gemm);
+  cudaFree(plan->token_info);
   delete plan;
   return MC_OK;
 }
 
-mc_status_t mc_qkv_plan_geometry(const mc_qkv_plan_t *plan, int32_t *splits, int32_t *ctas, size_t *workspace_bytes) {
+mc_status_t mc_qkv_plan_geometry(const mc_qkv_plan_t *plan, int32_t *pieces, int32_t *ctas, size_t *workspace_bytes) {
   if (!plan) return MC_ERR_INVALID_ARG;
-  if (splits) *splits = mc::qkv_splits(plan->gemm);
-  if (ctas) *ctas = mc::qkv_ctas(plan->gemm);
+  if (pieces) *pieces = mc::qkv_pieces(plan->gemm);
+  if (ctas) *ctas = mc::qkv_ctas(plan->gemm) * mc::qkv_passes(plan->gemm);
   if (workspace_bytes) *workspace_bytes = mc::qkv_workspace_bytes(plan->gemm);
   return MC_OK;
 }
@@ -1021,8 +1078,6 @@ mc_status_t mc_qkv_append(mc_qkv_plan_t *plan, const void *x, void *q_out, const
   if (theta_base < 0.0 || (theta_base == 0.0 && pos_offset)) return MC_ERR_INVALID_ARG;
   Layout *L = plan->L;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  mc_status_t s = mc::launch_qkv_gemm(plan->gemm, x, L->dev_status, st);
-  if (s != MC_OK) return s;
   mc::RopeLevels lv;
   lv.n = 1 + L->n_outer;
   for (int k = 0; k < lv.n; ++k) {
@@ -1031,20 +1086,31 @@ mc_status_t mc_qkv_append(mc_qkv_plan_t *plan, const void *x, void *q_out, const
     lv.group_offsets[k] = pk.group_offsets;
     lv.prefix_len[k] = pk.prefix_len;
   }
+  mc::QkvToken *tok = reinterpret_cast<mc::QkvToken *>(plan->token_info);
+  float2 *rot = reinterpret_cast<float2 *>(static_cast<unsigned char *>(plan->token_info) +
+                                           mc::align_up(sizeof(mc::QkvToken) * (size_t)L->p.B, 256));
+  const bool pdl = mc::env_int("MC_PDL", 1) != 0;
+  mc::qkv_prep_kernel<<<L->p.B, 64, 0, st>>>(L->p, lv, pos_offset, theta_base > 0.0 ? std::log2(theta_base) : 0.0,
+                                            L->desc.suffix_len, tok, rot);
+  mc::count_launch();
+  if (mc::check_launch() != MC_OK) return MC_ERR_CUDA;
+  mc_status_t s = mc::launch_qkv_gemm(plan->gemm, x, L->dev_status, st, pdl);
+  if (s != MC_OK) return s;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)L->p.B);
+  cfg.gridDim = dim3((unsigned)L->p.B, (unsigned)((L->p.Hq + 2 * L->p.Hkv + 15) / 16));
   cfg.blockDim = dim3(256);
   cfg.stream = st;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = mc::env_int("MC_PDL", 1) ? 1 : 0;
+  cfg.numAttrs = pdl ? 1 : 0;
   const cudaError_t e = cudaLaunchKernelEx(
-      &cfg, mc::qkv_finish_kernel, L->p, lv, mc::qkv_partials(plan->gemm), mc::qkv_splits(plan->gemm),
-      mc::qkv_row_stride(plan->gemm), (L->p.Hq + 2 * L->p.Hkv) * 128, reinterpret_cast<const __nv_bfloat16 *>(plan->bias),
-      reinterpret_cast<__nv_bfloat16 *>(q_out), pos_offset, theta_base > 0.0 ? std::log2(theta_base) : 0.0,
-      L->desc.suffix_len);
+      &cfg, mc::qkv_finish_kernel, L->p, mc::qkv_partials(plan->gemm), mc::qkv_ctas(plan->gemm),
+      mc::qkv_kb_per_pair(plan->gemm), (L->p.Hq + 2 * L->p.Hkv + 1) / 2, mc::qkv_row_stride(plan->gemm),
+      mc::qkv_feature_stride(plan->gemm), reinterpret_cast<const __nv_bfloat16 *>(plan->bias),
+      reinterpret_cast<__nv_bfloat16 *>(q_out), static_cast<const mc::QkvToken *>(tok), static_cast<const float2 *>(rot),
+      theta_base > 0.0 ? 1 : 0);
   mc::count_launch();
   return e == cudaSuccess ? mc::check_launch() : MC_ERR_CUDA;
 }

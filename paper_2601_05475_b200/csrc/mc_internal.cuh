@@ -160,16 +160,25 @@ mc_status_t launch_append_fp8(const Params &p, const void *k_new, const void *v_
 mc_status_t launch_append_tokens_fp8(const Params &p, const void *k_new, const void *v_new, int n_max,
                                      const int32_t *n_new, const int32_t *suffix_len, cudaStream_t stream);
 
-// The q/k/v projection y = x W^T on the tensor cores (bf16, heads of 128 features): fp32 partial sums
-// [piece][row stride][N] of `splits` pieces of the hidden dimension, in a workspace the plan owns
+// The q/k/v projection y = x W^T on the tensor cores (bf16, heads of 128 features).  A persistent grid shares out
+// the k-blocks (64 hidden elements) of all head pairs in equal contiguous runs; the fp32 sums of a run's part of a
+// head pair are a "piece": partials [piece][row stride][feature stride], in a workspace the plan owns.  The pieces of
+// pair r are those of CTAs first(r) .. last(r), piece index = CTA - first(r), where the CTA holding k-block u of
+// the numbering pair * kb_per_pair + kb is ((u + 1) * ctas - 1) / (pairs * kb_per_pair).
 struct QkvPlan;
 QkvPlan *qkv_plan(int B, int heads, int hidden, const void *w, int sms);
 void qkv_plan_free(QkvPlan *plan);
-int qkv_splits(const QkvPlan *plan);
-int qkv_ctas(const QkvPlan *plan);
+int qkv_pieces(const QkvPlan *plan);        // most pieces any head pair has
+int qkv_ctas(const QkvPlan *plan);          // CTAs of one pass
+int qkv_passes(const QkvPlan *plan);        // passes over the candidates (256 rows each at most)
+int qkv_kb_per_pair(const QkvPlan *plan);
 int qkv_row_stride(const QkvPlan *plan);
+int qkv_feature_stride(const QkvPlan *plan);
 size_t qkv_workspace_bytes(const QkvPlan *plan);
 const float *qkv_partials(const QkvPlan *plan);
-mc_status_t launch_qkv_gemm(const QkvPlan *plan, const void *x, int32_t *status, cudaStream_t stream);
+// `beside_previous`: launched as the programmatic dependent of the kernel in front of it, whose completion it awaits
+// before it lets its own dependent start
+mc_status_t launch_qkv_gemm(const QkvPlan *plan, const void *x, int32_t *status, cudaStream_t stream,
+                            bool beside_previous);
 
 }  // namespace mc
