@@ -84,7 +84,8 @@ typedef struct {
   int32_t batch;                 /* B >= 1, total candidates */
   int32_t num_q_heads;           /* Hq, a multiple of Hkv */
   int32_t num_kv_heads;          /* Hkv */
-  int32_t head_dim;              /* d: 64 or 128 */
+  int32_t head_dim;              /* d: 64, 128 or 256 (256: every pass on the plain-ALU kernel; MC_FP8_E4M3, the
+                                    tensor-core passes and mc_decode_attn_static: see their own limits) */
   int32_t page_size;             /* tokens per page: 16, 32 or 64 (MC_FP8_E4M3 and mc_decode_attn_static: 16) */
   int32_t num_pages;             /* pages in each pool */
   int32_t max_prefix_pages;      /* row stride of prefix_pages */

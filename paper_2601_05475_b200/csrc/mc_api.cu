@@ -634,7 +634,7 @@ mc_status_t mc_kv_layout_create_cascade(const mc_kv_layout_desc_t *d, const mc_p
     if ((long long)outer[k].max_pages * upp * mc::kPage > 0x7fffffffLL) return MC_ERR_UNSUPPORTED;
   if (d->dtype == MC_FP8_E4M3 && lr != 0) return MC_ERR_UNSUPPORTED;   // page scales are per 16-token page
   if (d->dtype != MC_F32 && d->dtype != MC_BF16 && d->dtype != MC_FP8_E4M3) return MC_ERR_UNSUPPORTED;
-  if (d->head_dim != 64 && d->head_dim != 128) return MC_ERR_UNSUPPORTED;
+  if (d->head_dim != 64 && d->head_dim != 128 && d->head_dim != 256) return MC_ERR_UNSUPPORTED;
   if ((long long)d->batch * d->num_q_heads > (1ll << 30)) return MC_ERR_UNSUPPORTED;
   const bool fp8 = d->dtype == MC_FP8_E4M3;
   if (fp8 && (!d->k_scale || !d->v_scale || (reinterpret_cast<uintptr_t>(d->k_scale) & 3u) ||

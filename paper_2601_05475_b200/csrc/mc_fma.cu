@@ -24,6 +24,14 @@ struct RowLoad<float, 4> {
     o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
   }
 };
+template <>
+struct RowLoad<float, 8> {
+  static __device__ __forceinline__ void ld(const float *p, float (&o)[8]) {
+    float4 a = __ldg(reinterpret_cast<const float4 *>(p)), b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w;
+    o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+  }
+};
 __device__ __forceinline__ void unpack_bf16x2(uint32_t w, float &lo, float &hi) {
   lo = __uint_as_float(w << 16);
   hi = __uint_as_float(w & 0xffff0000u);
@@ -41,6 +49,17 @@ struct RowLoad<__nv_bfloat16, 4> {
     uint2 w = __ldg(reinterpret_cast<const uint2 *>(p));
     unpack_bf16x2(w.x, o[0], o[1]);
     unpack_bf16x2(w.y, o[2], o[3]);
+  }
+};
+
+template <>
+struct RowLoad<__nv_bfloat16, 8> {
+  static __device__ __forceinline__ void ld(const __nv_bfloat16 *p, float (&o)[8]) {
+    uint4 w = __ldg(reinterpret_cast<const uint4 *>(p));
+    unpack_bf16x2(w.x, o[0], o[1]);
+    unpack_bf16x2(w.y, o[2], o[3]);
+    unpack_bf16x2(w.z, o[4], o[5]);
+    unpack_bf16x2(w.w, o[6], o[7]);
   }
 };
 
@@ -161,9 +180,11 @@ mc_status_t launch_fma(const Params &p, int dtype, int mode, const void *q, floa
   if (dtype == MC_F32) {
     if (p.d == 64) return launch_t<float, 64>(p, mode, q, scale, o_part, lse_part, stream);
     if (p.d == 128) return launch_t<float, 128>(p, mode, q, scale, o_part, lse_part, stream);
+    if (p.d == 256) return launch_t<float, 256>(p, mode, q, scale, o_part, lse_part, stream);
   } else if (dtype == MC_BF16) {
     if (p.d == 64) return launch_t<__nv_bfloat16, 64>(p, mode, q, scale, o_part, lse_part, stream);
     if (p.d == 128) return launch_t<__nv_bfloat16, 128>(p, mode, q, scale, o_part, lse_part, stream);
+    if (p.d == 256) return launch_t<__nv_bfloat16, 256>(p, mode, q, scale, o_part, lse_part, stream);
   }
   return MC_ERR_UNSUPPORTED;
 }

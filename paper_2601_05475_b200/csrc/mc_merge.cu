@@ -19,6 +19,11 @@ __device__ __forceinline__ void store_row<float, 4>(float *dst, const float (&v)
   *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
 }
 template <>
+__device__ __forceinline__ void store_row<float, 8>(float *dst, const float (&v)[8]) {
+  reinterpret_cast<float4 *>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+  reinterpret_cast<float4 *>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+template <>
 __device__ __forceinline__ void store_row<__nv_bfloat16, 2>(__nv_bfloat16 *dst, const float (&v)[2]) {
   *reinterpret_cast<__nv_bfloat162 *>(dst) = __floats2bfloat162_rn(v[0], v[1]);
 }
@@ -29,6 +34,18 @@ __device__ __forceinline__ void store_row<__nv_bfloat16, 4>(__nv_bfloat16 *dst, 
   w.x = *reinterpret_cast<uint32_t *>(&a);
   w.y = *reinterpret_cast<uint32_t *>(&b);
   *reinterpret_cast<uint2 *>(dst) = w;
+}
+
+template <>
+__device__ __forceinline__ void store_row<__nv_bfloat16, 8>(__nv_bfloat16 *dst, const float (&v)[8]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 w;
+  w.x = *reinterpret_cast<uint32_t *>(&a);
+  w.y = *reinterpret_cast<uint32_t *>(&b);
+  w.z = *reinterpret_cast<uint32_t *>(&c);
+  w.w = *reinterpret_cast<uint32_t *>(&d);
+  *reinterpret_cast<uint4 *>(dst) = w;
 }
 
 template <typename T, int D>
@@ -70,7 +87,15 @@ merge_lse_kernel(int rows, int n_parts, const float *__restrict__ o_part, const 
         for (int k = 0; k < kBatch; ++k) {
           wi[k] = __shfl_sync(0xffffffffu, w, (i0 + k) & 31);   // lanes past the last part hold 0
           const float *src = op + (size_t)(base + i0 + k) * D;
-          if constexpr (VEC == 4) {
+          if constexpr (VEC == 8) {
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f), t2 = t;
+            if (wi[k] != 0.f) {
+              t = reinterpret_cast<const float4 *>(src)[0];
+              t2 = reinterpret_cast<const float4 *>(src)[1];
+            }
+            v[k][0] = t.x; v[k][1] = t.y; v[k][2] = t.z; v[k][3] = t.w;
+            v[k][4] = t2.x; v[k][5] = t2.y; v[k][6] = t2.z; v[k][7] = t2.w;
+          } else if constexpr (VEC == 4) {
             float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
             if (wi[k] != 0.f) t = *reinterpret_cast<const float4 *>(src);
             v[k][0] = t.x; v[k][1] = t.y; v[k][2] = t.z; v[k][3] = t.w;
@@ -122,9 +147,11 @@ mc_status_t launch_merge(const Params &p, int dtype, const float *o_part, const 
   if (dtype == MC_F32) {
     if (p.d == 64) return launch_t<float, 64>(p, o_part, lse_part, o, lse, stream, beside_previous);
     if (p.d == 128) return launch_t<float, 128>(p, o_part, lse_part, o, lse, stream, beside_previous);
+    if (p.d == 256) return launch_t<float, 256>(p, o_part, lse_part, o, lse, stream, beside_previous);
   } else if (dtype == MC_BF16) {
     if (p.d == 64) return launch_t<__nv_bfloat16, 64>(p, o_part, lse_part, o, lse, stream, beside_previous);
     if (p.d == 128) return launch_t<__nv_bfloat16, 128>(p, o_part, lse_part, o, lse, stream, beside_previous);
+    if (p.d == 256) return launch_t<__nv_bfloat16, 256>(p, o_part, lse_part, o, lse, stream, beside_previous);
   }
   return MC_ERR_UNSUPPORTED;
 }

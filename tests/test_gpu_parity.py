@@ -351,6 +351,49 @@ def test_bf16_head_dim_64_on_the_warp_level_tensor_path(g):
     dp.close()
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_head_dim_256(dtype):
+    """d = 256 runs on the plain-ALU kernel (the tensor-core kernels are built around 128-wide heads): ragged
+    prefixes, permuted pages, several chunks, appends (plain and rotary), an outer cascade level."""
+    from oracle import rope
+    cfg = wl.Config("d256", dtype, 2, 3, 4, 2, 256, ("loguniform", 40, 700), ("uniform", 0, 500), permute_pages=True,
+                    append_steps=3, seed=22)
+    hp = wl.make_host_problem(cfg)
+    wl.add_outer_level(hp, [0, cfg.B], [130])
+    dp = DeviceProblem.from_host(hp)
+    assert dp.geom.prefix_ctas == 0 and dp.geom.head_dim == 256
+
+    def reference(q):
+        levels = [(lv.k, lv.v, lv.group_offsets.tolist()) for lv in hp.outer]
+        levels.append((hp.k_prefix, hp.v_prefix, hp.tables.group_offsets.tolist()))
+        return orc.decode_attention_cascade(q, levels, hp.k_suffix, hp.v_suffix, cfg.scale)
+
+    for step in range(4):
+        q = wl.draw_q(cfg, step)
+        if step in (1, 2):
+            k_new, v_new = wl.draw_append(cfg, step)
+            mc.mc_kv_append(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new))
+            hp.append(k_new, v_new)
+        if step == 3:          # a rotated key: the cache must hold what the rotation's definition gives
+            k_new, v_new = wl.draw_append(cfg, step)
+            pos = [130 + int(hp.prefix_len[b // cfg.C]) + int(hp.suffix_len[b]) for b in range(cfg.B)]
+            mc.mc_kv_append_rope(dp.layout, to_device(cfg, k_new), to_device(cfg, v_new), None, None, 10000.0)
+            k_rot = np.stack([np.stack([rope.rope_rotate(k_new[b, h], pos[b], 10000.0) for h in range(cfg.Hkv)])
+                              for b in range(cfg.B)])
+            torch.cuda.synchronize()
+            s_new = hp.suffix_len.copy()
+            got = np.stack([dp.k_pool[int(hp.tables.suffix_pages[b, s_new[b] // 16]), :, s_new[b] % 16].float().cpu().numpy()
+                            for b in range(cfg.B)])
+            tol = (2.0 ** -8 if dtype == "bf16" else 2.0 ** -20) * np.abs(k_rot).max() * 2 + 1e-6
+            assert np.abs(got - k_rot).max() <= tol
+            hp.append(got.astype(np.float32), v_new)      # attention is checked on the rows the cache holds
+        o, lse = dp.decode(to_device(cfg, q))
+        torch.cuda.synchronize()
+        assert mc.mc_get_last_status(dp.layout) == mc.MC_OK
+        check_close(cfg, o, lse, *reference(q))
+    dp.close()
+
+
 def test_unequal_group_sizes():
     cfg = wl.Config("unequal", "bf16", 2, 2, 8, 2, 128, ("fixed", 0), ("fixed", (5, 40, 0, 100)), seed=4)
     hp = wl.make_host_problem(cfg, prefix_len=np.array([64, 200], dtype=np.int32))
