@@ -10,10 +10,13 @@
 //     128-row tile (re-read by every CTA from L2, evict-last), both with the 128-byte swizzle, consumed by four
 //     tcgen05.mma (M = 128, N = 256, k = 16) per row tile; four stages (three with two row tiles) keep 96-128 KB
 //     of W in flight per SM;
-//   * what bounds it is not HBM but what an SM can take in: every k-block brings 32 KB of W and 16 KB of x per row
-//     tile into shared memory, 250 MB in all for 168 MB of weights, at the 60 GB/s per SM that the copies reach
-//     (W re-tiled into contiguous 32 KB boxes streams no faster: tried).  Sharing x between SMs would lift
-//     that; on one SM the kernel runs level with the library GEMM of the same shape;
+//   * what bounds it is the bytes an SM can have on their way: a copy issued while HBM runs near its rate arrives
+//     about 3 us later (x, from L2, about half that), shared memory holds four k-blocks of 48 KB, and four k-blocks
+//     per 3 us per SM is the 5 TB/s the kernel reaches - level with the library GEMM of the same shape.  Tried and
+//     measured, none faster: W re-tiled into contiguous 32 KB boxes (the same: DRAM locality is not the limit),
+//     the x copies left out (the same: the SM's intake is not the limit), separate rings of five W boxes and two x
+//     slots (slower: two slots do not cover x's latency).  What would help is a smaller share of x per byte of W
+//     in shared memory: x shared between SMs (cluster multicast or CTA pairs) or between two W tiles;
 //   * where a CTA's share crosses from one head pair to the next, it stores the fp32 sums of the piece it has
 //     ([piece][row][feature]; piece = the CTA's ordinal among the CTAs that share the pair) and starts over; the
 //     kernel that rotates and appends adds the pieces of a pair up in that fixed order (no atomics: the result does
