@@ -128,6 +128,10 @@ CONFIGS: Dict[str, Config] = {
     # cfg4 over an e4m3 cache with per-(page, kv head) scales: half the bytes per cached token
     "cfg4_fp8": Config("cfg4_fp8", "fp8", 4, 32, 64, 8, 128, ("fixed", 4096), ("uniform", 16384, 32768),
                        permute_pages=True, append_steps=64),
+    # eight of cfg3's sixteen problems (2.3 GB): the same chunk geometry and one-row-tile prefix items at a size a
+    # profiler can replay
+    "cfg3g8": Config("cfg3g8", "bf16", 8, 16, 32, 8, 128, ("loguniform", 1024, 16384), ("uniform", 0, 8192),
+                     k_outlier_prob=0.01, k_outlier_scale=8.0),
     # one of cfg4's four prompt groups alone (3.2 GB): the same chunk geometry at a size a profiler can replay
     "cfg4g1": Config("cfg4g1", "bf16", 1, 32, 64, 8, 128, ("fixed", 4096), ("uniform", 16384, 32768),
                      permute_pages=True, append_steps=64),
